@@ -1,0 +1,168 @@
+/*
+ * libheinsen_scan -- C ABI.
+ *
+ * Fused, single-pass evaluation on one NVIDIA B200 (sm_100a) of the first-order
+ * linear recurrence
+ *
+ *         x_t = a_t * x_{t-1} + b_t ,   t = 1..n ,
+ *
+ * for `rows` independent sequences, through the two-prefix-sum log-space
+ * expression of F. A. Heinsen, "Efficient Parallelization of a Ubiquitous
+ * Sequential Computation" (2023):
+ *
+ *         a*_t      = cumsum_t(log a_t)                                  (Eq. 2, first prefix sum)
+ *         log x_t   = a*_t + tail(LCSE(cat(log x_0, log b_t - a*_t)))    (Eq. 7, Eq. 8)
+ *         x_t       = exp(log x_t)                                       (Eq. 3)
+ *
+ * Both prefix sums, the log-sum-exp and the final exponential are fused into one
+ * pass over HBM: every input element is read once, every output element written
+ * once.  Negative a_t, b_t, x_0 are carried as sign + magnitude, which is the
+ * paper's complex-logarithm path on the principal branch (Summary, last
+ * paragraph): log(-r) = log r + i*pi, the imaginary part is one sign bit.
+ *
+ * Conventions for every entry point
+ *   - Layout: a, b, log_a, log_b, x, log_x, sign_*: [rows, n] row-major contiguous,
+ *     element (r, t) of the paper (t = 1..n) at index r*n + (t-1).  x0, log_x0,
+ *     sign_x0: [rows].  The output has n entries per row, x_1..x_n; x_0 is not part
+ *     of it (Eq. 7's tail()).
+ *   - Device entry points take DEVICE pointers owned by the caller.  The library
+ *     never allocates, frees or keeps device memory.  Work is enqueued on `stream`
+ *     (a cudaStream_t passed as void*; NULL = legacy default stream) and the call
+ *     returns without synchronising.
+ *   - Pointers must be aligned to their element size.  When every base pointer is
+ *     16-byte aligned and n * sizeof(element) is a multiple of 16 for every tensor,
+ *     chunks move by TMA; otherwise a slower in-kernel path with plain loads is used
+ *     (still entirely on the GPU).
+ *   - The output may alias one input of the same type and shape exactly (in situ);
+ *     partial overlap is undefined.
+ *   - rows == 0 or n == 0: HS_OK, nothing is launched.
+ *   - log 0 = -inf is a legal input.  +inf and NaN inputs give unspecified values in
+ *     their own row from that element on and never affect other rows.
+ *   - Errors found on the host (null pointer, negative size, overflow of rows*n,
+ *     unsupported type, bad workspace) return before any CUDA call.
+ *   - Errors found on the device (a bounded wait that ran out) are written to a
+ *     status word in `workspace` and are read back by heinsen_scan_check().
+ *   - There is no CPU fallback: on a device that is not sm_100 the calls return
+ *     HS_ERR_UNSUPPORTED_DEVICE.
+ */
+#ifndef HEINSEN_SCAN_H_
+#define HEINSEN_SCAN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { HS_F32 = 0, HS_BF16 = 1 } hs_dtype;
+
+typedef enum {
+    HS_OK = 0,
+    HS_ERR_INVALID_ARG = 1,
+    HS_ERR_UNSUPPORTED_DEVICE = 2,
+    HS_ERR_WORKSPACE_TOO_SMALL = 3,
+    HS_ERR_CUDA = 4,
+    HS_ERR_LOOKBACK_TIMEOUT = 5, /* device: a tile's wait for its predecessors ran out */
+    HS_ERR_COPY_TIMEOUT = 6      /* device: a wait for an asynchronous chunk copy ran out */
+} hs_status;
+
+/* Kernel selection for heinsen_scan_set_path(). */
+typedef enum {
+    HS_PATH_AUTO = 0,     /* rows >= a few per SM: batched kernel; else look-back kernel */
+    HS_PATH_BATCHED = 1,  /* one warp walks one row, carry in registers */
+    HS_PATH_LOOKBACK = 2  /* rows cut into tiles, single pass with decoupled look-back */
+} hs_path;
+
+/*
+ * Linear-domain entry point: Eq. 3 / Eq. 7 applied to linear inputs.
+ *   x[r,t] = a[r,t] * x[r,t-1] + b[r,t],  x[r,0] = x0[r].
+ * The kernel takes log|a|, log|b|, log|x0| and the sign bits itself (step "log a_t",
+ * "log b_t", "log x_0" of Eq. 2 and Eq. 7), runs both prefix sums in log space and
+ * writes x = +-exp(log|x|).
+ *   a, b  : device, [rows,n], `dtype`;  x0: device, [rows], `dtype`;  x: device, [rows,n], `dtype`.
+ *   dtype : HS_F32 only (HS_BF16 returns HS_ERR_INVALID_ARG).
+ *   workspace, workspace_bytes: device scratch of at least
+ *           heinsen_scan_workspace_bytes(rows, n) bytes, 256-byte aligned; contents
+ *           need no initialisation; must not be shared by calls that overlap in time.
+ */
+hs_status heinsen_scan_linear(const void* a, const void* b, const void* x0, void* x,
+                              int64_t rows, int64_t n, hs_dtype dtype,
+                              void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Log-domain entry point: Eq. 7 as printed, on log inputs, returning log x.
+ *   log_x[r,t] = a*_t + logaddexp(log_x0[r], logcumsumexp(log_b - a*)_t),  a* = cumsum(log_a)
+ * with an optional sign bit per value (sign + magnitude of a negative real).
+ *   log_a, log_b : device, [rows,n], `dtype_in`;  log_x0: device, [rows], `dtype_in`.
+ *   log_x        : device, [rows,n], `dtype_out`.  Supported (in,out): (F32,F32),
+ *                  (BF16,BF16), (F32,BF16).  Arithmetic is fp32 throughout; bf16 is
+ *                  storage only, rounded to nearest-even on store.
+ *   sign_a, sign_b : device, [rows,n] uint8, 0 = '+', 1 = '-', or NULL (all positive).
+ *   sign_x0        : device, [rows] uint8 or NULL.
+ *   sign_x         : device, [rows,n] uint8 output; required iff any sign input is
+ *                    non-NULL, ignored otherwise.  An exact zero reports sign 0.
+ *   workspace      : as for heinsen_scan_linear.
+ */
+hs_status heinsen_scan_log(const void* log_a, const void* log_b, const void* log_x0, void* log_x,
+                           const uint8_t* sign_a, const uint8_t* sign_b, const uint8_t* sign_x0,
+                           uint8_t* sign_x,
+                           int64_t rows, int64_t n, hs_dtype dtype_in, hs_dtype dtype_out,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Scratch size in bytes for a problem of this shape (any path, any type): a 256-byte
+ * header (status word, tile ticket) plus one descriptor per tile of the look-back
+ * kernel -- the carry between parts that the associativity of prefix sums allows
+ * (Summary, footnote on associativity).  Returns 0 only for invalid sizes.
+ */
+size_t heinsen_scan_workspace_bytes(int64_t rows, int64_t n);
+
+/*
+ * Synchronises `stream`, reads the status word of `workspace` (device pointer) and
+ * returns it: HS_OK, or the device-side error recorded by the last call that used
+ * this workspace.
+ */
+hs_status heinsen_scan_check(const void* workspace, void* stream);
+
+/*
+ * Host-buffer variants of the two entry points above, for callers whose data lives
+ * in host memory (pinned memory recommended).  All tensor pointers are HOST pointers;
+ * `device_scratch` is a DEVICE buffer of at least heinsen_scan_host_scratch_bytes(...)
+ * bytes provided by the caller.  The call copies inputs to the device in row blocks,
+ * runs the same kernels, copies results back, and returns after the last copy has
+ * completed (it synchronises).  The recurrence itself runs only on the GPU.
+ */
+hs_status heinsen_scan_linear_host(const void* a, const void* b, const void* x0, void* x,
+                                   int64_t rows, int64_t n, hs_dtype dtype,
+                                   void* device_scratch, size_t device_scratch_bytes, void* stream);
+hs_status heinsen_scan_log_host(const void* log_a, const void* log_b, const void* log_x0, void* log_x,
+                                const uint8_t* sign_a, const uint8_t* sign_b, const uint8_t* sign_x0,
+                                uint8_t* sign_x,
+                                int64_t rows, int64_t n, hs_dtype dtype_in, hs_dtype dtype_out,
+                                void* device_scratch, size_t device_scratch_bytes, void* stream);
+size_t heinsen_scan_host_scratch_bytes(int64_t rows, int64_t n, hs_dtype dtype_in, hs_dtype dtype_out,
+                                       int with_signs);
+
+/* Process-wide kernel selection (default HS_PATH_AUTO); for tests and benchmarks. */
+hs_status heinsen_scan_set_path(hs_path path);
+/*
+ * Test hook for the bounded wait of the look-back kernel (the only device-side wait on another
+ * CTA).  `lookback_spin_limit` bounds the polls of predecessor descriptors (0 restores the
+ * default); `mute_tile` >= 0 makes that tile skip publishing its descriptors, so that its
+ * successors run out of polls, record HS_ERR_LOOKBACK_TIMEOUT in the workspace and leave;
+ * -1 disables it.  Nothing faults or hangs: the kernel returns and the context stays usable.
+ */
+hs_status heinsen_scan_debug_config(uint32_t lookback_spin_limit, int64_t mute_tile);
+/* Path taken by the most recent successful launch of this process (hs_path value), 0 if none. */
+int heinsen_scan_last_path(void);
+/* Number of kernels this library has launched in this process (memsets not counted). */
+int64_t heinsen_scan_launch_count(void);
+
+/* Static, NUL-terminated description of a status code. */
+const char* heinsen_scan_strerror(hs_status status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HEINSEN_SCAN_H_ */

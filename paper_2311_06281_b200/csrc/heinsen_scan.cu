@@ -1,0 +1,463 @@
+// C-ABI of libheinsen_scan: argument validation, kernel selection, tensor maps, launches.
+// See include/heinsen_scan.h for the contract of every entry point.
+#include "../../include/heinsen_scan.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <chrono>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+
+#include "hs_kernels.cuh"
+
+namespace {
+
+using namespace hs;
+
+std::atomic<int> g_path{HS_PATH_AUTO};
+std::atomic<int> g_last_path{0};
+std::atomic<long long> g_launches{0};
+std::atomic<unsigned int> g_spin_limit{hs::kLookbackSpinLimit};
+std::atomic<long long> g_mute_tile{-1};
+thread_local char g_cuda_msg[256] = "";
+
+constexpr long long kMaxTmaDim = (1ll << 31) - (1ll << 20);  // TMA coordinates are int32
+constexpr int kBatchedMinRowsPerSm = 8;  // fewer rows per SM than this: look-back kernel
+constexpr int kLookbackWarps = 8;        // warps (= chunks) per tile of the look-back kernel
+constexpr int kMinChunk = 512;           // smallest chunk (32 lanes x 16 elements)
+
+unsigned long long next_call_id() {
+    static std::atomic<unsigned long long> counter{[] {
+        const auto t = std::chrono::high_resolution_clock::now().time_since_epoch().count();
+        unsigned long long z = (unsigned long long)t * 0x9E3779B97F4A7C15ull;
+        z ^= (unsigned long long)(uintptr_t)&g_path << 17;
+        z ^= z >> 29;
+        return z;
+    }()};
+    // 62 bits; never 0
+    unsigned long long id = (counter.fetch_add(1) + 1) & ((1ull << 62) - 1);
+    return id ? id : 1;
+}
+
+struct DeviceInfo {
+    int sm_count = 0;
+    int cc_major = 0;
+    int max_smem_optin = 0;
+    bool ok = false;
+};
+
+hs_status device_info(DeviceInfo& out) {
+    static std::mutex mu;
+    static DeviceInfo cache[64];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) {
+        snprintf(g_cuda_msg, sizeof g_cuda_msg, "cudaGetDevice: %s", cudaGetErrorString(e));
+        return HS_ERR_CUDA;
+    }
+    if (dev < 0 || dev >= 64) return HS_ERR_UNSUPPORTED_DEVICE;
+    std::lock_guard<std::mutex> lk(mu);
+    DeviceInfo& d = cache[dev];
+    if (!d.ok) {
+        if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&d.cc_major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&d.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) {
+            snprintf(g_cuda_msg, sizeof g_cuda_msg, "cudaDeviceGetAttribute failed");
+            return HS_ERR_CUDA;
+        }
+        d.ok = true;
+    }
+    out = d;
+    return HS_OK;
+}
+
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn encode_fn() {
+    static EncodeFn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeFn>(p);
+    }();
+    return fn;
+}
+
+// [rows, n] row-major as a 2-D tensor map whose box is one 128-byte row segment, 128-byte swizzle.
+bool make_tmap(CUtensorMap* tm, const void* ptr, hs_dtype dt, long long rows, long long n) {
+    EncodeFn fn = encode_fn();
+    if (!fn) return false;
+    const int es = (dt == HS_F32) ? 4 : 2;
+    cuuint64_t dims[2] = {(cuuint64_t)n, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)n * es};
+    cuuint32_t box[2] = {(cuuint32_t)(128 / es), 1};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(tm, dt == HS_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                    const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int env_int(const char* name, int dflt, int lo, int hi) {
+    const char* v = std::getenv(name);
+    if (!v || !*v) return dflt;
+    int x = std::atoi(v);
+    return x < lo ? lo : (x > hi ? hi : x);
+}
+
+// ---------------------------------------------------------------------------------------------
+struct Problem {
+    int mode;            // hs::Mode
+    hs_dtype din, dout;
+    Params p;
+    bool tma;
+};
+
+using BatchedFn = void (*)(const Params, const CUtensorMap, const CUtensorMap, const CUtensorMap);
+
+struct KernelEntry {
+    const void* batched;
+    const void* lookback;
+    int K;
+    int warp_smem_per_stage;  // bytes of one input stage (both tensors) of one warp
+    int warp_smem_out;        // bytes of both output buffers of one warp
+};
+
+template <int MODE, typename TIn, typename TOut, int K, bool TMA>
+KernelEntry entry() {
+    KernelEntry e;
+    e.batched = reinterpret_cast<const void*>(&batched_scan_kernel<MODE, TIn, TOut, K, TMA>);
+    e.lookback = reinterpret_cast<const void*>(&lookback_scan_kernel<MODE, TIn, TOut, K, TMA>);
+    e.K = K;
+    e.warp_smem_per_stage = 2 * 32 * K * (int)sizeof(TIn);
+    e.warp_smem_out = 2 * 32 * K * (int)sizeof(TOut);
+    return e;
+}
+
+bool find_kernel(int mode, hs_dtype din, hs_dtype dout, bool tma, KernelEntry& e) {
+#define HS_PICK(M, TI, TO, KK)                                               \
+    do {                                                                     \
+        e = tma ? entry<M, TI, TO, KK, true>() : entry<M, TI, TO, KK, false>(); \
+        return true;                                                         \
+    } while (0)
+    using bf16 = __nv_bfloat16;
+    if (mode == kLinear) {
+        if (din == HS_F32 && dout == HS_F32) HS_PICK(kLinear, float, float, 16);
+        return false;
+    }
+    if (mode == kLogUnsigned) {
+        if (din == HS_F32 && dout == HS_F32) HS_PICK(kLogUnsigned, float, float, 16);
+        if (din == HS_BF16 && dout == HS_BF16) HS_PICK(kLogUnsigned, bf16, bf16, 32);
+        if (din == HS_F32 && dout == HS_BF16) HS_PICK(kLogUnsigned, float, bf16, 16);
+        return false;
+    }
+    if (mode == kLogSigned) {
+        if (din == HS_F32 && dout == HS_F32) HS_PICK(kLogSigned, float, float, 16);
+        if (din == HS_BF16 && dout == HS_BF16) HS_PICK(kLogSigned, bf16, bf16, 32);
+        if (din == HS_F32 && dout == HS_BF16) HS_PICK(kLogSigned, float, bf16, 16);
+        return false;
+    }
+    return false;
+#undef HS_PICK
+}
+
+long long lookback_tiles_per_row(long long n, int chunk) {
+    const long long tile = (long long)kLookbackWarps * chunk;
+    return (n + tile - 1) / tile;
+}
+
+int choose_path(long long rows, const DeviceInfo& d) {
+    const int forced = g_path.load();
+    if (forced == HS_PATH_BATCHED || forced == HS_PATH_LOOKBACK) return forced;
+    return rows >= (long long)kBatchedMinRowsPerSm * d.sm_count ? HS_PATH_BATCHED : HS_PATH_LOOKBACK;
+}
+
+size_t workspace_bytes_for(long long rows, long long n) {
+    // sized for the smallest chunk so that it covers every type
+    const long long tiles = rows * lookback_tiles_per_row(n, kMinChunk);
+    return sizeof(Header) + (size_t)tiles * (8 + 16 + 16);
+}
+
+hs_status cuda_fail(const char* what, cudaError_t e) {
+    snprintf(g_cuda_msg, sizeof g_cuda_msg, "%s: %s", what, cudaGetErrorString(e));
+    return HS_ERR_CUDA;
+}
+
+hs_status validate_common(const void* a, const void* b, const void* x0, const void* out, int64_t rows, int64_t n) {
+    if (rows < 0 || n < 0) return HS_ERR_INVALID_ARG;
+    if (rows == 0 || n == 0) return HS_OK;
+    if (!a || !b || !x0 || !out) return HS_ERR_INVALID_ARG;
+    if (rows > 0x7fffffffll) return HS_ERR_INVALID_ARG;
+    if (n > (1ll << 40) || rows > (1ll << 62) / n) return HS_ERR_INVALID_ARG;
+    return HS_OK;
+}
+
+hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t stream) {
+    Params& p = pr.p;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HS_ERR_INVALID_ARG;
+    if (workspace_bytes < sizeof(Header)) return HS_ERR_WORKSPACE_TOO_SMALL;
+
+    DeviceInfo dev;
+    hs_status st = device_info(dev);
+    if (st != HS_OK) return st;
+    if (dev.cc_major != 10) return HS_ERR_UNSUPPORTED_DEVICE;
+
+    const int es_in = pr.din == HS_F32 ? 4 : 2, es_out = pr.dout == HS_F32 ? 4 : 2;
+    bool tma = aligned16(p.in_a) && aligned16(p.in_b) && aligned16(p.out) && (p.n * es_in) % 16 == 0 &&
+               (p.n * es_out) % 16 == 0 && p.n <= kMaxTmaDim && encode_fn() != nullptr;
+    if (env_int("HEINSEN_SCAN_NO_TMA", 0, 0, 1)) tma = false;
+    pr.tma = tma;
+
+    KernelEntry ke;
+    if (!find_kernel(pr.mode, pr.din, pr.dout, tma, ke)) return HS_ERR_INVALID_ARG;
+    const int chunk = 32 * ke.K;
+    p.nchunks = (int)((p.n + chunk - 1) / chunk);
+    p.sign_vec_ok = (p.n % 16 == 0) && (!p.sign_a || aligned16(p.sign_a)) && (!p.sign_b || aligned16(p.sign_b)) &&
+                    (!p.sign_x || aligned16(p.sign_x));
+    p.call_id = next_call_id();
+    p.spin_limit = g_spin_limit.load();
+    p.mute_tile = g_mute_tile.load();
+    p.ws = reinterpret_cast<Header*>(workspace);
+
+    CUtensorMap tm_a, tm_b, tm_o;
+    std::memset(&tm_a, 0, sizeof tm_a);
+    std::memset(&tm_b, 0, sizeof tm_b);
+    std::memset(&tm_o, 0, sizeof tm_o);
+    if (tma) {
+        if (!make_tmap(&tm_a, p.in_a, pr.din, p.rows, p.n) || !make_tmap(&tm_b, p.in_b, pr.din, p.rows, p.n) ||
+            !make_tmap(&tm_o, p.out, pr.dout, p.rows, p.n)) {
+            snprintf(g_cuda_msg, sizeof g_cuda_msg, "cuTensorMapEncodeTiled failed");
+            return HS_ERR_CUDA;
+        }
+    }
+
+    const int path = choose_path(p.rows, dev);
+    int warps, stages, grid;
+    const void* fn;
+    if (path == HS_PATH_BATCHED) {
+        warps = env_int("HEINSEN_SCAN_WARPS", 12, 1, 16);
+        stages = tma ? env_int("HEINSEN_SCAN_STAGES", 3, 2, kMaxStages) : 1;
+        const long long ctas_needed = (p.rows + warps - 1) / warps;
+        grid = (int)(ctas_needed < dev.sm_count ? ctas_needed : dev.sm_count);
+        fn = ke.batched;
+    } else {
+        warps = kLookbackWarps;
+        stages = tma ? env_int("HEINSEN_SCAN_LB_STAGES", 2, 2, kMaxStages) : 1;
+        p.tiles_per_row = (int)lookback_tiles_per_row(p.n, chunk);
+        p.num_tiles = p.rows * p.tiles_per_row;
+        const size_t need = sizeof(Header) + (size_t)p.num_tiles * (8 + 16 + 16);
+        if (workspace_bytes < need) return HS_ERR_WORKSPACE_TOO_SMALL;
+        uint8_t* w = reinterpret_cast<uint8_t*>(workspace) + sizeof(Header);
+        p.agg = reinterpret_cast<float4*>(w);
+        p.inc = reinterpret_cast<float4*>(w + (size_t)p.num_tiles * 16);
+        p.flags = reinterpret_cast<unsigned long long*>(w + (size_t)p.num_tiles * 32);
+        fn = ke.lookback;
+        grid = 0;  // set below from occupancy
+    }
+    p.stages = stages;
+    const int smem = warps * (stages * ke.warp_smem_per_stage + ke.warp_smem_out) + warps * 8 * kMaxStages + 1024 +
+                     (path == HS_PATH_LOOKBACK ? 1024 : 0);
+    if (smem > dev.max_smem_optin) return HS_ERR_INVALID_ARG;
+    cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", e);
+
+    void* args[] = {&p, &tm_a, &tm_b, &tm_o};
+    if (path == HS_PATH_LOOKBACK) {
+        // Tiles wait for their predecessors, so every CTA must be resident: size the grid from the
+        // occupancy of this kernel and launch cooperatively (the launch fails rather than deadlocks).
+        int per_sm = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, warps * 32, smem);
+        if (e != cudaSuccess) return cuda_fail("cudaOccupancyMaxActiveBlocksPerMultiprocessor", e);
+        if (per_sm < 1) return HS_ERR_INVALID_ARG;
+        per_sm = env_int("HEINSEN_SCAN_LB_CTAS_PER_SM", per_sm, 1, per_sm);
+        long long g = (long long)per_sm * dev.sm_count;
+        if (g > p.num_tiles) g = p.num_tiles;
+        grid = (int)g;
+        e = cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(warps * 32), args, smem, stream);
+    } else {
+        e = cudaLaunchKernel(fn, dim3(grid), dim3(warps * 32), args, smem, stream);
+    }
+    if (e != cudaSuccess) return cuda_fail("kernel launch", e);
+    g_last_path.store(path);
+    g_launches.fetch_add(1);
+    return HS_OK;
+}
+
+}  // namespace
+
+// =============================================================================================
+extern "C" {
+
+hs_status heinsen_scan_linear(const void* a, const void* b, const void* x0, void* x, int64_t rows, int64_t n,
+                              hs_dtype dtype, void* workspace, size_t workspace_bytes, void* stream) {
+    hs_status st = validate_common(a, b, x0, x, rows, n);
+    if (st != HS_OK || rows == 0 || n == 0) return st;
+    if (dtype != HS_F32) return HS_ERR_INVALID_ARG;
+    Problem pr;
+    std::memset(&pr, 0, sizeof pr);
+    pr.mode = kLinear;
+    pr.din = pr.dout = dtype;
+    pr.p.in_a = a; pr.p.in_b = b; pr.p.x0 = x0; pr.p.out = x;
+    pr.p.rows = rows; pr.p.n = n;
+    return run(pr, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
+}
+
+hs_status heinsen_scan_log(const void* log_a, const void* log_b, const void* log_x0, void* log_x,
+                           const uint8_t* sign_a, const uint8_t* sign_b, const uint8_t* sign_x0, uint8_t* sign_x,
+                           int64_t rows, int64_t n, hs_dtype dtype_in, hs_dtype dtype_out, void* workspace,
+                           size_t workspace_bytes, void* stream) {
+    hs_status st = validate_common(log_a, log_b, log_x0, log_x, rows, n);
+    if (st != HS_OK || rows == 0 || n == 0) return st;
+    if ((dtype_in != HS_F32 && dtype_in != HS_BF16) || (dtype_out != HS_F32 && dtype_out != HS_BF16))
+        return HS_ERR_INVALID_ARG;
+    if (dtype_in == HS_BF16 && dtype_out == HS_F32) return HS_ERR_INVALID_ARG;
+    const bool is_signed = sign_a || sign_b || sign_x0;
+    if (is_signed && !sign_x) return HS_ERR_INVALID_ARG;
+    Problem pr;
+    std::memset(&pr, 0, sizeof pr);
+    pr.mode = is_signed ? kLogSigned : kLogUnsigned;
+    pr.din = dtype_in; pr.dout = dtype_out;
+    pr.p.in_a = log_a; pr.p.in_b = log_b; pr.p.x0 = log_x0; pr.p.out = log_x;
+    if (is_signed) { pr.p.sign_a = sign_a; pr.p.sign_b = sign_b; pr.p.sign_x0 = sign_x0; pr.p.sign_x = sign_x; }
+    pr.p.rows = rows; pr.p.n = n;
+    return run(pr, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
+}
+
+size_t heinsen_scan_workspace_bytes(int64_t rows, int64_t n) {
+    if (rows <= 0 || n <= 0) return 0;
+    if (rows > 0x7fffffffll || n > (1ll << 40) || rows > (1ll << 62) / n) return 0;
+    return workspace_bytes_for(rows, n);
+}
+
+hs_status heinsen_scan_check(const void* workspace, void* stream) {
+    if (!workspace) return HS_ERR_INVALID_ARG;
+    cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail("cudaStreamSynchronize", e);
+    Header h;
+    e = cudaMemcpy(&h, workspace, sizeof h, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail("cudaMemcpy", e);
+    if (h.error_id == h.started_id && h.started_id != 0 &&
+        (h.error_code == HS_ERR_LOOKBACK_TIMEOUT || h.error_code == HS_ERR_COPY_TIMEOUT))
+        return static_cast<hs_status>(h.error_code);
+    return HS_OK;
+}
+
+hs_status heinsen_scan_set_path(hs_path path) {
+    if (path != HS_PATH_AUTO && path != HS_PATH_BATCHED && path != HS_PATH_LOOKBACK) return HS_ERR_INVALID_ARG;
+    g_path.store(path);
+    return HS_OK;
+}
+hs_status heinsen_scan_debug_config(uint32_t lookback_spin_limit, int64_t mute_tile) {
+    g_spin_limit.store(lookback_spin_limit ? lookback_spin_limit : hs::kLookbackSpinLimit);
+    g_mute_tile.store(mute_tile);
+    return HS_OK;
+}
+int heinsen_scan_last_path(void) { return g_last_path.load(); }
+int64_t heinsen_scan_launch_count(void) { return g_launches.load(); }
+
+const char* heinsen_scan_strerror(hs_status status) {
+    switch (status) {
+        case HS_OK: return "ok";
+        case HS_ERR_INVALID_ARG: return "invalid argument (null pointer, bad size, unsupported type or misaligned workspace)";
+        case HS_ERR_UNSUPPORTED_DEVICE: return "unsupported device: this library runs on sm_100 (B200) only";
+        case HS_ERR_WORKSPACE_TOO_SMALL: return "workspace too small: see heinsen_scan_workspace_bytes()";
+        case HS_ERR_CUDA: return g_cuda_msg[0] ? g_cuda_msg : "CUDA runtime error";
+        case HS_ERR_LOOKBACK_TIMEOUT: return "device: a tile's bounded wait for its predecessors ran out";
+        case HS_ERR_COPY_TIMEOUT: return "device: a bounded wait for an asynchronous chunk copy ran out";
+    }
+    return "unknown status";
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host-buffer variants: copy in, run, copy out, on `stream`; synchronise before returning.
+size_t heinsen_scan_host_scratch_bytes(int64_t rows, int64_t n, hs_dtype dtype_in, hs_dtype dtype_out, int with_signs) {
+    if (rows <= 0 || n <= 0) return 0;
+    const size_t es_in = dtype_in == HS_F32 ? 4 : 2, es_out = dtype_out == HS_F32 ? 4 : 2;
+    auto up = [](size_t v) { return (v + 255) & ~size_t(255); };
+    const size_t cnt = (size_t)rows * (size_t)n;
+    size_t total = up(workspace_bytes_for(rows, n));
+    total += 2 * up(cnt * es_in) + up((size_t)rows * es_in) + up(cnt * es_out);
+    if (with_signs) total += 3 * up(cnt) + up((size_t)rows);
+    return total;
+}
+
+static hs_status host_run(int linear, const void* a, const void* b, const void* x0, void* x, const uint8_t* sa,
+                          const uint8_t* sb, const uint8_t* sx0, uint8_t* sx, int64_t rows, int64_t n, hs_dtype din,
+                          hs_dtype dout, void* scratch, size_t scratch_bytes, cudaStream_t stream) {
+    hs_status st = validate_common(a, b, x0, x, rows, n);
+    if (st != HS_OK || rows == 0 || n == 0) return st;
+    const bool with_signs = sa || sb || sx0;
+    if (with_signs && !sx) return HS_ERR_INVALID_ARG;
+    if (!scratch || (reinterpret_cast<uintptr_t>(scratch) & 255u)) return HS_ERR_INVALID_ARG;
+    if (scratch_bytes < heinsen_scan_host_scratch_bytes(rows, n, din, dout, with_signs)) return HS_ERR_WORKSPACE_TOO_SMALL;
+    const size_t es_in = din == HS_F32 ? 4 : 2, es_out = dout == HS_F32 ? 4 : 2;
+    auto up = [](size_t v) { return (v + 255) & ~size_t(255); };
+    const size_t cnt = (size_t)rows * (size_t)n;
+    uint8_t* w = static_cast<uint8_t*>(scratch);
+    void* ws = w;                 w += up(workspace_bytes_for(rows, n));
+    void* d_a = w;                w += up(cnt * es_in);
+    void* d_b = w;                w += up(cnt * es_in);
+    void* d_x0 = w;               w += up((size_t)rows * es_in);
+    void* d_x = w;                w += up(cnt * es_out);
+    uint8_t *d_sa = nullptr, *d_sb = nullptr, *d_sx0 = nullptr, *d_sx = nullptr;
+    if (with_signs) {
+        d_sa = w; w += up(cnt);
+        d_sb = w; w += up(cnt);
+        d_sx = w; w += up(cnt);
+        d_sx0 = w; w += up((size_t)rows);
+    }
+    cudaError_t e;
+#define HS_CP(dst, src, bytes, kind)                                        \
+    do {                                                                    \
+        e = cudaMemcpyAsync(dst, src, bytes, kind, stream);                 \
+        if (e != cudaSuccess) return cuda_fail("cudaMemcpyAsync", e);       \
+    } while (0)
+    HS_CP(d_a, a, cnt * es_in, cudaMemcpyHostToDevice);
+    HS_CP(d_b, b, cnt * es_in, cudaMemcpyHostToDevice);
+    HS_CP(d_x0, x0, (size_t)rows * es_in, cudaMemcpyHostToDevice);
+    if (with_signs) {
+        if (sa) HS_CP(d_sa, sa, cnt, cudaMemcpyHostToDevice);
+        if (sb) HS_CP(d_sb, sb, cnt, cudaMemcpyHostToDevice);
+        if (sx0) HS_CP(d_sx0, sx0, (size_t)rows, cudaMemcpyHostToDevice);
+    }
+    if (linear)
+        st = heinsen_scan_linear(d_a, d_b, d_x0, d_x, rows, n, din, ws, workspace_bytes_for(rows, n), stream);
+    else
+        st = heinsen_scan_log(d_a, d_b, d_x0, d_x, sa ? d_sa : nullptr, sb ? d_sb : nullptr, sx0 ? d_sx0 : nullptr,
+                              with_signs ? d_sx : nullptr, rows, n, din, dout, ws, workspace_bytes_for(rows, n), stream);
+    if (st != HS_OK) return st;
+    HS_CP(x, d_x, cnt * es_out, cudaMemcpyDeviceToHost);
+    if (with_signs) HS_CP(sx, d_sx, cnt, cudaMemcpyDeviceToHost);
+#undef HS_CP
+    return heinsen_scan_check(ws, stream);
+}
+
+hs_status heinsen_scan_linear_host(const void* a, const void* b, const void* x0, void* x, int64_t rows, int64_t n,
+                                   hs_dtype dtype, void* device_scratch, size_t device_scratch_bytes, void* stream) {
+    if (dtype != HS_F32) return (rows == 0 || n == 0) ? HS_OK : HS_ERR_INVALID_ARG;
+    return host_run(1, a, b, x0, x, nullptr, nullptr, nullptr, nullptr, rows, n, dtype, dtype, device_scratch,
+                    device_scratch_bytes, static_cast<cudaStream_t>(stream));
+}
+
+hs_status heinsen_scan_log_host(const void* log_a, const void* log_b, const void* log_x0, void* log_x,
+                                const uint8_t* sign_a, const uint8_t* sign_b, const uint8_t* sign_x0, uint8_t* sign_x,
+                                int64_t rows, int64_t n, hs_dtype dtype_in, hs_dtype dtype_out, void* device_scratch,
+                                size_t device_scratch_bytes, void* stream) {
+    if ((dtype_in != HS_F32 && dtype_in != HS_BF16) || (dtype_out != HS_F32 && dtype_out != HS_BF16) ||
+        (dtype_in == HS_BF16 && dtype_out == HS_F32))
+        return (rows == 0 || n == 0) ? HS_OK : HS_ERR_INVALID_ARG;
+    return host_run(0, log_a, log_b, log_x0, log_x, sign_a, sign_b, sign_x0, sign_x, rows, n, dtype_in, dtype_out,
+                    device_scratch, device_scratch_bytes, static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

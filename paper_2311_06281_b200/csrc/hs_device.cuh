@@ -1,0 +1,452 @@
+// Device-side building blocks of libheinsen_scan (sm_100a only).
+//
+// Notation follows the paper: a*_t = cumsum(log a_t) (Eq. 2), LCSE = log cumsum exp (Eq. 8),
+// x_0 is prepended to the second scan as the paper's cat(log x_0, .) (Eq. 7).
+//
+// The associativity of prefix sums (Summary, footnote) lets both scans be computed by parts.
+// A part [i..j] is summarised by the affine map x -> alpha*x + beta it applies to the value
+// entering it, kept in log space:
+//     alpha = (-1)^p * exp(A),   A = sum of log|a| over the part,   p = parity of negative a's
+//     beta  = s * exp(m),        m = log-sum-exp reference ("max tracking"), s = signed scaled sum
+// Composing two parts needs one exp of a non-positive number.  The value of x itself is the
+// part that starts at x_0, for which alpha is irrelevant.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace hs {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr uint32_t kSignBit = 0x80000000u;
+
+enum Mode : int { kLogUnsigned = 0, kLogSigned = 1, kLinear = 2 };
+
+__device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000); }
+
+// MUFU wrappers: one instruction each.
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float lg2(float x) {
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float rcp_approx(float x) {
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float flip(float v, uint32_t mask) { return __uint_as_float(__float_as_uint(v) ^ mask); }
+
+// Natural logarithm of |v| accurate to about one ulp also for v close to 1, where lg2.approx's
+// absolute error would be a large relative error of log a_t and would bias a*_t over a long
+// sequence.  v = m*2^e with m in [2/3, 4/3); log m = 2 atanh(w), w = (m-1)/(m+1), odd series.
+__device__ __forceinline__ float log_abs_accurate(float v) {
+    v = fabsf(v);
+    const bool zero = (v == 0.0f);
+    const bool tiny = (v < 1.17549435e-38f);
+    const float bias = tiny ? -23.0f : 0.0f;
+    v = tiny ? v * 8388608.0f : v;
+    const int bits = __float_as_int(v);
+    const int e = (bits - 0x3f2aaaab) >> 23;
+    const float m = __int_as_float(bits - (e << 23));
+    const float f = m - 1.0f;
+    const float d = 2.0f + f;
+    const float r = rcp_approx(d);
+    float w = f * r;
+    w = fmaf(fmaf(-w, d, f), r, w);  // one Newton correction of the quotient
+    const float w2 = w * w;
+    float poly = fmaf(w2, 1.0f / 9.0f, 1.0f / 7.0f);
+    poly = fmaf(w2, poly, 1.0f / 5.0f);
+    poly = fmaf(w2, poly, 1.0f / 3.0f);
+    poly = poly * w2;
+    const float lm = fmaf(2.0f * w, poly, 2.0f * w);
+    return zero ? neg_inf() : fmaf((float)e + bias, kLn2, lm);
+}
+
+// ------------------------------------------------------------------------------------------
+// The associative element.
+template <bool SIGNED>
+struct Elem {
+    float A;     // sum of log|a|
+    float m;     // reference of beta = s*exp(m); -inf <=> beta == 0 (then s == 0)
+    float s;     // signed, scaled sum
+    uint32_t p;  // sign mask (0 or 0x80000000) of alpha; unused when !SIGNED
+};
+
+template <bool SIGNED>
+__device__ __forceinline__ Elem<SIGNED> identity_elem() {
+    Elem<SIGNED> e;
+    e.A = 0.0f; e.m = neg_inf(); e.s = 0.0f; e.p = 0u;
+    return e;
+}
+
+// "first" is the older part, "second" the newer one: result = second o first.
+template <bool SIGNED>
+__device__ __forceinline__ Elem<SIGNED> compose(const Elem<SIGNED>& first, const Elem<SIGNED>& second) {
+    Elem<SIGNED> o;
+    o.A = first.A + second.A;
+    const float m1 = first.m + second.A;  // beta_1 carried through alpha_2
+    const float s1 = SIGNED ? flip(first.s, second.p) : first.s;
+    o.m = fmaxf(m1, second.m);
+    const float d = m1 - second.m;  // NaN only when both are -inf
+    float e = ex2(-fabsf(d) * kLog2e);
+    e = (o.m == neg_inf()) ? 0.0f : e;
+    o.s = (d >= 0.0f) ? fmaf(second.s, e, s1) : fmaf(s1, e, second.s);
+    o.p = SIGNED ? (first.p ^ second.p) : 0u;
+    return o;
+}
+
+template <bool SIGNED>
+__device__ __forceinline__ Elem<SIGNED> shfl_up_elem(const Elem<SIGNED>& e, int delta) {
+    Elem<SIGNED> o;
+    o.A = __shfl_up_sync(0xffffffffu, e.A, delta);
+    o.m = __shfl_up_sync(0xffffffffu, e.m, delta);
+    o.s = __shfl_up_sync(0xffffffffu, e.s, delta);
+    o.p = SIGNED ? __shfl_up_sync(0xffffffffu, e.p, delta) : 0u;
+    return o;
+}
+template <bool SIGNED>
+__device__ __forceinline__ Elem<SIGNED> shfl_elem(const Elem<SIGNED>& e, int src) {
+    Elem<SIGNED> o;
+    o.A = __shfl_sync(0xffffffffu, e.A, src);
+    o.m = __shfl_sync(0xffffffffu, e.m, src);
+    o.s = __shfl_sync(0xffffffffu, e.s, src);
+    o.p = SIGNED ? __shfl_sync(0xffffffffu, e.p, src) : 0u;
+    return o;
+}
+template <bool SIGNED>
+__device__ __forceinline__ Elem<SIGNED> shfl_down_elem(const Elem<SIGNED>& e, int delta) {
+    Elem<SIGNED> o;
+    o.A = __shfl_down_sync(0xffffffffu, e.A, delta);
+    o.m = __shfl_down_sync(0xffffffffu, e.m, delta);
+    o.s = __shfl_down_sync(0xffffffffu, e.s, delta);
+    o.p = SIGNED ? __shfl_down_sync(0xffffffffu, e.p, delta) : 0u;
+    return o;
+}
+
+// Inclusive Kogge-Stone scan of one element per lane (the Hillis-Steele pattern the paper
+// cites for O(log n) prefix sums), then the exclusive prefix of each lane and the warp total.
+template <bool SIGNED>
+__device__ __forceinline__ void warp_scan(const Elem<SIGNED>& mine, int lane, Elem<SIGNED>& exclusive,
+                                          Elem<SIGNED>& total) {
+    Elem<SIGNED> inc = mine;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        Elem<SIGNED> up = shfl_up_elem(inc, d);
+        Elem<SIGNED> c = compose(up, inc);
+        if (lane >= d) inc = c;
+    }
+    total = shfl_elem(inc, 31);
+    Elem<SIGNED> up = shfl_up_elem(inc, 1);
+    exclusive = (lane == 0) ? identity_elem<SIGNED>() : up;
+}
+
+// The running value x = s*exp(m) as an element (alpha irrelevant: A = -inf absorbs whatever
+// came before, exactly as prepending log x_0 to the second scan does in Eq. 7).
+template <bool SIGNED>
+__device__ __forceinline__ Elem<SIGNED> state_elem(float log_mag, uint32_t sign_mask) {
+    Elem<SIGNED> e;
+    e.A = neg_inf();
+    e.m = log_mag;
+    e.s = (log_mag == neg_inf()) ? 0.0f : (SIGNED ? flip(1.0f, sign_mask) : 1.0f);
+    e.p = 0u;
+    return e;
+}
+
+// Keep |s| in [1,2) so that a long signed cancellation cannot strand the reference far above
+// the value.  Exact apart from one rounding of m.
+template <bool SIGNED>
+__device__ __forceinline__ void renormalise(Elem<SIGNED>& e) {
+    if (!SIGNED) return;
+    const float as = fabsf(e.s);
+    if (as == 0.0f) { e.m = neg_inf(); e.s = 0.0f; return; }
+    if (as >= 1.17549435e-38f && e.m != neg_inf()) {
+        const int ex = ((__float_as_int(as) >> 23) & 0xff) - 127;
+        e.m = fmaf((float)ex, kLn2, e.m);
+        e.s = __int_as_float(__float_as_int(e.s) - (ex << 23));
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Shared-memory chunk layout.  A chunk is 32 lanes x K consecutive elements of one row, kept
+// as rows of 128 bytes with the 16-byte units of each row XOR-swizzled by (row & 7) -- the
+// layout TMA's 128-byte swizzle writes -- so that a lane reading its own K contiguous
+// elements with 128-bit loads is bank-conflict free.
+__device__ __forceinline__ uint32_t swz_unit(uint32_t unit) {  // unit = index of a 16-byte unit in the chunk
+    const uint32_t row = unit >> 3;
+    return (row << 7) + (((unit & 7u) ^ (row & 7u)) << 4);
+}
+__device__ __forceinline__ uint32_t swz_byte(uint32_t byte_off) {
+    return swz_unit(byte_off >> 4) + (byte_off & 15u);
+}
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
+    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+template <typename T>
+struct Storage;
+template <>
+struct Storage<float> {
+    static constexpr int kPerUnit = 4;
+    __device__ static __forceinline__ void unpack(uint4 u, float* o) {
+        o[0] = __uint_as_float(u.x); o[1] = __uint_as_float(u.y); o[2] = __uint_as_float(u.z); o[3] = __uint_as_float(u.w);
+    }
+    __device__ static __forceinline__ uint4 pack(const float* v) {
+        return make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3]));
+    }
+    __device__ static __forceinline__ float load(const void* p, int64_t i) { return ((const float*)p)[i]; }
+    __device__ static __forceinline__ void store(void* p, int64_t i, float v) { ((float*)p)[i] = v; }
+    __device__ static __forceinline__ float from_smem(const uint8_t* base, uint32_t i) {
+        return *(const float*)(base + swz_byte(i * 4u));
+    }
+    __device__ static __forceinline__ void to_smem(uint8_t* base, uint32_t i, float v) {
+        *(float*)(base + swz_byte(i * 4u)) = v;
+    }
+};
+template <>
+struct Storage<__nv_bfloat16> {
+    static constexpr int kPerUnit = 8;
+    __device__ static __forceinline__ void unpack(uint4 u, float* o) {
+        o[0] = __uint_as_float(u.x << 16); o[1] = __uint_as_float(u.x & 0xffff0000u);
+        o[2] = __uint_as_float(u.y << 16); o[3] = __uint_as_float(u.y & 0xffff0000u);
+        o[4] = __uint_as_float(u.z << 16); o[5] = __uint_as_float(u.z & 0xffff0000u);
+        o[6] = __uint_as_float(u.w << 16); o[7] = __uint_as_float(u.w & 0xffff0000u);
+    }
+    __device__ static __forceinline__ uint32_t pack2(float lo, float hi) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+        return *reinterpret_cast<uint32_t*>(&h);
+    }
+    __device__ static __forceinline__ uint4 pack(const float* v) {
+        return make_uint4(pack2(v[0], v[1]), pack2(v[2], v[3]), pack2(v[4], v[5]), pack2(v[6], v[7]));
+    }
+    __device__ static __forceinline__ float load(const void* p, int64_t i) {
+        return __bfloat162float(((const __nv_bfloat16*)p)[i]);
+    }
+    __device__ static __forceinline__ void store(void* p, int64_t i, float v) {
+        ((__nv_bfloat16*)p)[i] = __float2bfloat16_rn(v);
+    }
+    __device__ static __forceinline__ float from_smem(const uint8_t* base, uint32_t i) {
+        return __bfloat162float(*(const __nv_bfloat16*)(base + swz_byte(i * 2u)));
+    }
+    __device__ static __forceinline__ void to_smem(uint8_t* base, uint32_t i, float v) {
+        *(__nv_bfloat16*)(base + swz_byte(i * 2u)) = __float2bfloat16_rn(v);
+    }
+};
+
+// ------------------------------------------------------------------------------------------
+// mbarrier / TMA wrappers (raw PTX).
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+// Bounded wait: returns false when the limit ran out (the caller records an error and leaves).
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t limit) {
+    for (uint32_t i = 0; i < limit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// One 2-D tiled TMA load (no multicast) of a {box_x, 1} box into shared memory.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* tmap, int32_t x, int32_t y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+        "l"(tmap), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const void* tmap, int32_t x, int32_t y, uint32_t src) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];" ::"l"(tmap), "r"(x),
+                 "r"(y), "r"(src)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+// ------------------------------------------------------------------------------------------
+// One lane's run of K consecutive elements.
+//
+// Fast form (within the run the second scan is taken relative to the run start, Eq. 2 written
+// for a part):  A_t = sum_{i<=t} log|a_i|,  u_t = log|b_t| - A_t,  r = max_t u_t (the
+// log-sum-exp reference, Eq. 8),  s_t = sum_{i<=t} +-exp(u_i - r).  Then, for a value
+// x_c = S_c exp(M_c) entering the run,
+//     x_t = +-exp(A_t + M) * (S_c exp(M_c - M) + s_t exp(r - M)),   M = max(M_c, r),
+// i.e. one exp per element for the scan, one log (log output) or one exp (linear output) per
+// element for the result, and O(1) transcendental per run for the carry.
+template <int MODE, typename TIn, typename TOut, int K>
+struct Run {
+    static constexpr bool SIGNED = (MODE != kLogUnsigned);
+    using E = Elem<SIGNED>;
+    static constexpr int IN_UNITS = K / Storage<TIn>::kPerUnit;    // 16-byte units per lane, input
+    static constexpr int OUT_UNITS = K / Storage<TOut>::kPerUnit;  // 16-byte units per lane, output
+    static constexpr int CHUNK = 32 * K;
+    static constexpr int IN_BYTES = CHUNK * (int)sizeof(TIn);
+    static constexpr int OUT_BYTES = CHUNK * (int)sizeof(TOut);
+
+    float A[K];     // A_t
+    float s[K];     // s_t (before that: u_t)
+    uint32_t P[K];  // parity mask of a_1..a_t (SIGNED only)
+    float r;        // reference of the run, -inf when the run has no non-zero b
+    bool bad;       // the fast form does not apply to this run (a_t = 0, inf or NaN in it)
+
+    // Load the lane's K inputs of both tensors from the swizzled chunk.
+    __device__ __forceinline__ static void load(const uint8_t* sm_a, const uint8_t* sm_b, int lane, float* va, float* vb) {
+        const uint32_t base_a = smem_u32(sm_a), base_b = smem_u32(sm_b);
+#pragma unroll
+        for (int j = 0; j < IN_UNITS; ++j) {
+            const uint32_t off = swz_unit((uint32_t)(lane * IN_UNITS + j));
+            Storage<TIn>::unpack(lds128(base_a + off), va + j * Storage<TIn>::kPerUnit);
+            Storage<TIn>::unpack(lds128(base_b + off), vb + j * Storage<TIn>::kPerUnit);
+        }
+    }
+
+    // va, vb: the stored inputs (log a, log b for the log modes; a, b for kLinear).
+    // sa, sb: per-element sign masks for kLogSigned (ignored otherwise).
+    __device__ __forceinline__ E pass1(const float* va, const float* vb, const uint32_t* sa, const uint32_t* sb) {
+        float acc = 0.0f;
+        uint32_t par = 0u;
+        float rr = neg_inf();
+#pragma unroll
+        for (int t = 0; t < K; ++t) {
+            float la, lbr;
+            if (MODE == kLinear) {
+                la = log_abs_accurate(va[t]);
+                par ^= __float_as_uint(va[t]) & kSignBit;
+                lbr = lg2(fabsf(vb[t])) * kLn2;  // rough: only seeds the reference
+            } else {
+                la = va[t];
+                lbr = vb[t];
+                if (MODE == kLogSigned) par ^= sa[t];
+            }
+            acc += la;
+            A[t] = acc;
+            if (SIGNED) P[t] = par;
+            const float u = lbr - acc;
+            s[t] = u;
+            rr = fmaxf(rr, u);
+        }
+        r = rr;
+        bad = !(acc >= -1e30f) || !(rr <= 1e30f);
+        const float ref = (rr == neg_inf()) ? 0.0f : rr;
+        const float c = -ref * kLog2e;
+        float sum = 0.0f;
+#pragma unroll
+        for (int t = 0; t < K; ++t) {
+            float e;
+            if (MODE == kLinear) {
+                e = vb[t] * ex2(fminf(fmaf(-A[t], kLog2e, c), 126.0f));
+                e = flip(e, P[t]);
+            } else {
+                e = ex2(fmaf(s[t], kLog2e, c));
+                if (MODE == kLogSigned) e = flip(e, sb[t] ^ P[t]);
+            }
+            sum += e;
+            s[t] = sum;
+        }
+        E agg;
+        agg.A = acc;
+        agg.m = rr + acc;
+        agg.s = SIGNED ? flip(sum, par) : sum;  // beta = alpha * (sum relative to the run start)
+        agg.p = par;
+        return agg;
+    }
+
+    // Apply the value entering the run and produce the K outputs.
+    // out_mag: log|x_t| (log modes) or x_t (kLinear);  out_sign: sign masks (kLogSigned).
+    // Returns false when an early prefix is too small relative to the run's reference for the
+    // fast form to be trusted (the caller then redoes the chunk with the tracked form).
+    __device__ __forceinline__ bool apply(const E& entering, float* out_mag, uint32_t* out_sign) const {
+        const float Mc = entering.m, Sc = entering.s;
+        float M = fmaxf(Mc, r);
+        const float d = Mc - r;
+        const float ed = ex2(-fabsf(d) * kLog2e);
+        float C = (d >= 0.0f) ? Sc : Sc * ed;
+        float w = (d >= 0.0f) ? ed : 1.0f;
+        const bool empty = (M == neg_inf());
+        if (empty) { C = 0.0f; w = 0.0f; M = 0.0f; }
+        const float S1 = fmaf(s[0], w, C);
+        const bool ok = empty || (fabsf(S1) >= 8.67361738e-19f /* 2^-60 */);
+#pragma unroll
+        for (int t = 0; t < K; ++t) {
+            const float S = fmaf(s[t], w, C);
+            if (MODE == kLinear) {
+                const float h = ex2((A[t] + M) * (0.5f * kLog2e));
+                out_mag[t] = flip((S * h) * h, P[t]);
+            } else {
+                out_mag[t] = fmaf(lg2(fabsf(S)), kLn2, A[t] + M);
+                if (MODE == kLogSigned) {
+                    const uint32_t sg = (__float_as_uint(S) ^ P[t]) & kSignBit;
+                    out_sign[t] = (S == 0.0f) ? 0u : sg;
+                }
+            }
+        }
+        return ok;
+    }
+};
+
+// ------------------------------------------------------------------------------------------
+// Tracked form, used for the rare chunk the fast form declines (a_t = 0 inside a run, or more
+// than ~60 binary orders of magnitude between an early prefix and a later term of one run).
+// Every step carries its own max reference; inputs are re-read from shared memory, so it needs
+// no registers of the fast form.
+template <int MODE, typename TIn>
+struct Leaf {
+    static constexpr bool SIGNED = (MODE != kLogUnsigned);
+    // Element t (0..CHUNK-1) of the chunk as a one-step part.
+    __device__ static __forceinline__ Elem<SIGNED> get(const uint8_t* sm_a, const uint8_t* sm_b, uint32_t i,
+                                                       uint32_t sa, uint32_t sb) {
+        Elem<SIGNED> e;
+        const float va = Storage<TIn>::from_smem(sm_a, i);
+        const float vb = Storage<TIn>::from_smem(sm_b, i);
+        float lb;
+        uint32_t psb;
+        if (MODE == kLinear) {
+            e.A = log_abs_accurate(va);
+            e.p = __float_as_uint(va) & kSignBit;
+            lb = log_abs_accurate(vb);
+            psb = __float_as_uint(vb) & kSignBit;
+        } else {
+            e.A = va;
+            e.p = SIGNED ? sa : 0u;
+            lb = vb;
+            psb = SIGNED ? sb : 0u;
+        }
+        e.m = lb;
+        e.s = (lb == neg_inf()) ? 0.0f : (SIGNED ? flip(1.0f, psb) : 1.0f);
+        return e;
+    }
+};
+
+}  // namespace hs

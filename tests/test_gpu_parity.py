@@ -1,0 +1,310 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the float64 CPU oracle on identical
+seeded inputs.  Tolerances are the benchmark contract's:
+  positive inputs : |log x_gpu - log x_ref| <= 2e-6 (1 + |a*_t| + |log(x0 + b*_t)|) + 1e-5
+  signed inputs   : |x_gpu - x_ref| <= 1e-3 max_row |x_ref|
+  bf16 storage    : relative error of the stored log x <= 1e-2 (+ the fp32 tolerance as floor)
+"""
+import numpy as np
+import pytest
+import torch
+
+from hs_testlib import assert_log_close, assert_signed_close, storage_f64, to_dev, to_f64, tol_positive
+from paper_2311_06281_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+
+
+def run_log(hs, oracle, t, path=None, signs=None, out_dtype=None, what=""):
+    """scan_log on the GPU vs oracle.scan_log; positive-input tolerance (bf16 tolerance if stored as bf16)."""
+    if path is not None:
+        hs.set_path(path)
+    la, lb, lx0 = to_dev(t["log_a"]), to_dev(t["log_b"]), to_dev(t["log_x0"])
+    rows, n = t["log_a"].shape
+    ws = hs.new_workspace(rows, n, "cuda")
+    out = hs.scan_log(la, lb, lx0, out_dtype=out_dtype, workspace=ws)
+    hs.check(ws)
+    got = to_f64(out)
+    ref, _ = oracle.scan_log(t["log_a"], t["log_b"], t["log_x0"])
+    tol = tol_positive(storage_f64(t["log_a"]), ref)
+    if out.dtype == torch.bfloat16:
+        tol = tol + 1e-2 * np.abs(np.where(np.isfinite(ref), ref, 0.0))
+    return assert_log_close(got, ref, tol, what)
+
+
+def run_linear(hs, oracle, t, path=None, signed=False, what=""):
+    if path is not None:
+        hs.set_path(path)
+    a, b, x0 = to_dev(t["a"]), to_dev(t["b"]), to_dev(t["x0"])
+    rows, n = t["a"].shape
+    ws = hs.new_workspace(rows, n, "cuda")
+    x = hs.scan_linear(a, b, x0, workspace=ws)
+    hs.check(ws)
+    got = to_f64(x)
+    ref = oracle.scan_linear(t["a"], t["b"], t["x0"])
+    if signed:
+        return assert_signed_close(got, ref, what)
+    assert (got > 0).all(), f"{what}: non-positive output for positive inputs"
+    logref = np.log(ref)
+    with np.errstate(divide="ignore"):
+        tol = tol_positive(np.log(t["a"].astype(np.float64)), logref)
+    return assert_log_close(np.log(got), logref, tol, what)
+
+
+# ------------------------------------------------------------------------------------------ configs, reduced
+def test_cfg1_single_sequence_linear(hs, oracle):
+    w = workloads.make(1)
+    r = run_linear(hs, oracle, w.tensors, what="cfg1")
+    assert hs.last_path() == hs.PATH_LOOKBACK
+    assert r < 1.0
+    run_linear(hs, oracle, w.tensors, path=hs.PATH_BATCHED, what="cfg1 batched")
+
+
+def test_cfg1_closed_form_constant_ab(hs):
+    # x_t = 10 - 9*0.95^t for a = 0.95, b = 0.5, x0 = 1, from the stored fp32 value of 0.95
+    n = 4096
+    a32 = np.float32(0.95)
+    t = np.arange(1, n + 1, dtype=np.float64)
+    af = float(a32)
+    ref = af ** t + 0.5 * (1 - af ** t) / (1 - af)
+    for path in (hs.PATH_LOOKBACK, hs.PATH_BATCHED):
+        hs.set_path(path)
+        x = hs.scan_linear(torch.full((1, n), 0.95, device="cuda"), torch.full((1, n), 0.5, device="cuda"),
+                           torch.ones(1, device="cuda"))
+        got = to_f64(x)[0]
+        tol = 2e-6 * (1 + np.abs(t * np.log(af)) + np.abs(np.log(ref) - t * np.log(af))) + 1e-5
+        assert (np.abs(np.log(got) - np.log(ref)) <= tol).all()
+
+
+@pytest.mark.parametrize("path", ["batched", "lookback"])
+def test_cfg2_reduced(hs, oracle, path):
+    w = workloads.make(2, rows=1500)
+    r = run_log(hs, oracle, w.tensors, path=getattr(hs, "PATH_" + path.upper()), what=f"cfg2/{path}")
+    assert r < 1.0
+
+
+@pytest.mark.parametrize("n", [(1 << 20) + 76, (1 << 18) + 3])  # TMA with ragged tail; unaligned pitch
+def test_cfg3_reduced_long_sequence(hs, oracle, n):
+    w = workloads.make(3, rows=1, n=n)
+    run_log(hs, oracle, w.tensors, what=f"cfg3 log n={n}")
+    assert hs.last_path() == hs.PATH_LOOKBACK
+    run_linear(hs, oracle, w.tensors, what=f"cfg3 linear n={n}")
+
+
+@pytest.mark.parametrize("path", ["batched", "lookback"])
+def test_cfg4_reduced_signed_linear(hs, oracle, path):
+    w = workloads.make(4, rows=96)
+    run_linear(hs, oracle, w.tensors, path=getattr(hs, "PATH_" + path.upper()), signed=True, what=f"cfg4/{path}")
+
+
+@pytest.mark.parametrize("path", ["batched", "lookback"])
+def test_cfg4_reduced_signed_log_with_sign_tensors(hs, oracle, path):
+    w = workloads.make(4, rows=64, n=4096)
+    t = w.tensors
+    a64, b64, x064 = (t[k].astype(np.float64) for k in ("a", "b", "x0"))
+    la = np.log(np.abs(a64)).astype(np.float32)
+    lb = np.log(np.abs(b64)).astype(np.float32)
+    lx0 = np.log(np.abs(x064)).astype(np.float32)
+    sa, sb, sx0 = (a64 < 0).astype(np.uint8), (b64 < 0).astype(np.uint8), (x064 < 0).astype(np.uint8)
+    hs.set_path(getattr(hs, "PATH_" + path.upper()))
+    lx, sx = hs.scan_log(to_dev(la), to_dev(lb), to_dev(lx0), sign_a=to_dev(sa), sign_b=to_dev(sb), sign_x0=to_dev(sx0))
+    ref_l, ref_s = oracle.scan_log(la, lb, lx0, sa, sb, sx0)
+    got = np.where(sx.cpu().numpy() == 1, -1.0, 1.0) * np.exp(to_f64(lx))
+    ref = np.where(ref_s == 1, -1.0, 1.0) * np.exp(ref_l)
+    assert set(np.unique(sx.cpu().numpy())) <= {0, 1}
+    assert_signed_close(got, ref, f"cfg4 log+signs/{path}")
+
+
+@pytest.mark.parametrize("path", ["batched", "lookback"])
+def test_cfg5_reduced_bf16(hs, oracle, path):
+    w = workloads.make(5, rows=1300 if path == "batched" else 40)
+    run_log(hs, oracle, w.tensors, path=getattr(hs, "PATH_" + path.upper()), what=f"cfg5/{path}")
+
+
+def test_f32_in_bf16_out(hs, oracle):
+    w = workloads.make(2, rows=1300, n=1024)
+    run_log(hs, oracle, w.tensors, out_dtype=torch.bfloat16, what="f32->bf16")
+
+
+# ------------------------------------------------------------------------------------------ shapes
+@pytest.mark.parametrize("rows", [1, 3, 149])
+@pytest.mark.parametrize("n", [1, 2, 3, 5, 15, 16, 17, 31, 33, 127, 511, 512, 513, 1028, 4100, 8195])
+def test_odd_shapes_both_paths(hs, oracle, rows, n):
+    w = workloads.make(2, rows=rows, n=n, seed=rows * 100003 + n)
+    for path in (hs.PATH_BATCHED, hs.PATH_LOOKBACK):
+        run_log(hs, oracle, w.tensors, path=path, what=f"{rows}x{n}/{path}")
+
+
+@pytest.mark.parametrize("n", [7, 520, 4099])
+def test_odd_shapes_signed_linear(hs, oracle, n):
+    w = workloads.make(4, rows=5, n=n, seed=n)
+    for path in (hs.PATH_BATCHED, hs.PATH_LOOKBACK):
+        run_linear(hs, oracle, w.tensors, path=path, signed=True, what=f"signed 5x{n}/{path}")
+
+
+def test_unaligned_base_pointer(hs, oracle):
+    w = workloads.make(2, rows=9, n=1000)
+    t = w.tensors
+    rows, n = 9, 1000
+    def shifted(arr):  # base pointer 4 bytes past a 16-byte boundary
+        buf = torch.empty(arr.size + 1, dtype=torch.float32, device="cuda")
+        v = buf[1:].view(arr.shape)
+        v.copy_(torch.from_numpy(arr))
+        return v
+    la, lb = shifted(t["log_a"]), shifted(t["log_b"])
+    out = hs.scan_log(la, lb, to_dev(t["log_x0"]))
+    ref, _ = oracle.scan_log(t["log_a"], t["log_b"], t["log_x0"])
+    assert_log_close(to_f64(out), ref, tol_positive(t["log_a"].astype(np.float64), ref), "unaligned base")
+
+
+# ------------------------------------------------------------------------------------------ degenerate inputs
+@pytest.mark.parametrize("path", ["batched", "lookback"])
+def test_zeros_resets_and_wide_range(hs, oracle, path):
+    """log 0 = -inf inputs, a_t = 0 (state reset), x0 = 0, and runs whose terms span hundreds of
+    orders of magnitude (the kernel's tracked form) all reproduce the oracle."""
+    rng = np.random.default_rng(11)
+    rows, n = 6, 3000
+    la = -rng.uniform(0, 0.3, (rows, n)).astype(np.float32)
+    lb = rng.normal(size=(rows, n)).astype(np.float32)
+    lx0 = rng.normal(size=rows).astype(np.float32)
+    lb[0, :] = -np.inf                                  # b == 0 everywhere: log x = log x0 + a*
+    lx0[1] = -np.inf                                    # x0 == 0
+    lb[1, :700] = -np.inf                               # ... and nothing added for 700 steps: x == 0 exactly
+    la[2, [5, 600, 601, 2999]] = -np.inf                # a_t == 0: the state resets to b_t
+    lb[3, ::7] = -np.inf                                # sparse zeros
+    lb[4, :] = rng.uniform(-300, 300, n).astype(np.float32)   # wide dynamic range inside every run
+    la[5, :] = -rng.uniform(5, 30, n).astype(np.float32)      # violent decay: a* ~ -50000
+    lx0[5] = 50.0
+    t = dict(log_a=la, log_b=lb, log_x0=lx0)
+    hs.set_path(getattr(hs, "PATH_" + path.upper()))
+    out = hs.scan_log(to_dev(la), to_dev(lb), to_dev(lx0))
+    got = to_f64(out)
+    ref, _ = oracle.scan_log(la, lb, lx0)
+    assert_log_close(got, ref, tol_positive(la.astype(np.float64), ref), f"degenerate/{path}")
+    assert np.isneginf(got[1, :700]).all()
+
+
+@pytest.mark.parametrize("path", ["batched", "lookback"])
+def test_linear_zeros_and_cancellation(hs, oracle, path):
+    rng = np.random.default_rng(12)
+    rows, n = 4, 2500
+    a = rng.uniform(0.5, 1.0, (rows, n)).astype(np.float32) * rng.choice([-1, 1], (rows, n)).astype(np.float32)
+    b = rng.normal(size=(rows, n)).astype(np.float32)
+    x0 = rng.normal(size=rows).astype(np.float32)
+    a[0, [0, 17, 1000]] = 0.0
+    b[1, :] = 0.0
+    x0[2] = 0.0
+    b[2, :40] = 0.0
+    a[3, :] = -1.0
+    b[3, :] = 0.0                                      # x_t = (-1)^t x0
+    hs.set_path(getattr(hs, "PATH_" + path.upper()))
+    x = hs.scan_linear(to_dev(a), to_dev(b), to_dev(x0))
+    ref = oracle.scan_linear(a, b, x0)
+    got = to_f64(x)
+    assert_signed_close(got, ref, f"linear degenerate/{path}")
+    assert (got[2, :40] == 0).all()
+    np.testing.assert_allclose(got[3], ref[3], rtol=1e-5)
+
+
+def test_nan_and_inf_stay_in_their_row(hs, oracle):
+    w = workloads.make(2, rows=8, n=2048)
+    t = {k: v.copy() for k, v in w.tensors.items()}
+    ref, _ = oracle.scan_log(t["log_a"], t["log_b"], t["log_x0"])
+    t["log_b"][3, 1000] = np.nan
+    t["log_a"][5, 77] = np.inf
+    for path in (hs.PATH_BATCHED, hs.PATH_LOOKBACK):
+        hs.set_path(path)
+        got = to_f64(hs.scan_log(to_dev(t["log_a"]), to_dev(t["log_b"]), to_dev(t["log_x0"])))
+        tol = tol_positive(w.tensors["log_a"].astype(np.float64), ref)
+        for r in (0, 1, 2, 4, 6, 7):
+            assert_log_close(got[r:r + 1], ref[r:r + 1], tol[r:r + 1], f"row {r}")
+        assert_log_close(got[3:4, :1000], ref[3:4, :1000], tol[3:4, :1000], "before the NaN")
+
+
+def test_in_place_and_guard_bands(hs, oracle):
+    """The output may alias an input; nothing outside [rows, n] is written (canaries on both sides)."""
+    w = workloads.make(2, rows=37, n=1540)
+    t = w.tensors
+    rows, n = 37, 1540
+    ref, _ = oracle.scan_log(t["log_a"], t["log_b"], t["log_x0"])
+    tol = tol_positive(t["log_a"].astype(np.float64), ref)
+    pad = 1024
+    for path in (hs.PATH_BATCHED, hs.PATH_LOOKBACK):
+        hs.set_path(path)
+        buf = torch.full((rows * n + 2 * pad,), float("nan"), device="cuda")
+        canary = torch.tensor(0x7FC0DEAD, dtype=torch.int32, device="cuda")
+        buf.view(torch.int32)[:pad] = canary
+        buf.view(torch.int32)[-pad:] = canary
+        out = buf[pad:pad + rows * n].view(rows, n)
+        out.copy_(torch.from_numpy(t["log_b"]))          # in situ: log_b is overwritten by log x
+        hs.scan_log(to_dev(t["log_a"]), out, to_dev(t["log_x0"]), log_x=out)
+        assert_log_close(to_f64(out), ref, tol, "in place")
+        assert (buf.view(torch.int32)[:pad] == canary).all() and (buf.view(torch.int32)[-pad:] == canary).all()
+
+
+def test_split_invariance_on_gpu(hs):
+    """[0,n) in one call equals [0,k) then [k,n) restarted from x_k, at chunk and tile borders +-1."""
+    w = workloads.make(2, rows=3, n=9000)
+    la, lb, lx0 = (to_dev(w.tensors[k]) for k in ("log_a", "log_b", "log_x0"))
+    whole = hs.scan_log(la, lb, lx0)
+    for k in (511, 512, 513, 4095, 4096, 4097):
+        head = hs.scan_log(la[:, :k].contiguous(), lb[:, :k].contiguous(), lx0)
+        tail = hs.scan_log(la[:, k:].contiguous(), lb[:, k:].contiguous(), head[:, -1].contiguous())
+        got = torch.cat([head, tail], dim=1)
+        assert (got - whole).abs().max().item() < 2e-5
+
+
+def test_empty_and_invalid_arguments(hs):
+    z = torch.empty((0, 16), device="cuda")
+    assert hs.scan_log(z, z, torch.empty(0, device="cuda")).shape == (0, 16)
+    L = hs.lib()
+    a = torch.zeros((2, 8), device="cuda")
+    x0 = torch.zeros(2, device="cuda")
+    ws = hs.new_workspace(2, 8, "cuda")
+    p = lambda t: t.data_ptr()
+    assert L.heinsen_scan_log(p(a), p(a), p(x0), p(a), None, None, None, None, 0, 8, 0, 0, p(ws), ws.numel(), None) == 0
+    assert L.heinsen_scan_log(None, p(a), p(x0), p(a), None, None, None, None, 2, 8, 0, 0, p(ws), ws.numel(), None) == 1
+    assert L.heinsen_scan_log(p(a), p(a), p(x0), p(a), None, None, None, None, -1, 8, 0, 0, p(ws), ws.numel(), None) == 1
+    assert L.heinsen_scan_log(p(a), p(a), p(x0), p(a), None, None, None, None, 2, 8, 1, 0, p(ws), ws.numel(), None) == 1
+    assert L.heinsen_scan_log(p(a), p(a), p(x0), p(a), None, None, None, None, 2, 8, 0, 0, p(ws), 16, None) == 3
+    assert L.heinsen_scan_log(p(a), p(a), p(x0), p(a), p(ws), None, None, None, 2, 8, 0, 0, p(ws), ws.numel(), None) == 1
+    assert L.heinsen_scan_linear(p(a), p(a), p(x0), p(a), 2, 8, 1, p(ws), ws.numel(), None) == 1
+    torch.cuda.synchronize()
+
+
+def test_lookback_wait_is_bounded_and_reported(hs):
+    """A tile that never publishes makes its successors give up after the poll limit: the call
+    reports HS_ERR_LOOKBACK_TIMEOUT, nothing hangs, and the next call works."""
+    w = workloads.make(2, rows=1, n=1 << 18)
+    la, lb, lx0 = (to_dev(w.tensors[k]) for k in ("log_a", "log_b", "log_x0"))
+    hs.set_path(hs.PATH_LOOKBACK)
+    ws = hs.new_workspace(1, 1 << 18, "cuda")
+    hs.debug_config(lookback_spin_limit=2000, mute_tile=3)
+    hs.scan_log(la, lb, lx0, workspace=ws)
+    with pytest.raises(hs.HeinsenScanError) as ei:
+        hs.check(ws)
+    assert ei.value.status == 5
+    hs.debug_config(0, -1)
+    good = hs.scan_log(la, lb, lx0, workspace=ws)
+    hs.check(ws)
+    assert torch.isfinite(good).all()
+
+
+def test_host_buffer_entry_point(hs, oracle):
+    w = workloads.make(2, rows=300, n=2048)
+    t = w.tensors
+    la, lb, lx0 = (torch.from_numpy(t[k]).pin_memory() for k in ("log_a", "log_b", "log_x0"))
+    out = torch.empty_like(la).pin_memory()
+    scratch = torch.empty(hs.host_scratch_bytes(300, 2048, torch.float32, torch.float32, False), dtype=torch.uint8,
+                          device="cuda")
+    hs.scan_log_host(la, lb, lx0, out, scratch)
+    ref, _ = oracle.scan_log(t["log_a"], t["log_b"], t["log_x0"])
+    assert_log_close(out.double().numpy(), ref, tol_positive(t["log_a"].astype(np.float64), ref), "host entry")
+
+
+def test_repeatability(hs):
+    w = workloads.make(3, rows=1, n=1 << 21)
+    la, lb, lx0 = (to_dev(w.tensors[k]) for k in ("log_a", "log_b", "log_x0"))
+    first = hs.scan_log(la, lb, lx0)
+    for _ in range(5):
+        again = hs.scan_log(la, lb, lx0)
+        assert (again - first).abs().max().item() < 1e-5
