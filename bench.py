@@ -1,0 +1,329 @@
+#!/usr/bin/env python
+"""Benchmark of the fused recurrence scan (one JSON line on stdout).
+
+A "step" is one pass of the whole hot path -- one call of the C ABI on one batch of seeded
+synthetic input.  Default workload: configuration 2 of the benchmark contract (16384 rows x 2048
+steps, fp32, log-space inputs of a linear-RNN layer), the configuration the headline metric is
+quoted on.  `value` is elements/s with the inputs resident in HBM; `e2e` is the same metric through
+the host-buffer entry point with pinned host buffers and both copies inside the timed region.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 2|3|4|5] [--impl reference]
+
+N > 1 is launched by torchrun (one rank per GPU); rows are independent, so every rank runs its own
+batch (weak scaling) and the only communication is the barrier and the max-over-ranks of the time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "recurrence_elements_per_s"
+UNIT = "elements/s"
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# captures summarised under profiles/ (None until a capture of that workload exists).
+NCU_TRAFFIC_BYTES = {2: None, 3: None, 4: None, 5: None}
+
+HBM_FALLBACK_GBS = 6650.0  # used only when MEASURED_PEAKS.json is absent
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", type=int, default=2, choices=[2, 3, 4, 5])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return HBM_FALLBACK_GBS, "fallback"
+
+
+def bytes_per_element(w) -> int:
+    es = 4 if w.storage == "f32" else 2
+    return 3 * es  # two inputs read once, one output written once
+
+
+def workload_name(cid, w):
+    return f"cfg{cid}: {w.name} ({w.rows} rows x n={w.n}, {'scan_linear' if w.kind == 'linear' else 'scan_log'}, {w.storage} storage)"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while a timed region runs."""
+    REASONS = {
+        0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+        0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+        0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting",
+    }
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def sample(self):
+        if self.nv is None:
+            return
+        try:
+            self.samples.append(int(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM)))
+            mask = int(self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+            for bit, name in self.REASONS.items():
+                if mask & bit and name != "gpu_idle":
+                    self.reasons.add(name)
+        except Exception:
+            pass
+
+    def start(self):
+        def loop():
+            while not self._stop.is_set():
+                self.sample()
+                time.sleep(0.005)
+        self._thread = threading.Thread(target=loop, daemon=True)
+        self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(s)}
+
+
+# ---------------------------------------------------------------------------------------------- reference arm
+def run_reference(args):
+    """Times the float64 CPU oracle, as it stands, on a bounded sample of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+    from oracle import heinsen_oracle
+    from paper_2311_06281_b200 import workloads
+
+    cid = args.workload
+    full = workloads.CONFIGS[cid]
+    # bounded sample: about 2^22 elements per step
+    if full["rows"] == 1:
+        rows, n = 1, min(full["n"], 1 << 22)
+    else:
+        rows, n = max(1, min(full["rows"], (1 << 22) // full["n"])), full["n"]
+    w = workloads.make(cid, rows=rows, n=n)
+    t = w.tensors
+    heinsen_oracle.build()
+    cores = heinsen_oracle.max_threads() if rows > 1 else 1
+
+    def step():
+        if w.kind == "linear":
+            heinsen_oracle.scan_linear(t["a"], t["b"], t["x0"], nthreads=cores)
+        else:
+            heinsen_oracle.scan_log(t["log_a"], t["log_b"], t["log_x0"], nthreads=cores)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    value = rows * n * args.steps / dt
+    sample = f"{rows} rows x n={n} of {workload_name(cid, workloads.Workload(**{**full, 'tensors': {}}))} per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_name(cid, workloads.Workload(**{**full, "tensors": {}})), "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------- our arm
+def run_ours(args):
+    import numpy as np
+    import torch
+
+    from paper_2311_06281_b200 import build_ext, heinsen_scan as hs, sharding, workloads
+
+    rank, world, local = sharding.init_from_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    build_ext.build()
+    hs.lib()
+
+    cid = args.workload
+    # weak scaling: every rank runs its own full batch, seeded by its rank
+    w = workloads.make(cid, seed=rank)
+    t = w.tensors
+    rows, n = w.rows, w.n
+    keys = ("a", "b", "x0") if w.kind == "linear" else ("log_a", "log_b", "log_x0")
+
+    def dev_tensor(arr):
+        x = torch.from_numpy(np.ascontiguousarray(arr))
+        if arr.dtype == np.uint16:
+            x = x.view(torch.bfloat16)
+        return x.to(dev)
+
+    # rotate independent buffer sets so that no step finds its inputs in L2 (each set alone exceeds L2)
+    nsets = 3
+    base = [dev_tensor(t[k]) for k in keys]
+    sets = [base] + [[x.clone() for x in base] for _ in range(nsets - 1)]
+    outs = [torch.empty((rows, n), dtype=base[0].dtype, device=dev) for _ in range(nsets)]
+    wss = [hs.new_workspace(rows, n, dev) for _ in range(nsets)]
+    call = hs.scan_linear if w.kind == "linear" else hs.scan_log
+
+    def step(i):
+        s = i % nsets
+        if w.kind == "linear":
+            hs.scan_linear(sets[s][0], sets[s][1], sets[s][2], x=outs[s], workspace=wss[s])
+        else:
+            hs.scan_log(sets[s][0], sets[s][1], sets[s][2], log_x=outs[s], workspace=wss[s])
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    torch.cuda.synchronize()
+    for ws in wss:
+        hs.check(ws)
+
+    sampler = ClockSampler(local)
+    launches0 = hs.launch_count()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sharding.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    start.record()
+    for i in range(args.steps):
+        step(i)
+    stop.record()
+    sampler.sample()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    sharding.barrier()
+    ms_local = start.elapsed_time(stop)
+    ms_total = sharding.max_over_ranks(ms_local, dev)
+    launches = hs.launch_count() - launches0
+    for ws in wss:
+        hs.check(ws)
+
+    elements = rows * n
+    ms_per_step = ms_total / args.steps
+    value = world * elements / (ms_per_step * 1e-3)
+
+    # roofline of the (single) kernel of a step: algorithmic bytes per launch / mean launch duration
+    peak, peak_kind = measured_peak()
+    bpe = bytes_per_element(w)
+    alg_bytes = elements * bpe + rows * (4 if w.storage == "f32" else 2)
+    achieved = alg_bytes / (ms_local / args.steps * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": NCU_TRAFFIC_BYTES.get(cid), "peak_source": f"{peak_kind} (MEASURED_PEAKS.json hbm_gbs)"
+                if peak_kind == "measured" else "fallback (no MEASURED_PEAKS.json)",
+                "algorithmic_bytes_per_launch": alg_bytes, "bytes_per_element": bpe,
+                "kernel": "batched_scan_kernel" if hs.last_path() == hs.PATH_BATCHED else "lookback_scan_kernel",
+                "frac_of_nominal_8TBs": achieved / 8000.0}
+
+    # end to end through the host-buffer entry point: pinned host buffers, H2D + kernel + D2H per step
+    e2e = None
+    if not args.no_e2e:
+        host_in = [torch.from_numpy(np.ascontiguousarray(t[k])) for k in keys]
+        host_in = [(x.view(torch.bfloat16) if x.dtype == torch.uint16 else x).pin_memory() for x in host_in]
+        host_out = torch.empty((rows, n), dtype=host_in[0].dtype).pin_memory()
+        scratch = torch.empty(hs.host_scratch_bytes(rows, n, host_in[0].dtype, host_out.dtype, False), dtype=torch.uint8,
+                              device=dev)
+        host_call = hs.scan_linear_host if w.kind == "linear" else hs.scan_log_host
+        e2e_steps = max(3, min(args.steps, 20))
+        for _ in range(3):
+            host_call(host_in[0], host_in[1], host_in[2], host_out, scratch)
+        sharding.barrier()
+        torch.cuda.synchronize()
+        start.record()
+        for _ in range(e2e_steps):
+            host_call(host_in[0], host_in[1], host_in[2], host_out, scratch)
+        stop.record()
+        torch.cuda.synchronize()
+        e2e_ms = sharding.max_over_ranks(start.elapsed_time(stop), dev) / e2e_steps
+        es = host_in[0].element_size()
+        e2e = {"value": world * elements / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 2 * elements * es + rows * es,
+               "d2h_bytes_per_step": elements * host_out.element_size(), "ms_per_step": e2e_ms, "steps": e2e_steps,
+               "entry_point": "heinsen_scan_linear_host" if w.kind == "linear" else "heinsen_scan_log_host"}
+        del scratch
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import heinsen_oracle
+        heinsen_oracle.build()
+        # bounded sample of the same workload: at most 2^25 elements per pass, repeated for a few seconds
+        if rows == 1:
+            srows, sn = 1, min(n, 1 << 25)
+        else:
+            srows, sn = max(1, min(rows, (1 << 25) // n)), n
+        sub = {k: (t[k][:srows, :sn] if t[k].ndim == 2 else t[k][:srows]) for k in keys}
+        sub = {k: np.ascontiguousarray(v) for k, v in sub.items()}
+        cores = heinsen_oracle.max_threads() if srows > 1 else 1
+        passes, t0 = 0, time.perf_counter()
+        while True:
+            if w.kind == "linear":
+                heinsen_oracle.scan_linear(sub["a"], sub["b"], sub["x0"], nthreads=cores)
+            else:
+                heinsen_oracle.scan_log(sub["log_a"], sub["log_b"], sub["log_x0"], nthreads=cores)
+            passes += 1
+            dt = time.perf_counter() - t0
+            if dt > 4.0 or passes >= 8:
+                break
+        cpu_baseline = {"value": srows * sn * passes / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+                        "sample": f"{passes} passes over {srows} rows x n={sn} of the bench workload "
+                                  f"({'whole batch' if srows * sn == elements else 'first rows'}), float64 sequential loop, "
+                                  f"OpenMP over rows"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": workload_name(cid, w), "rows_per_gpu": rows, "n": n, "storage": w.storage,
+                       "entry_point": "heinsen_scan_linear" if w.kind == "linear" else "heinsen_scan_log",
+                       "l2": f"{nsets} rotating buffer sets of {alg_bytes / 1e6:.0f} MB each (every set exceeds the 126 MB L2)",
+                       "parallelism": f"rows sharded, {world} rank(s), no data-path collective"},
+            "clocks": clocks, "gpu_launches": launches, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu_baseline,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
