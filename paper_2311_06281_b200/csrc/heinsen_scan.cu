@@ -27,6 +27,7 @@ thread_local char g_cuda_msg[256] = "";
 
 constexpr long long kMaxTmaDim = (1ll << 31) - (1ll << 20);  // TMA coordinates are int32
 constexpr int kBatchedMinRowsPerSm = 8;  // fewer rows per SM than this: look-back kernel
+constexpr int kBatchedMinWarpsPerSm = 12; // rows per warp are chosen to keep at least this many warps per SM
 constexpr int kLookbackWarps = 8;        // warps (= chunks) per tile of the look-back kernel
 constexpr int kMinChunk = 512;           // smallest chunk (32 lanes x 16 elements)
 
@@ -91,14 +92,14 @@ EncodeFn encode_fn() {
     return fn;
 }
 
-// [rows, n] row-major as a 2-D tensor map whose box is one 128-byte row segment, 128-byte swizzle.
-bool make_tmap(CUtensorMap* tm, const void* ptr, hs_dtype dt, long long rows, long long n) {
+// [rows, n] row-major as a 2-D tensor map whose box is {128 bytes of a row, box_rows rows}, 128-byte swizzle.
+bool make_tmap(CUtensorMap* tm, const void* ptr, hs_dtype dt, long long rows, long long n, int box_rows) {
     EncodeFn fn = encode_fn();
     if (!fn) return false;
     const int es = (dt == HS_F32) ? 4 : 2;
     cuuint64_t dims[2] = {(cuuint64_t)n, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)n * es};
-    cuuint32_t box[2] = {(cuuint32_t)(128 / es), 1};
+    cuuint32_t box[2] = {(cuuint32_t)(128 / es), (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(tm, dt == HS_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
                     const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -188,6 +189,46 @@ size_t workspace_bytes_for(long long rows, long long n) {
     return sizeof(Header) + (size_t)tiles * (8 + 16 + 16);
 }
 
+// cudaFuncSetAttribute and the occupancy query cost microseconds per call; remember what was set.
+struct FnCache {
+    const void* fn;
+    int dev;
+    int smem_set;
+    int occ_threads, occ_smem, occ_value;
+};
+std::mutex g_fn_mu;
+FnCache g_fn_cache[128];
+int g_fn_count = 0;
+
+FnCache* fn_slot(const void* fn) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    for (int i = 0; i < g_fn_count; ++i)
+        if (g_fn_cache[i].fn == fn && g_fn_cache[i].dev == dev) return &g_fn_cache[i];
+    if (g_fn_count >= 128) return nullptr;
+    FnCache* c = &g_fn_cache[g_fn_count++];
+    c->fn = fn; c->dev = dev; c->smem_set = -1; c->occ_threads = c->occ_smem = c->occ_value = -1;
+    return c;
+}
+
+cudaError_t ensure_smem_attr(const void* fn, int smem) {
+    std::lock_guard<std::mutex> lk(g_fn_mu);
+    FnCache* c = fn_slot(fn);
+    if (c && c->smem_set >= smem) return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess && c) c->smem_set = smem;
+    return e;
+}
+
+cudaError_t cached_occupancy(int* per_sm, const void* fn, int threads, int smem) {
+    std::lock_guard<std::mutex> lk(g_fn_mu);
+    FnCache* c = fn_slot(fn);
+    if (c && c->occ_threads == threads && c->occ_smem == smem) { *per_sm = c->occ_value; return cudaSuccess; }
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(per_sm, fn, threads, smem);
+    if (e == cudaSuccess && c) { c->occ_threads = threads; c->occ_smem = smem; c->occ_value = *per_sm; }
+    return e;
+}
+
 hs_status cuda_fail(const char* what, cudaError_t e) {
     snprintf(g_cuda_msg, sizeof g_cuda_msg, "%s: %s", what, cudaGetErrorString(e));
     return HS_ERR_CUDA;
@@ -229,28 +270,29 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
     p.mute_tile = g_mute_tile.load();
     p.ws = reinterpret_cast<Header*>(workspace);
 
-    CUtensorMap tm_a, tm_b, tm_o;
-    std::memset(&tm_a, 0, sizeof tm_a);
-    std::memset(&tm_b, 0, sizeof tm_b);
-    std::memset(&tm_o, 0, sizeof tm_o);
-    if (tma) {
-        if (!make_tmap(&tm_a, p.in_a, pr.din, p.rows, p.n) || !make_tmap(&tm_b, p.in_b, pr.din, p.rows, p.n) ||
-            !make_tmap(&tm_o, p.out, pr.dout, p.rows, p.n)) {
-            snprintf(g_cuda_msg, sizeof g_cuda_msg, "cuTensorMapEncodeTiled failed");
-            return HS_ERR_CUDA;
-        }
-    }
-
     const int path = choose_path(p.rows, dev);
     int warps, stages, grid;
     const void* fn;
     if (path == HS_PATH_BATCHED) {
-        warps = env_int("HEINSEN_SCAN_WARPS", 12, 1, 16);
-        stages = tma ? env_int("HEINSEN_SCAN_STAGES", 3, 2, kMaxStages) : 1;
-        const long long ctas_needed = (p.rows + warps - 1) / warps;
+        // R rows per warp (32/R lanes per row): the largest R that still leaves about a dozen warps
+        // per SM, so that rows with many steps use few scan steps and few rows still fill the GPU.
+        int R = 8;
+        while (R > 1 && (p.rows + R - 1) / R < (long long)kBatchedMinWarpsPerSm * dev.sm_count) R >>= 1;
+        R = env_int("HEINSEN_SCAN_ROWS_PER_WARP", R, 1, 8);
+        while (R & (R - 1)) R &= R - 1;  // power of two
+        p.rows_per_warp = R;
+        p.nchunks = (int)((p.n + (32 / R) * ke.K - 1) / ((32 / R) * ke.K));
+        const long long groups = (p.rows + R - 1) / R;
+        stages = tma ? env_int("HEINSEN_SCAN_STAGES", 2, 2, kMaxStages) : 1;
+        const int max_warps = 16;
+        long long per_sm = (groups + dev.sm_count - 1) / dev.sm_count;
+        warps = (int)(per_sm < 1 ? 1 : (per_sm > max_warps ? max_warps : per_sm));
+        warps = env_int("HEINSEN_SCAN_WARPS", warps, 1, 16);
+        const long long ctas_needed = (groups + warps - 1) / warps;
         grid = (int)(ctas_needed < dev.sm_count ? ctas_needed : dev.sm_count);
         fn = ke.batched;
     } else {
+        p.rows_per_warp = 1;
         warps = kLookbackWarps;
         stages = tma ? env_int("HEINSEN_SCAN_LB_STAGES", 2, 2, kMaxStages) : 1;
         p.tiles_per_row = (int)lookback_tiles_per_row(p.n, chunk);
@@ -264,11 +306,24 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         fn = ke.lookback;
         grid = 0;  // set below from occupancy
     }
+
+    CUtensorMap tm_a, tm_b, tm_o;
+    std::memset(&tm_a, 0, sizeof tm_a);
+    std::memset(&tm_b, 0, sizeof tm_b);
+    std::memset(&tm_o, 0, sizeof tm_o);
+    if (tma) {
+        const int br = p.rows_per_warp;
+        if (!make_tmap(&tm_a, p.in_a, pr.din, p.rows, p.n, br) || !make_tmap(&tm_b, p.in_b, pr.din, p.rows, p.n, br) ||
+            !make_tmap(&tm_o, p.out, pr.dout, p.rows, p.n, br)) {
+            snprintf(g_cuda_msg, sizeof g_cuda_msg, "cuTensorMapEncodeTiled failed");
+            return HS_ERR_CUDA;
+        }
+    }
     p.stages = stages;
     const int smem = warps * (stages * ke.warp_smem_per_stage + ke.warp_smem_out) + warps * 8 * kMaxStages + 1024 +
                      (path == HS_PATH_LOOKBACK ? 1024 : 0);
     if (smem > dev.max_smem_optin) return HS_ERR_INVALID_ARG;
-    cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t e = ensure_smem_attr(fn, smem);
     if (e != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", e);
 
     void* args[] = {&p, &tm_a, &tm_b, &tm_o};
@@ -276,7 +331,7 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         // Tiles wait for their predecessors, so every CTA must be resident: size the grid from the
         // occupancy of this kernel and launch cooperatively (the launch fails rather than deadlocks).
         int per_sm = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, warps * 32, smem);
+        e = cached_occupancy(&per_sm, fn, warps * 32, smem);
         if (e != cudaSuccess) return cuda_fail("cudaOccupancyMaxActiveBlocksPerMultiprocessor", e);
         if (per_sm < 1) return HS_ERR_INVALID_ARG;
         per_sm = env_int("HEINSEN_SCAN_LB_CTAS_PER_SM", per_sm, 1, per_sm);

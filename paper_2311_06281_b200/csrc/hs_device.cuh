@@ -20,6 +20,9 @@ namespace hs {
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr uint32_t kSignBit = 0x80000000u;
+// Reference of an empty sum (beta == 0, s == 0).  A large finite value instead of -inf keeps
+// differences of references free of inf - inf without a guard in the inner combine.
+constexpr float kEmpty = -1e20f;
 
 enum Mode : int { kLogUnsigned = 0, kLogSigned = 1, kLinear = 2 };
 
@@ -74,7 +77,7 @@ __device__ __forceinline__ float log_abs_accurate(float v) {
 template <bool SIGNED>
 struct Elem {
     float A;     // sum of log|a|
-    float m;     // reference of beta = s*exp(m); -inf <=> beta == 0 (then s == 0)
+    float m;     // reference of beta = s*exp(m), always finite (>= about kEmpty); beta == 0 <=> s == 0
     float s;     // signed, scaled sum
     uint32_t p;  // sign mask (0 or 0x80000000) of alpha; unused when !SIGNED
 };
@@ -82,11 +85,13 @@ struct Elem {
 template <bool SIGNED>
 __device__ __forceinline__ Elem<SIGNED> identity_elem() {
     Elem<SIGNED> e;
-    e.A = 0.0f; e.m = neg_inf(); e.s = 0.0f; e.p = 0u;
+    e.A = 0.0f; e.m = kEmpty; e.s = 0.0f; e.p = 0u;
     return e;
 }
 
 // "first" is the older part, "second" the newer one: result = second o first.
+// second.m must be finite (it always is: leaves and aggregates clamp at kEmpty); first.m + second.A
+// may be -inf (a_t = 0 inside the second part wipes out the first part's beta).
 template <bool SIGNED>
 __device__ __forceinline__ Elem<SIGNED> compose(const Elem<SIGNED>& first, const Elem<SIGNED>& second) {
     Elem<SIGNED> o;
@@ -94,10 +99,12 @@ __device__ __forceinline__ Elem<SIGNED> compose(const Elem<SIGNED>& first, const
     const float m1 = first.m + second.A;  // beta_1 carried through alpha_2
     const float s1 = SIGNED ? flip(first.s, second.p) : first.s;
     o.m = fmaxf(m1, second.m);
-    const float d = m1 - second.m;  // NaN only when both are -inf
-    float e = ex2(-fabsf(d) * kLog2e);
-    e = (o.m == neg_inf()) ? 0.0f : e;
-    o.s = (d >= 0.0f) ? fmaf(second.s, e, s1) : fmaf(s1, e, second.s);
+    const float d = m1 - second.m;
+    const float e = ex2(-fabsf(d) * kLog2e);
+    const bool first_is_ref = (d >= 0.0f);
+    const float hi = first_is_ref ? s1 : second.s;
+    const float lo = first_is_ref ? second.s : s1;
+    o.s = fmaf(lo, e, hi);
     o.p = SIGNED ? (first.p ^ second.p) : 0u;
     return o;
 }
@@ -130,21 +137,32 @@ __device__ __forceinline__ Elem<SIGNED> shfl_down_elem(const Elem<SIGNED>& e, in
     return o;
 }
 
-// Inclusive Kogge-Stone scan of one element per lane (the Hillis-Steele pattern the paper
-// cites for O(log n) prefix sums), then the exclusive prefix of each lane and the warp total.
+// Inclusive Kogge-Stone scan (the Hillis-Steele pattern the paper cites for O(log n) prefix sums)
+// over the lanes that share a row.  A warp holds R rows (R = 1, 2, 4 or 8); lane = i*R + g is
+// segment i of row g, so the lanes of one row are R apart and the scan takes log2(32/R) steps.
+// Returns the exclusive prefix of each lane and the total of its row (held by every lane of the row).
 template <bool SIGNED>
-__device__ __forceinline__ void warp_scan(const Elem<SIGNED>& mine, int lane, Elem<SIGNED>& exclusive,
-                                          Elem<SIGNED>& total) {
+__device__ __forceinline__ void row_scan(const Elem<SIGNED>& mine, int lane, int R, Elem<SIGNED>& exclusive,
+                                         Elem<SIGNED>& total) {
     Elem<SIGNED> inc = mine;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
-        Elem<SIGNED> up = shfl_up_elem(inc, d);
-        Elem<SIGNED> c = compose(up, inc);
-        if (lane >= d) inc = c;
+        if (d >= R) {  // warp-uniform
+            Elem<SIGNED> up = shfl_up_elem(inc, d);
+            Elem<SIGNED> c = compose(up, inc);
+            if (lane >= d) inc = c;
+        }
     }
-    total = shfl_elem(inc, 31);
-    Elem<SIGNED> up = shfl_up_elem(inc, 1);
-    exclusive = (lane == 0) ? identity_elem<SIGNED>() : up;
+    total = shfl_elem(inc, 32 - R + (lane & (R - 1)));
+    Elem<SIGNED> up = shfl_up_elem(inc, R);
+    exclusive = (lane < R) ? identity_elem<SIGNED>() : up;
+}
+
+// Plain 32-lane scan (one row per warp), used for the per-warp aggregates of a look-back tile.
+template <bool SIGNED>
+__device__ __forceinline__ void warp_scan(const Elem<SIGNED>& mine, int lane, Elem<SIGNED>& exclusive,
+                                          Elem<SIGNED>& total) {
+    row_scan(mine, lane, 1, exclusive, total);
 }
 
 // The running value x = s*exp(m) as an element (alpha irrelevant: A = -inf absorbs whatever
@@ -153,7 +171,7 @@ template <bool SIGNED>
 __device__ __forceinline__ Elem<SIGNED> state_elem(float log_mag, uint32_t sign_mask) {
     Elem<SIGNED> e;
     e.A = neg_inf();
-    e.m = log_mag;
+    e.m = fmaxf(log_mag, kEmpty);
     e.s = (log_mag == neg_inf()) ? 0.0f : (SIGNED ? flip(1.0f, sign_mask) : 1.0f);
     e.p = 0u;
     return e;
@@ -165,8 +183,8 @@ template <bool SIGNED>
 __device__ __forceinline__ void renormalise(Elem<SIGNED>& e) {
     if (!SIGNED) return;
     const float as = fabsf(e.s);
-    if (as == 0.0f) { e.m = neg_inf(); e.s = 0.0f; return; }
-    if (as >= 1.17549435e-38f && e.m != neg_inf()) {
+    if (as == 0.0f) { e.m = kEmpty; e.s = 0.0f; return; }
+    if (as >= 1.17549435e-38f) {
         const int ex = ((__float_as_int(as) >> 23) & 0xff) - 127;
         e.m = fmaf((float)ex, kLn2, e.m);
         e.s = __int_as_float(__float_as_int(e.s) - (ex << 23));
@@ -174,16 +192,16 @@ __device__ __forceinline__ void renormalise(Elem<SIGNED>& e) {
 }
 
 // ------------------------------------------------------------------------------------------
-// Shared-memory chunk layout.  A chunk is 32 lanes x K consecutive elements of one row, kept
-// as rows of 128 bytes with the 16-byte units of each row XOR-swizzled by (row & 7) -- the
-// layout TMA's 128-byte swizzle writes -- so that a lane reading its own K contiguous
-// elements with 128-bit loads is bank-conflict free.
-__device__ __forceinline__ uint32_t swz_unit(uint32_t unit) {  // unit = index of a 16-byte unit in the chunk
-    const uint32_t row = unit >> 3;
-    return (row << 7) + (((unit & 7u) ^ (row & 7u)) << 4);
-}
-__device__ __forceinline__ uint32_t swz_byte(uint32_t byte_off) {
-    return swz_unit(byte_off >> 4) + (byte_off & 15u);
+// Shared-memory chunk layout.  A warp's chunk is R rows x (32/R lanes x K elements): every row
+// contributes one contiguous piece, fetched by TMA as boxes of {128 bytes, R rows} with the
+// 128-byte swizzle.  Box b of a chunk lands at byte b*R*128; inside, row g of the box is the
+// shared-memory row b*R+g, whose 16-byte units are XORed with (row & 7).  A lane reading its own
+// K contiguous elements with 128-bit loads is then bank-conflict free (the 8 lanes of a
+// wavefront fall on 8 different unit positions).
+// byte_in_row: byte offset inside the row's piece of the chunk.
+__device__ __forceinline__ uint32_t chunk_off(int R, int g, uint32_t byte_in_row) {
+    const uint32_t srow = (byte_in_row >> 7) * (uint32_t)R + (uint32_t)g;
+    return (srow << 7) + (((((byte_in_row >> 4) ^ srow) & 7u)) << 4) + (byte_in_row & 15u);
 }
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -210,11 +228,11 @@ struct Storage<float> {
     }
     __device__ static __forceinline__ float load(const void* p, int64_t i) { return ((const float*)p)[i]; }
     __device__ static __forceinline__ void store(void* p, int64_t i, float v) { ((float*)p)[i] = v; }
-    __device__ static __forceinline__ float from_smem(const uint8_t* base, uint32_t i) {
-        return *(const float*)(base + swz_byte(i * 4u));
+    __device__ static __forceinline__ float from_smem(const uint8_t* base, uint32_t off) {
+        return *(const float*)(base + off);
     }
-    __device__ static __forceinline__ void to_smem(uint8_t* base, uint32_t i, float v) {
-        *(float*)(base + swz_byte(i * 4u)) = v;
+    __device__ static __forceinline__ void to_smem(uint8_t* base, uint32_t off, float v) {
+        *(float*)(base + off) = v;
     }
 };
 template <>
@@ -239,11 +257,11 @@ struct Storage<__nv_bfloat16> {
     __device__ static __forceinline__ void store(void* p, int64_t i, float v) {
         ((__nv_bfloat16*)p)[i] = __float2bfloat16_rn(v);
     }
-    __device__ static __forceinline__ float from_smem(const uint8_t* base, uint32_t i) {
-        return __bfloat162float(*(const __nv_bfloat16*)(base + swz_byte(i * 2u)));
+    __device__ static __forceinline__ float from_smem(const uint8_t* base, uint32_t off) {
+        return __bfloat162float(*(const __nv_bfloat16*)(base + off));
     }
-    __device__ static __forceinline__ void to_smem(uint8_t* base, uint32_t i, float v) {
-        *(__nv_bfloat16*)(base + swz_byte(i * 2u)) = __float2bfloat16_rn(v);
+    __device__ static __forceinline__ void to_smem(uint8_t* base, uint32_t off, float v) {
+        *(__nv_bfloat16*)(base + off) = __float2bfloat16_rn(v);
     }
 };
 
@@ -268,6 +286,7 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 }
 // Bounded wait: returns false when the limit ran out (the caller records an error and leaves).
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t limit) {
+#pragma unroll 1
     for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
     }
@@ -276,7 +295,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
 __device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-// One 2-D tiled TMA load (no multicast) of a {box_x, 1} box into shared memory.
+// One 2-D tiled TMA load (no multicast) of one box into shared memory.
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* tmap, int32_t x, int32_t y, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
@@ -321,14 +340,15 @@ struct Run {
     float r;        // reference of the run, -inf when the run has no non-zero b
     bool bad;       // the fast form does not apply to this run (a_t = 0, inf or NaN in it)
 
-    // Load the lane's K inputs of both tensors from the swizzled chunk.
-    __device__ __forceinline__ static void load(const uint8_t* sm_a, const uint8_t* sm_b, int lane, float* va, float* vb) {
+    // Load the lane's K inputs of both tensors from the swizzled chunk; `off` holds the lane's
+    // IN_UNITS unit offsets (chunk_off), computed once per kernel.
+    __device__ __forceinline__ static void load(const uint8_t* sm_a, const uint8_t* sm_b, const uint32_t* off, float* va,
+                                                float* vb) {
         const uint32_t base_a = smem_u32(sm_a), base_b = smem_u32(sm_b);
 #pragma unroll
         for (int j = 0; j < IN_UNITS; ++j) {
-            const uint32_t off = swz_unit((uint32_t)(lane * IN_UNITS + j));
-            Storage<TIn>::unpack(lds128(base_a + off), va + j * Storage<TIn>::kPerUnit);
-            Storage<TIn>::unpack(lds128(base_b + off), vb + j * Storage<TIn>::kPerUnit);
+            Storage<TIn>::unpack(lds128(base_a + off[j]), va + j * Storage<TIn>::kPerUnit);
+            Storage<TIn>::unpack(lds128(base_b + off[j]), vb + j * Storage<TIn>::kPerUnit);
         }
     }
 
@@ -377,7 +397,7 @@ struct Run {
         }
         E agg;
         agg.A = acc;
-        agg.m = rr + acc;
+        agg.m = fmaxf(rr + acc, kEmpty);
         agg.s = SIGNED ? flip(sum, par) : sum;  // beta = alpha * (sum relative to the run start)
         agg.p = par;
         return agg;
@@ -388,16 +408,14 @@ struct Run {
     // Returns false when an early prefix is too small relative to the run's reference for the
     // fast form to be trusted (the caller then redoes the chunk with the tracked form).
     __device__ __forceinline__ bool apply(const E& entering, float* out_mag, uint32_t* out_sign) const {
-        const float Mc = entering.m, Sc = entering.s;
-        float M = fmaxf(Mc, r);
+        const float Mc = entering.m, Sc = entering.s;  // Mc is finite (>= kEmpty); r may be -inf
+        const float M = fmaxf(Mc, r);
         const float d = Mc - r;
         const float ed = ex2(-fabsf(d) * kLog2e);
-        float C = (d >= 0.0f) ? Sc : Sc * ed;
-        float w = (d >= 0.0f) ? ed : 1.0f;
-        const bool empty = (M == neg_inf());
-        if (empty) { C = 0.0f; w = 0.0f; M = 0.0f; }
+        const float C = (d >= 0.0f) ? Sc : Sc * ed;
+        const float w = (d >= 0.0f) ? ed : 1.0f;
         const float S1 = fmaf(s[0], w, C);
-        const bool ok = empty || (fabsf(S1) >= 8.67361738e-19f /* 2^-60 */);
+        const bool ok = (fabsf(S1) >= 8.67361738e-19f /* 2^-60 */) || (Sc == 0.0f && r == neg_inf());
 #pragma unroll
         for (int t = 0; t < K; ++t) {
             const float S = fmaf(s[t], w, C);
@@ -424,12 +442,9 @@ struct Run {
 template <int MODE, typename TIn>
 struct Leaf {
     static constexpr bool SIGNED = (MODE != kLogUnsigned);
-    // Element t (0..CHUNK-1) of the chunk as a one-step part.
-    __device__ static __forceinline__ Elem<SIGNED> get(const uint8_t* sm_a, const uint8_t* sm_b, uint32_t i,
-                                                       uint32_t sa, uint32_t sb) {
+    // One element (stored values va, vb; sign masks sa, sb for kLogSigned) as a one-step part.
+    __device__ static __forceinline__ Elem<SIGNED> get(float va, float vb, uint32_t sa, uint32_t sb) {
         Elem<SIGNED> e;
-        const float va = Storage<TIn>::from_smem(sm_a, i);
-        const float vb = Storage<TIn>::from_smem(sm_b, i);
         float lb;
         uint32_t psb;
         if (MODE == kLinear) {
@@ -443,7 +458,7 @@ struct Leaf {
             lb = vb;
             psb = SIGNED ? sb : 0u;
         }
-        e.m = lb;
+        e.m = fmaxf(lb, kEmpty);
         e.s = (lb == neg_inf()) ? 0.0f : (SIGNED ? flip(1.0f, psb) : 1.0f);
         return e;
     }

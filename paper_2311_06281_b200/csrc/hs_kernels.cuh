@@ -48,6 +48,7 @@ struct Params {
     int nchunks;        // chunks per row
     int stages;         // input stages per warp (2..kMaxStages)
     int sign_vec_ok;    // sign tensors may be accessed with 16-byte vectors
+    int rows_per_warp;  // R: rows held by one warp of the batched kernel (1, 2, 4, 8); look-back: 1
     unsigned long long call_id;
     Header* ws;
     // look-back kernel only
@@ -76,161 +77,191 @@ __device__ __forceinline__ float neutral_a() { return MODE == kLinear ? 1.0f : 0
 template <int MODE>
 __device__ __forceinline__ float neutral_b() { return MODE == kLinear ? 0.0f : neg_inf(); }
 
+// Where a lane sits in its warp's chunk: the warp holds R rows, lane = i*R + g is segment i
+// (K consecutive elements) of row g; a row's piece of the chunk is W = (32/R)*K elements wide.
+struct LaneMap {
+    int R;     // rows per warp: 1, 2, 4 or 8
+    int g;     // row within the warp's group
+    int i;     // segment within the row's piece
+    int W;     // elements per row per chunk
+};
+
 // ------------------------------------------------------------------------------------------
 // Per-warp chunk engine shared by both kernels: everything between "the chunk's inputs are in
 // shared memory" and "the chunk's outputs are in shared memory".
 template <int MODE, typename TIn, typename TOut, int K>
 struct ChunkEngine {
-    using R = Run<MODE, TIn, TOut, K>;
-    static constexpr bool SIGNED = R::SIGNED;
+    using R_ = Run<MODE, TIn, TOut, K>;
+    static constexpr bool SIGNED = R_::SIGNED;
     using E = Elem<SIGNED>;
+    static constexpr int IN_UNITS = R_::IN_UNITS;
+    static constexpr int OUT_UNITS = R_::OUT_UNITS;
 
-    // sign masks of the lane's K elements from a uint8 tensor (0/1 per element)
-    __device__ static __forceinline__ void load_signs(const uint8_t* g, long long base, long long col0, long long n,
-                                                      bool vec, uint32_t* mask) {
+    struct Offsets {
+        uint32_t in[IN_UNITS];    // the lane's 16-byte input units inside a stage
+        uint32_t out[OUT_UNITS];  // the lane's 16-byte output units inside an output buffer
+    };
+    __device__ static __forceinline__ Offsets offsets(const LaneMap& lm) {
+        Offsets o;
+#pragma unroll
+        for (int j = 0; j < IN_UNITS; ++j) o.in[j] = chunk_off(lm.R, lm.g, (uint32_t)((lm.i * IN_UNITS + j) * 16));
+#pragma unroll
+        for (int j = 0; j < OUT_UNITS; ++j) o.out[j] = chunk_off(lm.R, lm.g, (uint32_t)((lm.i * OUT_UNITS + j) * 16));
+        return o;
+    }
+
+    // sign masks of the lane's K elements from a uint8 tensor (0/1 per element); idx0 = index of
+    // the lane's first element, `left` = elements of the row from there on (may be <= 0).
+    __device__ static __forceinline__ void load_signs(const uint8_t* g, long long idx0, long long left, bool vec,
+                                                      uint32_t* mask) {
         if (g == nullptr) {
 #pragma unroll
             for (int t = 0; t < K; ++t) mask[t] = 0u;
             return;
         }
-        if (vec && col0 + K <= n) {
+        if (vec && left >= K) {
 #pragma unroll
             for (int j = 0; j < K / 16; ++j) {
-                const uint4 v = __ldg(reinterpret_cast<const uint4*>(g + base + col0 + 16 * j));
+                const uint4 v = __ldg(reinterpret_cast<const uint4*>(g + idx0 + 16 * j));
                 const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
                 for (int t = 0; t < 16; ++t) mask[16 * j + t] = (w[t >> 2] << (31 - 8 * (t & 3))) & kSignBit;
             }
         } else {
 #pragma unroll
-            for (int t = 0; t < K; ++t) mask[t] = (col0 + t < n) ? (((uint32_t)g[base + col0 + t] & 1u) << 31) : 0u;
+            for (int t = 0; t < K; ++t) mask[t] = (t < left) ? (((uint32_t)g[idx0 + t] & 1u) << 31) : 0u;
         }
     }
-    __device__ static __forceinline__ void store_signs(uint8_t* g, long long base, long long col0, long long n,
-                                                       bool vec, const uint32_t* mask) {
-        if (vec && col0 + K <= n) {
+    __device__ static __forceinline__ void store_signs(uint8_t* g, long long idx0, long long left, bool vec,
+                                                       const uint32_t* mask) {
+        if (vec && left >= K) {
 #pragma unroll
             for (int j = 0; j < K / 16; ++j) {
                 uint32_t w[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
                 for (int t = 0; t < 16; ++t) w[t >> 2] |= (mask[16 * j + t] >> 31) << (8 * (t & 3));
-                *reinterpret_cast<uint4*>(g + base + col0 + 16 * j) = make_uint4(w[0], w[1], w[2], w[3]);
+                *reinterpret_cast<uint4*>(g + idx0 + 16 * j) = make_uint4(w[0], w[1], w[2], w[3]);
             }
         } else {
 #pragma unroll
             for (int t = 0; t < K; ++t)
-                if (col0 + t < n) g[base + col0 + t] = (uint8_t)(mask[t] >> 31);
+                if (t < left) g[idx0 + t] = (uint8_t)(mask[t] >> 31);
         }
     }
 
     // Tracked form, pass 1: the lane's run as one part, every step with its own reference.
-    __device__ static __noinline__ E slow_pass1(const uint8_t* sm_a, const uint8_t* sm_b, int lane, const uint8_t* gsa,
-                                                const uint8_t* gsb, long long gbase, int valid) {
+    // idx0/left as above (`left` <= 0: the run lies wholly beyond the row).
+    __device__ static __noinline__ E slow_pass1(const uint8_t* sm_a, const uint8_t* sm_b, LaneMap lm, const uint8_t* gsa,
+                                                const uint8_t* gsb, long long idx0, long long left) {
         E e = identity_elem<SIGNED>();
         for (int t = 0; t < K; ++t) {
-            const int i = lane * K + t;
-            if (i < valid) {
-                const uint32_t sa = gsa ? (((uint32_t)gsa[gbase + i] & 1u) << 31) : 0u;
-                const uint32_t sb = gsb ? (((uint32_t)gsb[gbase + i] & 1u) << 31) : 0u;
-                e = compose(e, Leaf<MODE, TIn>::get(sm_a, sm_b, (uint32_t)i, sa, sb));
+            if (t < left) {
+                const uint32_t off = chunk_off(lm.R, lm.g, (uint32_t)((lm.i * K + t) * sizeof(TIn)));
+                const uint32_t sa = gsa ? (((uint32_t)gsa[idx0 + t] & 1u) << 31) : 0u;
+                const uint32_t sb = gsb ? (((uint32_t)gsb[idx0 + t] & 1u) << 31) : 0u;
+                e = compose(e, Leaf<MODE, TIn>::get(Storage<TIn>::from_smem(sm_a, off), Storage<TIn>::from_smem(sm_b, off),
+                                                    sa, sb));
             }
         }
         return e;
     }
-    // Tracked form, pass 2: step the value through the lane's run and write each output.
-    __device__ static __noinline__ void slow_apply(E st, const uint8_t* sm_a, const uint8_t* sm_b, uint8_t* sm_out,
-                                                   int lane, const uint8_t* gsa, const uint8_t* gsb, uint8_t* gsx,
-                                                   long long gbase, int valid) {
+    struct SlowOut {
+        float vals[K];
+        uint32_t sgn[MODE == kLogSigned ? K : 1];
+    };
+    // Tracked form, pass 2: step the value through the lane's run; returns outputs (and signs).
+    __device__ static __noinline__ SlowOut slow_apply(E st, const uint8_t* sm_a, const uint8_t* sm_b, LaneMap lm,
+                                                      const uint8_t* gsa, const uint8_t* gsb, long long idx0,
+                                                      long long left) {
+        SlowOut so;
         for (int t = 0; t < K; ++t) {
-            const int i = lane * K + t;
-            if (i < valid) {
-                const uint32_t sa = gsa ? (((uint32_t)gsa[gbase + i] & 1u) << 31) : 0u;
-                const uint32_t sb = gsb ? (((uint32_t)gsb[gbase + i] & 1u) << 31) : 0u;
-                st = compose(st, Leaf<MODE, TIn>::get(sm_a, sm_b, (uint32_t)i, sa, sb));
+            float v = 0.0f;
+            uint32_t sg = 0u;
+            if (t < left) {
+                const uint32_t off = chunk_off(lm.R, lm.g, (uint32_t)((lm.i * K + t) * sizeof(TIn)));
+                const uint32_t sa = gsa ? (((uint32_t)gsa[idx0 + t] & 1u) << 31) : 0u;
+                const uint32_t sb = gsb ? (((uint32_t)gsb[idx0 + t] & 1u) << 31) : 0u;
+                st = compose(st, Leaf<MODE, TIn>::get(Storage<TIn>::from_smem(sm_a, off), Storage<TIn>::from_smem(sm_b, off),
+                                                     sa, sb));
                 renormalise(st);
-                float v;
                 if (MODE == kLinear) {
                     const float h = ex2(st.m * (0.5f * kLog2e));
-                    v = (st.s * h) * h;
-                    if (st.s == 0.0f) v = 0.0f;
+                    v = (st.s == 0.0f) ? 0.0f : (st.s * h) * h;
                 } else {
-                    v = fmaf(lg2(fabsf(st.s)), kLn2, st.m);
-                    if (st.s == 0.0f) v = neg_inf();
+                    v = (st.s == 0.0f) ? neg_inf() : fmaf(lg2(fabsf(st.s)), kLn2, st.m);
+                    sg = (st.s < 0.0f) ? kSignBit : 0u;
                 }
-                Storage<TOut>::to_smem(sm_out, (uint32_t)i, v);
-                if (MODE == kLogSigned && gsx) gsx[gbase + i] = (st.s < 0.0f) ? 1 : 0;
             }
+            so.vals[t] = v;
+            if (MODE == kLogSigned) so.sgn[t] = sg;
         }
+        return so;
     }
 
-    // Runs the chunk.  `entering_chunk` is the value of x entering the chunk when `known` is
-    // true (batched kernel).  Returns the chunk's aggregate through `total`; writes outputs to
-    // sm_out.  The look-back kernel calls the two halves separately (see below).
     struct Pending {  // what phase 2 needs from phase 1
-        R run;
-        E excl;       // parts of this chunk before the lane's run
+        R_ run;
+        E excl;       // parts of this row's chunk before the lane's run
         bool slow;
     };
 
-    __device__ static __forceinline__ void phase1(const Params& p, const uint8_t* sm_a, const uint8_t* sm_b, int lane,
-                                                  long long row, int chunk, Pending& pd, E& total) {
+    // Phase 1: inputs from shared memory, the lane's run, the scan over the lanes of the row.
+    // `row` is the lane's row (may be >= rows for a padded group), col0 its first column.
+    __device__ static __forceinline__ void phase1(const Params& p, const uint8_t* sm_a, const uint8_t* sm_b,
+                                                  const Offsets& off, const LaneMap& lm, int lane, long long row,
+                                                  long long col0, Pending& pd, E& total) {
         float va[K], vb[K];
-        uint32_t sa[SIGNED ? K : 1], sb[SIGNED ? K : 1];
-        R::load(sm_a, sm_b, lane, va, vb);
-        const long long col0 = (long long)chunk * R::CHUNK + lane * K;
-        const long long gbase = row * p.n;
-        if ((long long)(chunk + 1) * R::CHUNK > p.n) {
+        uint32_t sa[MODE == kLogSigned ? K : 1], sb[MODE == kLogSigned ? K : 1];
+        R_::load(sm_a, sm_b, off.in, va, vb);
+        const long long left = (row < p.rows) ? p.n - col0 : 0;
+        if (left < K) {
 #pragma unroll
             for (int t = 0; t < K; ++t) {
-                if (col0 + t >= p.n) { va[t] = neutral_a<MODE>(); vb[t] = neutral_b<MODE>(); }
+                if (t >= left) { va[t] = neutral_a<MODE>(); vb[t] = neutral_b<MODE>(); }
             }
         }
         if (MODE == kLogSigned) {
-            load_signs(p.sign_a, gbase, col0, p.n, p.sign_vec_ok != 0, sa);
-            load_signs(p.sign_b, gbase, col0, p.n, p.sign_vec_ok != 0, sb);
+            load_signs(p.sign_a, row * p.n + col0, left, p.sign_vec_ok != 0, sa);
+            load_signs(p.sign_b, row * p.n + col0, left, p.sign_vec_ok != 0, sb);
         }
         E agg = pd.run.pass1(va, vb, sa, sb);
         pd.slow = __any_sync(0xffffffffu, pd.run.bad);
         if (pd.slow) {
-            const long long rem = p.n - (long long)chunk * R::CHUNK;
-            const int valid = rem < R::CHUNK ? (int)rem : R::CHUNK;
-            agg = slow_pass1(sm_a, sm_b, lane, MODE == kLogSigned ? p.sign_a : nullptr,
-                             MODE == kLogSigned ? p.sign_b : nullptr, gbase + (long long)chunk * R::CHUNK, valid);
+            agg = slow_pass1(sm_a, sm_b, lm, MODE == kLogSigned ? p.sign_a : nullptr,
+                             MODE == kLogSigned ? p.sign_b : nullptr, row * p.n + col0, left);
         }
-        warp_scan(agg, lane, pd.excl, total);
+        row_scan(agg, lane, lm.R, pd.excl, total);
     }
 
-    // `entering_chunk`: value of x entering the chunk.
+    // Phase 2: `entering_row` is the value of x entering this row's piece of the chunk.
     __device__ static __forceinline__ void phase2(const Params& p, const uint8_t* sm_a, const uint8_t* sm_b,
-                                                  uint8_t* sm_out, int lane, long long row, int chunk,
-                                                  const Pending& pd, const E& entering_chunk) {
-        const E entering = compose(entering_chunk, pd.excl);
-        const long long col0 = (long long)chunk * R::CHUNK + lane * K;
-        const long long gbase = row * p.n;
+                                                  uint8_t* sm_out, const Offsets& off, const LaneMap& lm, long long row,
+                                                  long long col0, const Pending& pd, const E& entering_row) {
+        const E entering = compose(entering_row, pd.excl);
+        const long long left = (row < p.rows) ? p.n - col0 : 0;
+        const uint32_t ob = smem_u32(sm_out);
         float out_mag[K];
         uint32_t out_sign[MODE == kLogSigned ? K : 1];
         bool ok = false;
         if (!pd.slow) ok = pd.run.apply(entering, out_mag, out_sign);
         ok = __all_sync(0xffffffffu, ok);
         if (ok) {
-            const uint32_t ob = smem_u32(sm_out);
 #pragma unroll
-            for (int j = 0; j < R::OUT_UNITS; ++j) {
-                sts128(ob + swz_unit((uint32_t)(lane * R::OUT_UNITS + j)),
-                       Storage<TOut>::pack(out_mag + j * Storage<TOut>::kPerUnit));
-            }
-            if (MODE == kLogSigned) store_signs(p.sign_x, gbase, col0, p.n, p.sign_vec_ok != 0, out_sign);
+            for (int j = 0; j < OUT_UNITS; ++j)
+                sts128(ob + off.out[j], Storage<TOut>::pack(out_mag + j * Storage<TOut>::kPerUnit));
+            if (MODE == kLogSigned) store_signs(p.sign_x, row * p.n + col0, left, p.sign_vec_ok != 0, out_sign);
         } else {
-            const long long rem = p.n - (long long)chunk * R::CHUNK;
-            const int valid = rem < R::CHUNK ? (int)rem : R::CHUNK;
-            slow_apply(entering, sm_a, sm_b, sm_out, lane, MODE == kLogSigned ? p.sign_a : nullptr,
-                       MODE == kLogSigned ? p.sign_b : nullptr, MODE == kLogSigned ? p.sign_x : nullptr,
-                       gbase + (long long)chunk * R::CHUNK, valid);
+            const SlowOut so = slow_apply(entering, sm_a, sm_b, lm, MODE == kLogSigned ? p.sign_a : nullptr,
+                                          MODE == kLogSigned ? p.sign_b : nullptr, row * p.n + col0, left);
+#pragma unroll
+            for (int j = 0; j < OUT_UNITS; ++j)
+                sts128(ob + off.out[j], Storage<TOut>::pack(so.vals + j * Storage<TOut>::kPerUnit));
+            if (MODE == kLogSigned) store_signs(p.sign_x, row * p.n + col0, left, p.sign_vec_ok != 0, so.sgn);
         }
     }
 
     // Value of x_0 of a row as the element that starts the second scan (Eq. 7's cat(log x_0, .)).
     __device__ static __forceinline__ E row_start(const Params& p, long long row) {
+        if (row >= p.rows) return state_elem<SIGNED>(neg_inf(), 0u);
         const float v = Storage<TIn>::load(p.x0, row);
         if (MODE == kLinear) return state_elem<SIGNED>(log_abs_accurate(v), __float_as_uint(v) & kSignBit);
         uint32_t sg = 0u;
@@ -239,22 +270,27 @@ struct ChunkEngine {
     }
 
     // Plain-load staging for rows that TMA cannot address (unaligned base or row pitch).
-    __device__ static __forceinline__ void generic_load(const Params& p, uint8_t* sm_a, uint8_t* sm_b, int lane,
-                                                        long long row, int chunk) {
-        const long long gbase = row * p.n;
-        for (int i = lane; i < R::CHUNK; i += 32) {
-            const long long col = (long long)chunk * R::CHUNK + i;
-            const bool in = col < p.n;
-            Storage<TIn>::to_smem(sm_a, (uint32_t)i, in ? Storage<TIn>::load(p.in_a, gbase + col) : neutral_a<MODE>());
-            Storage<TIn>::to_smem(sm_b, (uint32_t)i, in ? Storage<TIn>::load(p.in_b, gbase + col) : neutral_b<MODE>());
+    // row0: first row of the warp's group, colbase: first column of the chunk.
+    __device__ static __forceinline__ void generic_load(const Params& p, uint8_t* sm_a, uint8_t* sm_b, const LaneMap& lm,
+                                                        int lane, long long row0, long long colbase) {
+        for (int e = lane; e < 32 * K; e += 32) {
+            const int rg = e / lm.W, c = e - rg * lm.W;
+            const long long row = row0 + rg, col = colbase + c;
+            const bool in = row < p.rows && col < p.n;
+            const uint32_t off = chunk_off(lm.R, rg, (uint32_t)(c * sizeof(TIn)));
+            Storage<TIn>::to_smem(sm_a, off, in ? Storage<TIn>::load(p.in_a, row * p.n + col) : neutral_a<MODE>());
+            Storage<TIn>::to_smem(sm_b, off, in ? Storage<TIn>::load(p.in_b, row * p.n + col) : neutral_b<MODE>());
         }
     }
-    __device__ static __forceinline__ void generic_store(const Params& p, const uint8_t* sm_out, int lane, long long row,
-                                                         int chunk) {
-        const long long gbase = row * p.n;
-        for (int i = lane; i < R::CHUNK; i += 32) {
-            const long long col = (long long)chunk * R::CHUNK + i;
-            if (col < p.n) Storage<TOut>::store(p.out, gbase + col, Storage<TOut>::from_smem(sm_out, (uint32_t)i));
+    __device__ static __forceinline__ void generic_store(const Params& p, const uint8_t* sm_out, const LaneMap& lm, int lane,
+                                                         long long row0, long long colbase) {
+        for (int e = lane; e < 32 * K; e += 32) {
+            const int rg = e / lm.W, c = e - rg * lm.W;
+            const long long row = row0 + rg, col = colbase + c;
+            if (row < p.rows && col < p.n) {
+                const uint32_t off = chunk_off(lm.R, rg, (uint32_t)(c * sizeof(TOut)));
+                Storage<TOut>::store(p.out, row * p.n + col, Storage<TOut>::from_smem(sm_out, off));
+            }
         }
     }
 };
@@ -270,20 +306,26 @@ __host__ __device__ constexpr int warp_smem_bytes(int stages) {
 }
 
 // Per-warp asynchronous chunk pipeline: TMA loads into a ring of input stages, TMA stores from
-// two output buffers.  Lane r moves the r-th 128-byte row of a chunk.
+// two output buffers.  A chunk is moved as boxes of {128 bytes, R rows}; lane b moves box b.
 template <typename TIn, typename TOut, int K>
 struct WarpPipe {
     static constexpr int IN_BYTES = 32 * K * (int)sizeof(TIn);
     static constexpr int OUT_BYTES = 32 * K * (int)sizeof(TOut);
-    static constexpr int IN_ROWS = IN_BYTES / 128;
-    static constexpr int OUT_ROWS = OUT_BYTES / 128;
-    static constexpr int IN_PER_ROW = 128 / (int)sizeof(TIn);
-    static constexpr int OUT_PER_ROW = 128 / (int)sizeof(TOut);
+    static constexpr int IN_PER_BOX = 128 / (int)sizeof(TIn);    // elements of a row in one box
+    static constexpr int OUT_PER_BOX = 128 / (int)sizeof(TOut);
     uint8_t* base;   // this warp's shared memory
     uint32_t bars;   // shared address of this warp's mbarriers
     int stages;
     int lane;
+    int R;           // rows per box
+    int in_boxes;    // boxes per tensor per chunk, input / output
+    int out_boxes;
 
+    __device__ __forceinline__ void setup(int rows_per_warp) {
+        R = rows_per_warp;
+        in_boxes = IN_BYTES / (128 * R);
+        out_boxes = OUT_BYTES / (128 * R);
+    }
     __device__ __forceinline__ uint8_t* in_a(int s) const { return base + s * 2 * IN_BYTES; }
     __device__ __forceinline__ uint8_t* in_b(int s) const { return base + s * 2 * IN_BYTES + IN_BYTES; }
     __device__ __forceinline__ uint8_t* out(int o) const { return base + stages * 2 * IN_BYTES + o * OUT_BYTES; }
@@ -295,14 +337,17 @@ struct WarpPipe {
         }
         __syncwarp();
     }
-    __device__ __forceinline__ void issue(const CUtensorMap* tm_a, const CUtensorMap* tm_b, long long row, int chunk, int s) {
+    // row0: first row of the group; colbase: first column of the chunk
+    __device__ __forceinline__ void issue(const CUtensorMap* tm_a, const CUtensorMap* tm_b, long long row0, long long colbase,
+                                          int s) {
         const uint32_t bar = bars + 8 * s;
         if (lane == 0) mbar_expect_tx(bar, 2 * IN_BYTES);
         __syncwarp();
-        if (lane < IN_ROWS) {
-            const int x = chunk * (32 * K) + lane * IN_PER_ROW;
-            tma_load_2d(smem_u32(in_a(s)) + lane * 128, tm_a, x, (int)row, bar);
-            tma_load_2d(smem_u32(in_b(s)) + lane * 128, tm_b, x, (int)row, bar);
+        if (lane < in_boxes) {
+            const int x = (int)colbase + lane * IN_PER_BOX;
+            const uint32_t dst = (uint32_t)(lane * R * 128);
+            tma_load_2d(smem_u32(in_a(s)) + dst, tm_a, x, (int)row0, bar);
+            tma_load_2d(smem_u32(in_b(s)) + dst, tm_b, x, (int)row0, bar);
         }
     }
     __device__ __forceinline__ bool wait(int s, uint32_t parity) const {
@@ -310,20 +355,20 @@ struct WarpPipe {
     }
     // before writing output buffer o: the store issued from it two chunks ago has been read
     __device__ __forceinline__ void acquire_out() const {
-        if (lane < OUT_ROWS) bulk_wait_read<1>();
+        if (lane < out_boxes) bulk_wait_read<1>();
         __syncwarp();
     }
-    __device__ __forceinline__ void store(const CUtensorMap* tm_o, long long row, int chunk, int o) const {
+    __device__ __forceinline__ void store(const CUtensorMap* tm_o, long long row0, long long colbase, int o) const {
         fence_async_smem();
         __syncwarp();
-        if (lane < OUT_ROWS) {
-            const int x = chunk * (32 * K) + lane * OUT_PER_ROW;
-            tma_store_2d(tm_o, x, (int)row, smem_u32(out(o)) + lane * 128);
+        if (lane < out_boxes) {
+            const int x = (int)colbase + lane * OUT_PER_BOX;
+            tma_store_2d(tm_o, x, (int)row0, smem_u32(out(o)) + (uint32_t)(lane * R * 128));
             bulk_commit();
         }
     }
     __device__ __forceinline__ void drain() const {
-        if (lane < OUT_ROWS) bulk_wait_all();
+        if (lane < out_boxes) bulk_wait_all();
         __syncwarp();
     }
     // Error exit: loads `consumed`..`issued`-1 are still in flight into this warp's stages; give
@@ -334,7 +379,9 @@ struct WarpPipe {
 };
 
 // ------------------------------------------------------------------------------------------
-// (a) Row-batched kernel.  Persistent: warp g of G handles rows g, g+G, g+2G, ...
+// (a) Row-batched kernel.  Persistent: warp w of G handles the row groups w, w+G, w+2G, ...; a
+// group is R consecutive rows (p.rows_per_warp), each walked chunk by chunk by 32/R lanes with
+// the value of x carried in registers.
 template <int MODE, typename TIn, typename TOut, int K, bool TMA>
 __global__ void __launch_bounds__(512, 1)
 batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
@@ -346,44 +393,56 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const int S = TMA ? p.stages : 1;
     const int per_warp = warp_smem_bytes<MODE, TIn, TOut, K>(S);
+    const int R = p.rows_per_warp;
+
+    LaneMap lm;
+    lm.R = R;
+    lm.g = lane & (R - 1);
+    lm.i = lane / R;
+    lm.W = (32 / R) * K;
+    const typename CE::Offsets off = CE::offsets(lm);
 
     WarpPipe<TIn, TOut, K> pipe;
     pipe.base = smem + warp * per_warp;
     pipe.bars = smem_u32(smem + nwarps * per_warp) + warp * (8 * kMaxStages);
     pipe.stages = S;
     pipe.lane = lane;
+    pipe.setup(R);
     if (TMA) pipe.init();
 
     if (blockIdx.x == 0 && threadIdx.x == 0) p.ws->started_id = p.call_id;
 
     const long long gw = (long long)blockIdx.x * nwarps + warp;
     const long long GW = (long long)gridDim.x * nwarps;
-    if (gw >= p.rows) return;
-    const long long my_rows = (p.rows - gw + GW - 1) / GW;
-    const long long items = my_rows * p.nchunks;
+    const long long groups = (p.rows + R - 1) / R;
+    if (gw >= groups) return;
+    const long long my_groups = (groups - gw + GW - 1) / GW;
+    const long long items = my_groups * p.nchunks;
 
     // producer cursor
-    long long prow = gw;
+    long long pgroup = gw;
     int pchunk = 0;
     long long issued = 0;
     if (TMA) {
         for (; issued < S - 1 && issued < items; ++issued) {
-            pipe.issue(&tm_a, &tm_b, prow, pchunk, (int)(issued % S));
-            if (++pchunk == p.nchunks) { pchunk = 0; prow += GW; }
+            pipe.issue(&tm_a, &tm_b, pgroup * R, (long long)pchunk * lm.W, (int)(issued % S));
+            if (++pchunk == p.nchunks) { pchunk = 0; pgroup += GW; }
         }
     }
 
-    long long row = gw;
+    long long group = gw;
     int chunk = 0;
+    long long row = group * R + lm.g;
     E state = CE::row_start(p, row);
     int stage = 0;
     uint32_t parity = 0;
     for (long long q = 0; q < items; ++q) {
+        const long long colbase = (long long)chunk * lm.W;
         if (TMA) {
             if (issued < items) {
-                pipe.issue(&tm_a, &tm_b, prow, pchunk, (int)(issued % S));
+                pipe.issue(&tm_a, &tm_b, pgroup * R, (long long)pchunk * lm.W, (int)(issued % S));
                 ++issued;
-                if (++pchunk == p.nchunks) { pchunk = 0; prow += GW; }
+                if (++pchunk == p.nchunks) { pchunk = 0; pgroup += GW; }
             }
             if (!pipe.wait(stage, parity)) {
                 if (lane == 0) record_error(p, kErrCopyTimeout, row);
@@ -391,33 +450,35 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
                 break;
             }
         } else {
-            CE::generic_load(p, pipe.in_a(0), pipe.in_b(0), lane, row, chunk);
+            CE::generic_load(p, pipe.in_a(0), pipe.in_b(0), lm, lane, group * R, colbase);
             __syncwarp();
         }
         const uint8_t* sm_a = pipe.in_a(stage);
         const uint8_t* sm_b = pipe.in_b(stage);
         uint8_t* sm_out = pipe.out((int)(q & 1));
+        const long long col0 = colbase + lm.i * K;
 
         typename CE::Pending pd;
         E total;
-        CE::phase1(p, sm_a, sm_b, lane, row, chunk, pd, total);
+        CE::phase1(p, sm_a, sm_b, off, lm, lane, row, col0, pd, total);
         if (TMA) pipe.acquire_out();
-        CE::phase2(p, sm_a, sm_b, sm_out, lane, row, chunk, pd, state);
+        CE::phase2(p, sm_a, sm_b, sm_out, off, lm, row, col0, pd, state);
         state = compose(state, total);
         renormalise(state);
 
         if (TMA) {
-            pipe.store(&tm_o, row, chunk, (int)(q & 1));
+            pipe.store(&tm_o, group * R, colbase, (int)(q & 1));
         } else {
             __syncwarp();
-            CE::generic_store(p, sm_out, lane, row, chunk);
+            CE::generic_store(p, sm_out, lm, lane, group * R, colbase);
         }
         __syncwarp();  // every lane is done with this input stage
 
         if (++chunk == p.nchunks) {
             chunk = 0;
-            row += GW;
-            if (row < p.rows) state = CE::row_start(p, row);
+            group += GW;
+            row = group * R + lm.g;
+            if (group < groups) state = CE::row_start(p, row);
         }
         if (++stage == S) { stage = 0; parity ^= 1u; }
     }
@@ -573,17 +634,23 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
     using LB = Lookback<MODE, TIn, TOut, K>;
     using E = typename CE::E;
     constexpr bool SIGNED = CE::SIGNED;
+    constexpr int CHUNK = 32 * K;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align_1024(smem_raw);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const int S = TMA ? p.stages : 1;
     const int per_warp = warp_smem_bytes<MODE, TIn, TOut, K>(S);
 
+    LaneMap lm;
+    lm.R = 1; lm.g = 0; lm.i = lane; lm.W = CHUNK;
+    const typename CE::Offsets off = CE::offsets(lm);
+
     WarpPipe<TIn, TOut, K> pipe;
     pipe.base = smem + warp * per_warp;
     pipe.bars = smem_u32(smem + nwarps * per_warp) + warp * (8 * kMaxStages);
     pipe.stages = S;
     pipe.lane = lane;
+    pipe.setup(1);
     Exchange* xc = reinterpret_cast<Exchange*>(smem + nwarps * per_warp + nwarps * 8 * kMaxStages);
     if (TMA) pipe.init();
     if (blockIdx.x == 0 && threadIdx.x == 0) p.ws->started_id = p.call_id;
@@ -599,7 +666,7 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
         if (issued_tile < p.num_tiles) {
             const long long r = issued_tile / tpr;
             const int jj = (int)(issued_tile - r * tpr);
-            pipe.issue(&tm_a, &tm_b, r, jj * nwarps + warp, issued % S);
+            pipe.issue(&tm_a, &tm_b, r, (long long)(jj * nwarps + warp) * CHUNK, issued % S);
             issued_tile += G;
             ++issued;
         }
@@ -614,13 +681,14 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
     for (long long T = blockIdx.x; T < p.num_tiles; T += G, ++q) {
         const long long row = T / tpr;
         const int j = (int)(T - row * tpr);
-        const int chunk = j * nwarps + warp;
+        const long long colbase = (long long)(j * nwarps + warp) * CHUNK;
+        const long long col0 = colbase + lane * K;
         bool copy_failed = false;
         if (TMA) {
             issue_next();
             copy_failed = !pipe.wait(stage, parity);
         } else {
-            CE::generic_load(p, pipe.in_a(0), pipe.in_b(0), lane, row, chunk);
+            CE::generic_load(p, pipe.in_a(0), pipe.in_b(0), lm, lane, row, colbase);
             __syncwarp();
         }
         const uint8_t* sm_a = pipe.in_a(stage);
@@ -629,7 +697,7 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
 
         typename CE::Pending pd;
         E total;
-        CE::phase1(p, sm_a, sm_b, lane, row, chunk, pd, total);
+        CE::phase1(p, sm_a, sm_b, off, lm, lane, row, col0, pd, total);
         if (lane == 0) xc->agg[warp] = pack_elem<SIGNED>(total);
         if (copy_failed && lane == 0) {
             record_error(p, kErrCopyTimeout, T);
@@ -673,12 +741,12 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
         carry.A = neg_inf(); carry.m = xc->carry.x; carry.s = xc->carry.y; carry.p = 0u;
         const E entering_chunk = compose(carry, unpack_elem<SIGNED>(xc->wexcl[warp]));
         if (TMA) pipe.acquire_out();
-        CE::phase2(p, sm_a, sm_b, sm_out, lane, row, chunk, pd, entering_chunk);
+        CE::phase2(p, sm_a, sm_b, sm_out, off, lm, row, col0, pd, entering_chunk);
         if (TMA) {
-            pipe.store(&tm_o, row, chunk, q & 1);
+            pipe.store(&tm_o, row, colbase, q & 1);
         } else {
             __syncwarp();
-            CE::generic_store(p, sm_out, lane, row, chunk);
+            CE::generic_store(p, sm_out, lm, lane, row, colbase);
         }
         __syncwarp();
         if (++stage == S) { stage = 0; parity ^= 1u; }

@@ -99,6 +99,26 @@ def _stream_ptr(device) -> ctypes.c_void_p:
     return ctypes.c_void_p(torch.cuda.current_stream(device).cuda_stream)
 
 
+class _on_device:
+    """Make `device` current for the duration of a call (the library launches on the current device);
+    free when it already is."""
+
+    def __init__(self, device):
+        self.idx = device.index if device.index is not None else torch.cuda.current_device()
+        self.prev = None
+
+    def __enter__(self):
+        cur = torch.cuda.current_device()
+        if cur != self.idx:
+            self.prev = cur
+            torch.cuda.set_device(self.idx)
+
+    def __exit__(self, *exc):
+        if self.prev is not None:
+            torch.cuda.set_device(self.prev)
+        return False
+
+
 def _require(t: torch.Tensor, shape, name: str, cuda: bool = True):
     if tuple(t.shape) != tuple(shape):
         raise ValueError(f"{name}: expected shape {tuple(shape)}, got {tuple(t.shape)}")
@@ -153,7 +173,7 @@ def scan_linear(a: torch.Tensor, b: torch.Tensor, x0: torch.Tensor, x: torch.Ten
         return x
     if workspace is None:
         workspace = new_workspace(rows, n, a.device)
-    with torch.cuda.device(a.device):
+    with _on_device(a.device):
         _check(lib().heinsen_scan_linear(_ptr(a), _ptr(b), _ptr(x0), _ptr(x), rows, n, _dtype_code(a),
                                          _ptr(workspace), workspace.numel(), _stream_ptr(a.device)))
     return x
@@ -185,7 +205,7 @@ def scan_log(log_a: torch.Tensor, log_b: torch.Tensor, log_x0: torch.Tensor, log
         return (log_x, sign_x) if signed else log_x
     if workspace is None:
         workspace = new_workspace(rows, n, log_a.device)
-    with torch.cuda.device(log_a.device):
+    with _on_device(log_a.device):
         _check(lib().heinsen_scan_log(_ptr(log_a), _ptr(log_b), _ptr(log_x0), _ptr(log_x), _ptr(sign_a), _ptr(sign_b),
                                       _ptr(sign_x0), _ptr(sign_x) if signed else None, rows, n, _dtype_code(log_a),
                                       _dtype_code(log_x), _ptr(workspace), workspace.numel(),
@@ -208,7 +228,7 @@ def scan_log_host(log_a, log_b, log_x0, log_x, device_scratch: torch.Tensor, sig
         if t.is_cuda:
             raise ValueError(f"{name} must be a host tensor")
     dev = device_scratch.device
-    with torch.cuda.device(dev):
+    with _on_device(dev):
         _check(lib().heinsen_scan_log_host(_ptr(log_a), _ptr(log_b), _ptr(log_x0), _ptr(log_x), _ptr(sign_a),
                                            _ptr(sign_b), _ptr(sign_x0), _ptr(sign_x), rows, n, _dtype_code(log_a),
                                            _dtype_code(log_x), _ptr(device_scratch), device_scratch.numel(),
@@ -224,7 +244,7 @@ def scan_linear_host(a, b, x0, x, device_scratch: torch.Tensor):
         if t.is_cuda:
             raise ValueError(f"{name} must be a host tensor")
     dev = device_scratch.device
-    with torch.cuda.device(dev):
+    with _on_device(dev):
         _check(lib().heinsen_scan_linear_host(_ptr(a), _ptr(b), _ptr(x0), _ptr(x), rows, n, _dtype_code(a),
                                               _ptr(device_scratch), device_scratch.numel(), _stream_ptr(dev)))
     return x
