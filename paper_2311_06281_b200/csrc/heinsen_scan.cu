@@ -28,7 +28,8 @@ thread_local char g_cuda_msg[256] = "";
 constexpr long long kMaxTmaDim = (1ll << 31) - (1ll << 20);  // TMA coordinates are int32
 constexpr int kBatchedMinRowsPerSm = 8;  // fewer rows per SM than this: look-back kernel
 constexpr int kBatchedMinWarpsPerSm = 12; // rows per warp are chosen to keep at least this many warps per SM
-constexpr int kLookbackWarps = 8;        // warps (= chunks) per tile of the look-back kernel
+constexpr int kLookbackMinWarps = 8;     // fewest compute warps (= chunks per tile) of the look-back kernel
+constexpr int kLookbackWarps = 12;       // default compute warps of the look-back kernel
 constexpr int kMinChunk = 512;           // smallest chunk (32 lanes x 16 elements)
 
 unsigned long long next_call_id() {
@@ -93,12 +94,18 @@ EncodeFn encode_fn() {
 }
 
 // [rows, n] row-major as a 2-D tensor map whose box is {128 bytes of a row, box_rows rows}, 128-byte swizzle.
-bool make_tmap(CUtensorMap* tm, const void* ptr, hs_dtype dt, long long rows, long long n, int box_rows) {
+// flat: the same memory as [rows*n*es/128, 128 bytes] (lines), box = box_rows consecutive lines.
+bool make_tmap(CUtensorMap* tm, const void* ptr, hs_dtype dt, long long rows, long long n, int box_rows, bool flat) {
     EncodeFn fn = encode_fn();
     if (!fn) return false;
     const int es = (dt == HS_F32) ? 4 : 2;
     cuuint64_t dims[2] = {(cuuint64_t)n, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)n * es};
+    if (flat) {
+        dims[0] = (cuuint64_t)(128 / es);
+        dims[1] = (cuuint64_t)(rows * n * es / 128);
+        strides[0] = 128;
+    }
     cuuint32_t box[2] = {(cuuint32_t)(128 / es), (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(tm, dt == HS_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
@@ -132,6 +139,7 @@ struct KernelEntry {
     int K;
     int warp_smem_per_stage;  // bytes of one input stage (both tensors) of one warp
     int warp_smem_out;        // bytes of both output buffers of one warp
+    int (*lb_smem)(int);      // dynamic shared memory of the look-back kernel for W compute warps
 };
 
 template <int MODE, typename TIn, typename TOut, int K, bool TMA>
@@ -142,6 +150,7 @@ KernelEntry entry() {
     e.K = K;
     e.warp_smem_per_stage = 2 * 32 * K * (int)sizeof(TIn);
     e.warp_smem_out = 2 * 32 * K * (int)sizeof(TOut);
+    e.lb_smem = [](int W) { return lb_total_smem_bytes<TIn, K>(W); };
     return e;
 }
 
@@ -172,8 +181,8 @@ bool find_kernel(int mode, hs_dtype din, hs_dtype dout, bool tma, KernelEntry& e
 #undef HS_PICK
 }
 
-long long lookback_tiles_per_row(long long n, int chunk) {
-    const long long tile = (long long)kLookbackWarps * chunk;
+long long lookback_tiles_per_row(long long n, int chunk, int warps) {
+    const long long tile = (long long)warps * chunk;
     return (n + tile - 1) / tile;
 }
 
@@ -185,8 +194,8 @@ int choose_path(long long rows, const DeviceInfo& d) {
 
 size_t workspace_bytes_for(long long rows, long long n) {
     // sized for the smallest chunk so that it covers every type
-    const long long tiles = rows * lookback_tiles_per_row(n, kMinChunk);
-    return sizeof(Header) + (size_t)tiles * (8 + 16 + 16);
+    const long long tiles = rows * lookback_tiles_per_row(n, kMinChunk, kLookbackMinWarps);
+    return sizeof(Header) + (size_t)tiles * 16;
 }
 
 // cudaFuncSetAttribute and the occupancy query cost microseconds per call; remember what was set.
@@ -268,6 +277,7 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
     p.call_id = next_call_id();
     p.spin_limit = g_spin_limit.load();
     p.mute_tile = g_mute_tile.load();
+    p.debug_flags = env_int("HEINSEN_SCAN_DEBUG_FLAGS", 0, 0, 255);
     p.ws = reinterpret_cast<Header*>(workspace);
 
     const int path = choose_path(p.rows, dev);
@@ -278,6 +288,8 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         // per SM, so that rows with many steps use few scan steps and few rows still fill the GPU.
         int R = 8;
         while (R > 1 && (p.rows + R - 1) / R < (long long)kBatchedMinWarpsPerSm * dev.sm_count) R >>= 1;
+        // whole chunks and enough rows: one row per warp, each chunk one contiguous 2 KB box
+        if (tma && p.n % chunk == 0 && p.rows >= (long long)kBatchedMinWarpsPerSm * dev.sm_count) R = 1;
         R = env_int("HEINSEN_SCAN_ROWS_PER_WARP", R, 1, 8);
         while (R & (R - 1)) R &= R - 1;  // power of two
         p.rows_per_warp = R;
@@ -293,16 +305,16 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         fn = ke.batched;
     } else {
         p.rows_per_warp = 1;
-        warps = kLookbackWarps;
-        stages = tma ? env_int("HEINSEN_SCAN_LB_STAGES", 2, 2, kMaxStages) : 1;
-        p.tiles_per_row = (int)lookback_tiles_per_row(p.n, chunk);
+        // W compute warps (as many as shared memory allows, at most the default) + 1 look-back warp
+        int W = env_int("HEINSEN_SCAN_LB_WARPS", kLookbackWarps, kLookbackMinWarps, kLbMaxWarps);
+        while (W > kLookbackMinWarps && ke.lb_smem(W) + 1024 > dev.max_smem_optin) --W;
+        warps = W + 1;
+        stages = kLbStages;
+        p.tiles_per_row = (int)lookback_tiles_per_row(p.n, chunk, W);
         p.num_tiles = p.rows * p.tiles_per_row;
-        const size_t need = sizeof(Header) + (size_t)p.num_tiles * (8 + 16 + 16);
+        const size_t need = sizeof(Header) + (size_t)p.num_tiles * 16;
         if (workspace_bytes < need) return HS_ERR_WORKSPACE_TOO_SMALL;
-        uint8_t* w = reinterpret_cast<uint8_t*>(workspace) + sizeof(Header);
-        p.agg = reinterpret_cast<float4*>(w);
-        p.inc = reinterpret_cast<float4*>(w + (size_t)p.num_tiles * 16);
-        p.flags = reinterpret_cast<unsigned long long*>(w + (size_t)p.num_tiles * 32);
+        p.desc = reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(workspace) + sizeof(Header));
         fn = ke.lookback;
         grid = 0;  // set below from occupancy
     }
@@ -312,16 +324,23 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
     std::memset(&tm_b, 0, sizeof tm_b);
     std::memset(&tm_o, 0, sizeof tm_o);
     if (tma) {
-        const int br = p.rows_per_warp;
-        if (!make_tmap(&tm_a, p.in_a, pr.din, p.rows, p.n, br) || !make_tmap(&tm_b, p.in_b, pr.din, p.rows, p.n, br) ||
-            !make_tmap(&tm_o, p.out, pr.dout, p.rows, p.n, br)) {
+        // one row per warp and whole chunks only: move a chunk as a single box of consecutive lines
+        const bool flat = p.rows_per_warp == 1 && p.n % chunk == 0 && p.rows * p.n * es_in / 128 < (1ll << 31) &&
+                          !env_int("HEINSEN_SCAN_NO_FLAT", 0, 0, 1);
+        p.flat_boxes = flat ? 1 : 0;
+        const int br_in = flat ? chunk * es_in / 128 : p.rows_per_warp;
+        const int br_out = flat ? chunk * es_out / 128 : p.rows_per_warp;
+        if (!make_tmap(&tm_a, p.in_a, pr.din, p.rows, p.n, br_in, flat) ||
+            !make_tmap(&tm_b, p.in_b, pr.din, p.rows, p.n, br_in, flat) ||
+            !make_tmap(&tm_o, p.out, pr.dout, p.rows, p.n, br_out, flat)) {
             snprintf(g_cuda_msg, sizeof g_cuda_msg, "cuTensorMapEncodeTiled failed");
             return HS_ERR_CUDA;
         }
     }
     p.stages = stages;
-    const int smem = warps * (stages * ke.warp_smem_per_stage + ke.warp_smem_out) + warps * 8 * kMaxStages + 1024 +
-                     (path == HS_PATH_LOOKBACK ? 1024 : 0);
+    const int smem = path == HS_PATH_LOOKBACK
+                         ? ke.lb_smem(warps - 1) + 1024
+                         : warps * (stages * ke.warp_smem_per_stage + ke.warp_smem_out) + warps * 8 * kMaxStages + 1024;
     if (smem > dev.max_smem_optin) return HS_ERR_INVALID_ARG;
     cudaError_t e = ensure_smem_attr(fn, smem);
     if (e != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", e);
@@ -338,6 +357,9 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         long long g = (long long)per_sm * dev.sm_count;
         if (g > p.num_tiles) g = p.num_tiles;
         grid = (int)g;
+        // every descriptor starts as "nothing yet"
+        e = cudaMemsetAsync(p.desc, 0, (size_t)p.num_tiles * 16, stream);
+        if (e != cudaSuccess) return cuda_fail("cudaMemsetAsync", e);
         e = cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(warps * 32), args, smem, stream);
     } else {
         e = cudaLaunchKernel(fn, dim3(grid), dim3(warps * 32), args, smem, stream);

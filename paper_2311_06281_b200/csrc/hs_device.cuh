@@ -352,6 +352,12 @@ struct Run {
         }
     }
 
+    __device__ __forceinline__ static void load_a(const uint8_t* sm_a, const uint32_t* off, float* va) {
+        const uint32_t base_a = smem_u32(sm_a);
+#pragma unroll
+        for (int j = 0; j < IN_UNITS; ++j) Storage<TIn>::unpack(lds128(base_a + off[j]), va + j * Storage<TIn>::kPerUnit);
+    }
+
     // va, vb: the stored inputs (log a, log b for the log modes; a, b for kLinear).
     // sa, sb: per-element sign masks for kLogSigned (ignored otherwise).
     __device__ __forceinline__ E pass1(const float* va, const float* vb, const uint32_t* sa, const uint32_t* sb) {
@@ -401,6 +407,26 @@ struct Run {
         agg.s = SIGNED ? flip(sum, par) : sum;  // beta = alpha * (sum relative to the run start)
         agg.p = par;
         return agg;
+    }
+
+    // Recompute A_t and the parity of a_1..a_t from the inputs (s_t and r come from elsewhere):
+    // the look-back kernel parks only s_t between its two phases.
+    __device__ __forceinline__ void rebuild(const float* va, const uint32_t* sa) {
+        float acc = 0.0f;
+        uint32_t par = 0u;
+#pragma unroll
+        for (int t = 0; t < K; ++t) {
+            if (MODE == kLinear) {
+                acc += log_abs_accurate(va[t]);
+                par ^= __float_as_uint(va[t]) & kSignBit;
+            } else {
+                acc += va[t];
+                if (MODE == kLogSigned) par ^= sa[t];
+            }
+            A[t] = acc;
+            if (SIGNED) P[t] = par;
+        }
+        bad = false;
     }
 
     // Apply the value entering the run and produce the K outputs.

@@ -49,16 +49,17 @@ struct Params {
     int stages;         // input stages per warp (2..kMaxStages)
     int sign_vec_ok;    // sign tensors may be accessed with 16-byte vectors
     int rows_per_warp;  // R: rows held by one warp of the batched kernel (1, 2, 4, 8); look-back: 1
+    int flat_boxes;     // R == 1 and n a multiple of the chunk: a chunk moves as ONE box of consecutive
+                        // 128-byte lines of the flat [rows*n/line, line] view instead of one box per line
     unsigned long long call_id;
     Header* ws;
     // look-back kernel only
     int tiles_per_row;
     long long num_tiles;
-    unsigned long long* flags;  // [num_tiles] (call_id << 2) | state
-    float4* agg;                // [num_tiles] tile aggregate (A, m, s, p)
-    float4* inc;                // [num_tiles] value of x after the tile (m, s, -, -)
+    uint4* desc;                // [num_tiles] tile descriptors, zeroed before the launch
     unsigned int spin_limit;    // bound on polls of predecessor flags
     long long mute_tile;        // test hook: this tile never publishes (-1: none)
+    int debug_flags;            // timing experiments only (results are wrong when non-zero)
 };
 
 // The first thread to report an error in this call records it; heinsen_scan_check() reports it
@@ -320,11 +321,15 @@ struct WarpPipe {
     int R;           // rows per box
     int in_boxes;    // boxes per tensor per chunk, input / output
     int out_boxes;
+    bool flat;       // one box per chunk, addressed by line number (see Params::flat_boxes)
+    long long n;     // row length, for line numbers
 
-    __device__ __forceinline__ void setup(int rows_per_warp) {
+    __device__ __forceinline__ void setup(int rows_per_warp, bool flat_boxes = false, long long row_len = 0) {
         R = rows_per_warp;
-        in_boxes = IN_BYTES / (128 * R);
-        out_boxes = OUT_BYTES / (128 * R);
+        flat = flat_boxes;
+        n = row_len;
+        in_boxes = flat ? 1 : IN_BYTES / (128 * R);
+        out_boxes = flat ? 1 : OUT_BYTES / (128 * R);
     }
     __device__ __forceinline__ uint8_t* in_a(int s) const { return base + s * 2 * IN_BYTES; }
     __device__ __forceinline__ uint8_t* in_b(int s) const { return base + s * 2 * IN_BYTES + IN_BYTES; }
@@ -343,7 +348,13 @@ struct WarpPipe {
         const uint32_t bar = bars + 8 * s;
         if (lane == 0) mbar_expect_tx(bar, 2 * IN_BYTES);
         __syncwarp();
-        if (lane < in_boxes) {
+        if (flat) {
+            if (lane == 0) {
+                const int line = (int)((row0 * n + colbase) / IN_PER_BOX);
+                tma_load_2d(smem_u32(in_a(s)), tm_a, 0, line, bar);
+                tma_load_2d(smem_u32(in_b(s)), tm_b, 0, line, bar);
+            }
+        } else if (lane < in_boxes) {
             const int x = (int)colbase + lane * IN_PER_BOX;
             const uint32_t dst = (uint32_t)(lane * R * 128);
             tma_load_2d(smem_u32(in_a(s)) + dst, tm_a, x, (int)row0, bar);
@@ -358,14 +369,22 @@ struct WarpPipe {
         if (lane < out_boxes) bulk_wait_read<1>();
         __syncwarp();
     }
-    __device__ __forceinline__ void store(const CUtensorMap* tm_o, long long row0, long long colbase, int o) const {
+    // store the chunk held in shared memory at `src`
+    __device__ __forceinline__ void store_from(const CUtensorMap* tm_o, long long row0, long long colbase, uint32_t src) const {
         fence_async_smem();
         __syncwarp();
         if (lane < out_boxes) {
-            const int x = (int)colbase + lane * OUT_PER_BOX;
-            tma_store_2d(tm_o, x, (int)row0, smem_u32(out(o)) + (uint32_t)(lane * R * 128));
+            if (flat) {
+                tma_store_2d(tm_o, 0, (int)((row0 * n + colbase) / OUT_PER_BOX), src);
+            } else {
+                const int x = (int)colbase + lane * OUT_PER_BOX;
+                tma_store_2d(tm_o, x, (int)row0, src + (uint32_t)(lane * R * 128));
+            }
             bulk_commit();
         }
+    }
+    __device__ __forceinline__ void store(const CUtensorMap* tm_o, long long row0, long long colbase, int o) const {
+        store_from(tm_o, row0, colbase, smem_u32(out(o)));
     }
     __device__ __forceinline__ void drain() const {
         if (lane < out_boxes) bulk_wait_all();
@@ -407,7 +426,7 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
     pipe.bars = smem_u32(smem + nwarps * per_warp) + warp * (8 * kMaxStages);
     pipe.stages = S;
     pipe.lane = lane;
-    pipe.setup(R);
+    pipe.setup(R, p.flat_boxes != 0, p.n);
     if (TMA) pipe.init();
 
     if (blockIdx.x == 0 && threadIdx.x == 0) p.ws->started_id = p.call_id;
@@ -488,117 +507,137 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
 // ------------------------------------------------------------------------------------------
 // (b) Single-pass kernel with decoupled look-back, for few long rows.
 //
-// A row is cut into tiles of WARPS chunks.  CTA c handles tiles c, c+G, c+2G, ... (all CTAs are
-// resident: cooperative launch), warp w the w-th chunk of each tile.  After the chunks' first
-// phase the tile's aggregate is published; the value of x entering the tile is then assembled
-// from the descriptors of the preceding tiles of the same row (aggregates until a tile whose
-// value of x is already known), which is the "by parts" evaluation that the associativity of
-// prefix sums allows, done in one pass.  Descriptor states carry the id of the call, so the
-// workspace never has to be cleared.
-__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
-    unsigned long long v;
-    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
-    return v;
+// A row is cut into tiles of W chunks (W = compute warps per CTA).  CTA c handles tiles c, c+G,
+// c+2G, ... (all CTAs are resident: cooperative launch); compute warp w owns the w-th chunk of
+// each tile, and one more warp does nothing but carry propagation.  The kernel is software
+// pipelined so that the latency of the look-back never stalls the arithmetic:
+//
+//   compute warp, iteration i :  phase 1 of tile i   (inputs -> partial sums s_t parked in shared
+//                                                     memory, chunk aggregate handed to the
+//                                                     look-back warp)
+//                                phase 2 of tile i-1 (whose entering value has arrived meanwhile:
+//                                                     outputs, TMA store)
+//   look-back warp, tile i    :  scan of the W chunk aggregates, publish the tile aggregate,
+//                                assemble the value of x entering the tile from the descriptors
+//                                of the preceding tiles (aggregates until a tile whose value is
+//                                known), publish the tile's own value, hand the carry back.
+//
+// This is the "by parts" evaluation that the associativity of prefix sums allows, done in one
+// pass over HBM.  Every wait is bounded; when one runs out the CTA records an error and leaves.
+// A tile's descriptor is one 16-byte word, read and written with single 128-bit accesses so that
+// state and payload always belong together:  {A, m, s, tag},  tag = state | parity << 2,
+// state 0 = nothing yet (the descriptor array is zeroed before every launch), 1 = the tile's
+// aggregate, 2 = the value of x after the tile (A = -inf).
+struct Desc { unsigned long long lo, hi; };
+__device__ __forceinline__ Desc ld_desc(const void* p) {
+    Desc d;
+    asm volatile("{\n\t.reg .b128 q;\n\tld.relaxed.gpu.global.b128 q, [%2];\n\tmov.b128 {%0, %1}, q;\n\t}"
+                 : "=l"(d.lo), "=l"(d.hi) : "l"(p) : "memory");
+    return d;
 }
-__device__ __forceinline__ void st_release_u64(unsigned long long* p, unsigned long long v) {
-    asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+__device__ __forceinline__ void st_desc(void* p, Desc d) {
+    asm volatile("{\n\t.reg .b128 q;\n\tmov.b128 q, {%1, %2};\n\tst.relaxed.gpu.global.b128 [%0], q;\n\t}"
+                 ::"l"(p), "l"(d.lo), "l"(d.hi) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
-constexpr int kLookPerLane = 4;                     // predecessors polled by each lane per round
+constexpr int kLookPerLane = 8;                     // predecessors polled by each lane per round
 constexpr int kLookWindow = 32 * kLookPerLane;      // tiles covered by one round
+constexpr int kLbMaxWarps = 16;                     // compute warps per CTA, at most
 
 template <int MODE, typename TIn, typename TOut, int K>
 struct Lookback {
     using CE = ChunkEngine<MODE, TIn, TOut, K>;
     static constexpr bool SIGNED = CE::SIGNED;
     using E = Elem<SIGNED>;
-    enum : int { kNotReady = 0, kAgg = 1, kInc = 2, kSkip = 3 };
+    enum : uint32_t { kNotReady = 0, kAgg = 1, kInc = 2 };
 
-    __device__ static __forceinline__ void publish_agg(const Params& p, long long T, const E& e) {
-        p.agg[T] = make_float4(e.A, e.m, e.s, __uint_as_float(e.p));
-        st_release_u64(p.flags + T, (p.call_id << 2) | 1ull);
+    __device__ static __forceinline__ Desc pack(const E& e, uint32_t state) {
+        Desc d;
+        d.lo = (unsigned long long)__float_as_uint(e.A) | ((unsigned long long)__float_as_uint(e.m) << 32);
+        d.hi = (unsigned long long)__float_as_uint(e.s) | ((unsigned long long)(state | ((e.p >> 31) << 2)) << 32);
+        return d;
     }
-    __device__ static __forceinline__ void publish_inc(const Params& p, long long T, const E& e) {
-        p.inc[T] = make_float4(e.m, e.s, 0.0f, 0.0f);
-        st_release_u64(p.flags + T, (p.call_id << 2) | 2ull);
+    __device__ static __forceinline__ uint32_t state_of(const Desc& d) { return (uint32_t)(d.hi >> 32) & 3u; }
+    __device__ static __forceinline__ E unpack(const Desc& d) {
+        E e;
+        e.A = __uint_as_float((uint32_t)d.lo);
+        e.m = __uint_as_float((uint32_t)(d.lo >> 32));
+        e.s = __uint_as_float((uint32_t)d.hi);
+        e.p = SIGNED ? ((((uint32_t)(d.hi >> 32)) >> 2) & 1u) << 31 : 0u;
+        return e;
+    }
+    __device__ static __forceinline__ void publish_agg(const Params& p, long long T, const E& e) {
+        st_desc(p.desc + T, pack(e, kAgg));
+    }
+    __device__ static __forceinline__ void publish_inc(const Params& p, long long T, E e) {
+        e.A = neg_inf();
+        e.p = 0u;
+        st_desc(p.desc + T, pack(e, kInc));
     }
 
     // Warp-collective.  Returns the value of x entering tile T (tile j of `row`), j >= 1.
-    __device__ static __forceinline__ E run(const Params& p, long long T, int j, long long row, int lane, bool& failed) {
+    // One round reads the descriptors of up to kLookWindow preceding tiles, all loads in flight
+    // at once; lane l looks at distances base + 8l .. base + 8l + 7, nearest first.
+    __device__ static __forceinline__ E run(const Params& p, long long T, int j, long long row, int lane, bool& failed,
+                                            unsigned int& total_polls) {
         E acc = identity_elem<SIGNED>();
         failed = false;
-        const unsigned long long id_agg = (p.call_id << 2) | 1ull, id_inc = (p.call_id << 2) | 2ull;
+        const E x0e = CE::row_start(p, row);
         for (int base = 1;; base += kLookWindow) {
-            int st[kLookPerLane];
+            Desc d[kLookPerLane];
             bool complete = false, has_inc = false;
             uint32_t inc_mask = 0u;
             unsigned int polls = 0;
             while (true) {
+#pragma unroll
+                for (int q = 0; q < kLookPerLane; ++q) {
+                    const int dist = base + kLookPerLane * lane + q;
+                    if (j - dist >= 0) d[q] = ld_desc(p.desc + (T - dist));
+                    else { d[q].lo = 0ull; d[q].hi = 0ull; }
+                }
                 complete = true;
                 has_inc = false;
 #pragma unroll
                 for (int q = 0; q < kLookPerLane; ++q) {
-                    const int dist = base + kLookPerLane * lane + q;
-                    const int jj = j - dist;
-                    int s;
-                    if (jj < -1) s = kSkip;
-                    else if (jj == -1) s = kInc;
-                    else {
-                        const unsigned long long f = ld_acquire_u64(p.flags + (T - dist));
-                        s = (f == id_inc) ? kInc : (f == id_agg) ? kAgg : kNotReady;
-                    }
-                    st[q] = s;
-                }
-                // ready prefix of this lane, nearest first, up to its first known value
-#pragma unroll
-                for (int q = 0; q < kLookPerLane; ++q) {
-                    if (!has_inc && complete) {
-                        if (st[q] == kNotReady) complete = false;
-                        else if (st[q] == kInc) has_inc = true;
+                    const int jj = j - (base + kLookPerLane * lane + q);
+                    const uint32_t s = (jj >= 0) ? state_of(d[q]) : (uint32_t)kInc;  // jj == -1: x_0; beyond: ignored
+                    if (!has_inc && complete) {  // ready prefix of this lane, up to its first known value
+                        if (s == kNotReady) complete = false;
+                        else if (s == kInc) has_inc = true;
                     }
                 }
                 inc_mask = __ballot_sync(0xffffffffu, complete && has_inc);
                 const uint32_t ok_mask = __ballot_sync(0xffffffffu, complete);
                 const uint32_t need = inc_mask ? ((2u << (__ffs(inc_mask) - 1)) - 1u) : 0xffffffffu;
+                ++total_polls;
                 if ((ok_mask & need) == need) break;
-                if (++polls >= p.spin_limit || ((polls & 255u) == 0u && *(volatile unsigned long long*)&p.ws->error_id == p.call_id)) {
+                if (++polls >= p.spin_limit ||
+                    ((polls & 255u) == 0u && *(volatile unsigned long long*)&p.ws->error_id == p.call_id)) {
                     failed = true;
                     return acc;
                 }
             }
             const int lstar = inc_mask ? (__ffs(inc_mask) - 1) : 31;
             E part = identity_elem<SIGNED>();
-            if (lane <= lstar) {
-                bool stop = false;
+            bool stop = lane > lstar;
 #pragma unroll
-                for (int q = 0; q < kLookPerLane; ++q) {
-                    if (!stop && st[q] != kSkip) {
-                        const int dist = base + kLookPerLane * lane + q;
-                        E e;
-                        if (st[q] == kInc) {
-                            if (j - dist == -1) {
-                                e = CE::row_start(p, row);
-                            } else {
-                                const float4 v = __ldcg(p.inc + (T - dist));
-                                e.A = neg_inf(); e.m = v.x; e.s = v.y; e.p = 0u;
-                            }
-                            stop = true;
-                        } else {
-                            const float4 v = __ldcg(p.agg + (T - dist));
-                            e.A = v.x; e.m = v.y; e.s = v.z; e.p = __float_as_uint(v.w);
-                        }
-                        part = compose(e, part);  // e is older than everything folded so far
-                    } else {
-                        stop = true;
-                    }
+            for (int q = 0; q < kLookPerLane; ++q) {
+                const int jj = j - (base + kLookPerLane * lane + q);
+                if (!stop) {
+                    const E e = (jj >= 0) ? unpack(d[q]) : x0e;
+                    if (jj < 0 || state_of(d[q]) == kInc) stop = true;
+                    part = compose(e, part);  // e is older than everything folded so far
                 }
             }
             // ordered reduction: lane 0 holds the newest tiles, higher lanes older ones
 #pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                E other = shfl_down_elem(part, d);
+            for (int dd = 1; dd < 32; dd <<= 1) {
+                E other = shfl_down_elem(part, dd);
                 E c = compose(other, part);
-                if (lane + d < 32) part = c;
+                if (lane + dd < 32) part = c;
             }
             const E window = shfl_elem(part, 0);
             acc = compose(window, acc);
@@ -607,11 +646,23 @@ struct Lookback {
     }
 };
 
+// CTA-level exchange between the compute warps and the look-back warp (two tiles in flight).
 struct alignas(16) Exchange {
-    float4 agg[16];    // per-warp aggregates of the current tile
-    float4 wexcl[16];  // per-warp exclusive prefixes within the tile
-    float4 carry;      // value of x entering the tile (m, s)
+    float4 agg[2][kLbMaxWarps];    // per-warp aggregates of a tile
+    float4 wexcl[2][kLbMaxWarps];  // per-warp exclusive prefixes within the tile
+    float4 carry[2];               // value of x entering the tile (m, s)
+    unsigned long long agg_ready[2];    // mbarrier: all compute warps have delivered their aggregate
+    unsigned long long carry_ready[2];  // mbarrier: the look-back warp has delivered wexcl and carry
     int abort;
+    int pad[3];
+};
+
+// Per-lane state parked between the two phases of a chunk (structure of arrays, one per buffer).
+struct LanePark {
+    float r[32];
+    float A[32], m[32], s[32];
+    uint32_t p[32];
+    int slow;
     int pad[3];
 };
 
@@ -626,132 +677,271 @@ __device__ __forceinline__ Elem<SIGNED> unpack_elem(const float4 v) {
     return e;
 }
 
+constexpr int kLbStages = 3;  // input stages per compute warp: tile i-1 (awaiting phase 2), i, i+1 (in flight)
+
+template <int K>
+__host__ __device__ constexpr int lb_park_bytes() { return 32 * K * 4; }  // s_t as fp32; outputs reuse it
+
+// Chunk buffers of one compute warp of the look-back kernel (a multiple of 1024 bytes: the
+// swizzled layouts need 1024-byte aligned buffers); its two LanePark records live after the
+// chunk buffers of all warps.
+template <typename TIn, int K>
+__host__ __device__ constexpr int lb_warp_smem_bytes() {
+    return kLbStages * 2 * 32 * K * (int)sizeof(TIn) + 2 * lb_park_bytes<K>();
+}
+static_assert(lb_warp_smem_bytes<float, 16>() % 1024 == 0 && lb_warp_smem_bytes<__nv_bfloat16, 32>() % 1024 == 0, "");
+// total dynamic shared memory of the look-back kernel for W compute warps (without alignment slack)
+template <typename TIn, int K>
+__host__ __device__ constexpr int lb_total_smem_bytes(int W) {
+    return W * (lb_warp_smem_bytes<TIn, K>() + 2 * (int)sizeof(LanePark)) + (int)sizeof(Exchange) + W * kLbStages * 8;
+}
+
 template <int MODE, typename TIn, typename TOut, int K, bool TMA>
-__global__ void __launch_bounds__(256, 2)
+__global__ void __launch_bounds__(544, 1)
 lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                      const __grid_constant__ CUtensorMap tm_o) {
     using CE = ChunkEngine<MODE, TIn, TOut, K>;
     using LB = Lookback<MODE, TIn, TOut, K>;
+    using R_ = Run<MODE, TIn, TOut, K>;
     using E = typename CE::E;
     constexpr bool SIGNED = CE::SIGNED;
     constexpr int CHUNK = 32 * K;
+    constexpr int IN_BYTES = CHUNK * (int)sizeof(TIn);
+    constexpr int S = kLbStages;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align_1024(smem_raw);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    const int S = TMA ? p.stages : 1;
-    const int per_warp = warp_smem_bytes<MODE, TIn, TOut, K>(S);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int W = (blockDim.x >> 5) - 1;  // compute warps; warp W is the look-back warp
+    constexpr int per_warp = lb_warp_smem_bytes<TIn, K>();
 
-    LaneMap lm;
-    lm.R = 1; lm.g = 0; lm.i = lane; lm.W = CHUNK;
-    const typename CE::Offsets off = CE::offsets(lm);
+    uint8_t* tail = smem + W * per_warp;
+    LanePark* all_parks = reinterpret_cast<LanePark*>(tail);  // [W][2]
+    Exchange* xc = reinterpret_cast<Exchange*>(tail + W * 2 * sizeof(LanePark));
+    const uint32_t warp_bars = smem_u32(reinterpret_cast<uint8_t*>(xc) + sizeof(Exchange));  // W x S stage mbarriers
+    const uint32_t agg_bar = smem_u32(&xc->agg_ready[0]), carry_bar = smem_u32(&xc->carry_ready[0]);
 
-    WarpPipe<TIn, TOut, K> pipe;
-    pipe.base = smem + warp * per_warp;
-    pipe.bars = smem_u32(smem + nwarps * per_warp) + warp * (8 * kMaxStages);
-    pipe.stages = S;
-    pipe.lane = lane;
-    pipe.setup(1);
-    Exchange* xc = reinterpret_cast<Exchange*>(smem + nwarps * per_warp + nwarps * 8 * kMaxStages);
-    if (TMA) pipe.init();
-    if (blockIdx.x == 0 && threadIdx.x == 0) p.ws->started_id = p.call_id;
-    if (threadIdx.x == 0) xc->abort = 0;
+    if (threadIdx.x == 0) {
+        xc->abort = 0;
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(agg_bar + 8 * b, W);
+            mbar_init(carry_bar + 8 * b, 1);
+        }
+        for (int i = 0; i < W * S; ++i) mbar_init(warp_bars + 8 * i, 1);
+        fence_mbar_init();
+        if (blockIdx.x == 0) p.ws->started_id = p.call_id;
+    }
     __syncthreads();
 
     const long long G = gridDim.x;
     const int tpr = p.tiles_per_row;
+    const long long first = blockIdx.x;
+    const long long my_tiles = first < p.num_tiles ? (p.num_tiles - first + G - 1) / G : 0;
 
-    long long issued_tile = blockIdx.x;
-    int issued = 0;
-    auto issue_next = [&]() {
-        if (issued_tile < p.num_tiles) {
-            const long long r = issued_tile / tpr;
-            const int jj = (int)(issued_tile - r * tpr);
-            pipe.issue(&tm_a, &tm_b, r, (long long)(jj * nwarps + warp) * CHUNK, issued % S);
-            issued_tile += G;
-            ++issued;
-        }
-    };
-    if (TMA) {
-        for (int s = 0; s < S - 1; ++s) issue_next();
-    }
-
-    int stage = 0;
-    uint32_t parity = 0;
-    int q = 0;
-    for (long long T = blockIdx.x; T < p.num_tiles; T += G, ++q) {
-        const long long row = T / tpr;
-        const int j = (int)(T - row * tpr);
-        const long long colbase = (long long)(j * nwarps + warp) * CHUNK;
-        const long long col0 = colbase + lane * K;
-        bool copy_failed = false;
-        if (TMA) {
-            issue_next();
-            copy_failed = !pipe.wait(stage, parity);
-        } else {
-            CE::generic_load(p, pipe.in_a(0), pipe.in_b(0), lm, lane, row, colbase);
-            __syncwarp();
-        }
-        const uint8_t* sm_a = pipe.in_a(stage);
-        const uint8_t* sm_b = pipe.in_b(stage);
-        uint8_t* sm_out = pipe.out(q & 1);
-
-        typename CE::Pending pd;
-        E total;
-        CE::phase1(p, sm_a, sm_b, off, lm, lane, row, col0, pd, total);
-        if (lane == 0) xc->agg[warp] = pack_elem<SIGNED>(total);
-        if (copy_failed && lane == 0) {
-            record_error(p, kErrCopyTimeout, T);
-            xc->abort = 1;
-        }
-        __syncthreads();  // (A) all chunk aggregates of the tile are in shared memory
-
-        if (warp == 0) {
-            E mine = (lane < nwarps) ? unpack_elem<SIGNED>(xc->agg[lane]) : identity_elem<SIGNED>();
-            E wex, tile_total;
-            warp_scan(mine, lane, wex, tile_total);
-            if (lane < nwarps) xc->wexcl[lane] = pack_elem<SIGNED>(wex);
-            const bool muted = (T == p.mute_tile);
-            E carry;
-            bool failed = false;
-            if (j == 0) {
-                carry = CE::row_start(p, row);
-            } else {
-                if (lane == 0 && !muted) LB::publish_agg(p, T, tile_total);
-                carry = LB::run(p, T, j, row, lane, failed);
+    if (warp == W) {
+        // ------------------------------------------------------------------ look-back warp
+        for (long long i = 0; i < my_tiles; ++i) {
+            const long long T = first + i * G;
+            const long long row = T / tpr;
+            const int j = (int)(T - row * tpr);
+            const int b = (int)(i & 1);
+            bool failed = !mbar_wait_bounded(agg_bar + 8 * b, (uint32_t)((i >> 1) & 1), kCopySpinLimit);
+            if (xc->abort) failed = true;
+            unsigned long long t_agg = 0;
+            unsigned int npolls = 0;
+            if (p.debug_flags & 2) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_agg));
+            E carry = identity_elem<SIGNED>();
+            if (!failed) {
+                E mine = (lane < W) ? unpack_elem<SIGNED>(xc->agg[b][lane]) : identity_elem<SIGNED>();
+                E wex, tile_total;
+                warp_scan(mine, lane, wex, tile_total);
+                if (lane < W) xc->wexcl[b][lane] = pack_elem<SIGNED>(wex);
+                const bool muted = (T == p.mute_tile);
+                if (j == 0) {
+                    carry = CE::row_start(p, row);
+                } else {
+                    if (lane == 0 && !muted) LB::publish_agg(p, T, tile_total);
+                    if (p.debug_flags & 1) carry = CE::row_start(p, row);
+                    else carry = LB::run(p, T, j, row, lane, failed, npolls);
+                }
+                if (!failed) {
+                    E incl = compose(carry, tile_total);
+                    renormalise(incl);
+                    if (lane == 0 && !muted) LB::publish_inc(p, T, incl);
+                }
             }
-            E incl = compose(carry, tile_total);
-            renormalise(incl);
             if (lane == 0) {
                 if (failed) {
                     record_error(p, kErrLookbackTimeout, T);
                     xc->abort = 1;
-                } else if (!muted) {
-                    LB::publish_inc(p, T, incl);
                 }
-                xc->carry = make_float4(carry.m, carry.s, 0.0f, 0.0f);
+                xc->carry[b] = make_float4(carry.m, carry.s, 0.0f, 0.0f);
+            }
+            if ((p.debug_flags & 2) && lane == 0) {
+                unsigned long long t_done;
+                asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_done));
+                reinterpret_cast<ulonglong2*>(p.desc + p.num_tiles)[T] = make_ulonglong2(t_agg, (t_done - t_agg) | ((unsigned long long)npolls << 32));
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(carry_bar + 8 * b);  // releases wexcl, carry and abort to the CTA
+            if (failed) break;
+        }
+        return;
+    }
+
+    // ---------------------------------------------------------------------- compute warps
+    LaneMap lm;
+    lm.R = 1; lm.g = 0; lm.i = lane; lm.W = CHUNK;
+    const typename CE::Offsets off = CE::offsets(lm);
+    uint32_t park_off[K / 4];  // the lane's K partial sums as fp32 units
+#pragma unroll
+    for (int jx = 0; jx < K / 4; ++jx) park_off[jx] = chunk_off(1, 0, (uint32_t)((lane * (K / 4) + jx) * 16));
+
+    WarpPipe<TIn, TOut, K> pipe;  // used for its TMA helpers; buffers are laid out here
+    uint8_t* wb = smem + warp * per_warp;
+    pipe.base = wb;
+    pipe.bars = warp_bars + warp * (8 * S);
+    pipe.stages = S;
+    pipe.lane = lane;
+    pipe.setup(1, p.flat_boxes != 0, p.n);
+    uint8_t* park_base = wb + S * 2 * IN_BYTES;
+    LanePark* lpark = all_parks + 2 * warp;
+    auto park_buf = [&](int b) { return park_base + b * lb_park_bytes<K>(); };
+
+    auto tile_coords = [&](long long i, long long& row, long long& colbase) {
+        const long long T = first + i * G;
+        row = T / tpr;
+        const int j = (int)(T - row * tpr);
+        colbase = ((long long)j * W + warp) * CHUNK;
+    };
+    long long issued = 0;
+    auto issue_next = [&]() {
+        if (issued < my_tiles) {
+            long long r, cb;
+            tile_coords(issued, r, cb);
+            pipe.issue(&tm_a, &tm_b, r, cb, (int)(issued % S));
+            ++issued;
+        }
+    };
+    if (TMA) issue_next();
+
+    bool aborted = false;
+    long long consumed = 0;
+    for (long long i = 0; i <= my_tiles && !aborted; ++i) {
+        // ---- phase 1 of tile i
+        if (i < my_tiles) {
+            long long row, colbase;
+            tile_coords(i, row, colbase);
+            const int st = (int)(i % S), b = (int)(i & 1);
+            if (TMA) {
+                issue_next();  // tile i+1 into the stage that tile i-2 left after its phase 2
+                if (!pipe.wait(st, (uint32_t)((i / S) & 1))) {
+                    if (lane == 0) { record_error(p, kErrCopyTimeout, first + i * G); xc->abort = 1; }
+                    aborted = true;
+                } else {
+                    ++consumed;
+                }
+            } else {
+                CE::generic_load(p, pipe.in_a(st), pipe.in_b(st), lm, lane, row, colbase);
+                __syncwarp();
+            }
+            if (!aborted) {
+                const long long col0 = colbase + lane * K;
+                typename CE::Pending pd;
+                E total;
+                CE::phase1(p, pipe.in_a(st), pipe.in_b(st), off, lm, lane, row, col0, pd, total);
+                // park what phase 2 needs; the store issued from this buffer two tiles ago has been read
+                if (TMA) { if (lane < pipe.out_boxes) bulk_wait_read<0>(); __syncwarp(); }
+                const uint32_t pb = smem_u32(park_buf(b));
+#pragma unroll
+                for (int jx = 0; jx < K / 4; ++jx) sts128(pb + park_off[jx], Storage<float>::pack(pd.run.s + 4 * jx));
+                LanePark& lp = lpark[b];
+                lp.r[lane] = pd.run.r;
+                lp.A[lane] = pd.excl.A; lp.m[lane] = pd.excl.m; lp.s[lane] = pd.excl.s;
+                if (SIGNED) lp.p[lane] = pd.excl.p;
+                if (lane == 0) {
+                    lp.slow = pd.slow ? 1 : 0;
+                    xc->agg[b][warp] = pack_elem<SIGNED>(total);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(agg_bar + 8 * b);
             }
         }
-        __syncthreads();  // (B) the value entering the tile is known
-        if (xc->abort) {
-            if (TMA) pipe.drain_loads(copy_failed ? q + 2 : q + 1, issued);
-            break;
+        // ---- phase 2 of tile i-1
+        if (i >= 1 && !aborted) {
+            const long long ip = i - 1;
+            long long row, colbase;
+            tile_coords(ip, row, colbase);
+            const int st = (int)(ip % S), b = (int)(ip & 1);
+            if (!mbar_wait_bounded(carry_bar + 8 * b, (uint32_t)((ip >> 1) & 1), kCopySpinLimit)) {
+                if (lane == 0) { record_error(p, kErrLookbackTimeout, first + ip * G); xc->abort = 1; }
+                aborted = true;
+            } else if (xc->abort) {
+                aborted = true;
+            }
+            if (!aborted) {
+                const long long col0 = colbase + lane * K;
+                const long long left = p.n - col0;
+                E carry;
+                carry.A = neg_inf(); carry.m = xc->carry[b].x; carry.s = xc->carry[b].y; carry.p = 0u;
+                const LanePark& lp = lpark[b];
+                E excl;
+                excl.A = lp.A[lane]; excl.m = lp.m[lane]; excl.s = lp.s[lane]; excl.p = SIGNED ? lp.p[lane] : 0u;
+                const E entering = compose(compose(carry, unpack_elem<SIGNED>(xc->wexcl[b][warp])), excl);
+                const uint8_t* sm_a = pipe.in_a(st);
+                const uint8_t* sm_b = pipe.in_b(st);
+                uint8_t* sm_out = park_buf(b);
+                const uint32_t pb = smem_u32(sm_out);
+                float out_mag[K];
+                uint32_t out_sign[MODE == kLogSigned ? K : 1];
+                bool ok = false;
+                if (!lp.slow) {
+                    // rebuild A_t (and the parity of a) from the inputs, fetch the parked s_t, apply
+                    float va[K];
+                    uint32_t sa[MODE == kLogSigned ? K : 1];
+                    R_::load_a(sm_a, off.in, va);
+                    if (left < K) {
+#pragma unroll
+                        for (int t = 0; t < K; ++t)
+                            if (t >= left) va[t] = neutral_a<MODE>();
+                    }
+                    if (MODE == kLogSigned) CE::load_signs(p.sign_a, row * p.n + col0, left, p.sign_vec_ok != 0, sa);
+                    R_ run;
+                    run.rebuild(va, sa);
+                    run.r = lp.r[lane];
+#pragma unroll
+                    for (int jx = 0; jx < K / 4; ++jx) Storage<float>::unpack(lds128(pb + park_off[jx]), run.s + 4 * jx);
+                    ok = run.apply(entering, out_mag, out_sign);
+                }
+                ok = __all_sync(0xffffffffu, ok);  // also: every lane has read its parked sums
+                if (ok) {
+#pragma unroll
+                    for (int jx = 0; jx < CE::OUT_UNITS; ++jx)
+                        sts128(pb + off.out[jx], Storage<TOut>::pack(out_mag + jx * Storage<TOut>::kPerUnit));
+                    if (MODE == kLogSigned) CE::store_signs(p.sign_x, row * p.n + col0, left, p.sign_vec_ok != 0, out_sign);
+                } else {
+                    const typename CE::SlowOut so =
+                        CE::slow_apply(entering, sm_a, sm_b, lm, MODE == kLogSigned ? p.sign_a : nullptr,
+                                       MODE == kLogSigned ? p.sign_b : nullptr, row * p.n + col0, left);
+#pragma unroll
+                    for (int jx = 0; jx < CE::OUT_UNITS; ++jx)
+                        sts128(pb + off.out[jx], Storage<TOut>::pack(so.vals + jx * Storage<TOut>::kPerUnit));
+                    if (MODE == kLogSigned) CE::store_signs(p.sign_x, row * p.n + col0, left, p.sign_vec_ok != 0, so.sgn);
+                }
+                if (TMA) {
+                    // a chunk wholly beyond the row end has nothing to store (a flat box is not clipped per row)
+                    if (colbase < p.n) pipe.store_from(&tm_o, row, colbase, pb);
+                } else {
+                    __syncwarp();
+                    CE::generic_store(p, sm_out, lm, lane, row, colbase);
+                }
+                __syncwarp();  // every lane is done with this tile's input stage
+            }
         }
-
-        E carry;
-        carry.A = neg_inf(); carry.m = xc->carry.x; carry.s = xc->carry.y; carry.p = 0u;
-        const E entering_chunk = compose(carry, unpack_elem<SIGNED>(xc->wexcl[warp]));
-        if (TMA) pipe.acquire_out();
-        CE::phase2(p, sm_a, sm_b, sm_out, off, lm, row, col0, pd, entering_chunk);
-        if (TMA) {
-            pipe.store(&tm_o, row, colbase, q & 1);
-        } else {
-            __syncwarp();
-            CE::generic_store(p, sm_out, lm, lane, row, colbase);
-        }
-        __syncwarp();
-        if (++stage == S) { stage = 0; parity ^= 1u; }
     }
-    if (TMA) pipe.drain();
+    if (TMA) {
+        if (aborted) pipe.drain_loads(consumed, issued);
+        pipe.drain();
+    }
 }
 
 }  // namespace hs
