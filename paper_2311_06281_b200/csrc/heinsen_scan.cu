@@ -139,18 +139,21 @@ struct KernelEntry {
     int K;
     int warp_smem_per_stage;  // bytes of one input stage (both tensors) of one warp
     int warp_smem_out;        // bytes of both output buffers of one warp
-    int (*lb_smem)(int);      // dynamic shared memory of the look-back kernel for W compute warps
+    int (*lb_smem)(int, int); // dynamic shared memory of the look-back kernel for W compute warps, S stages
+    int lb_K;                 // elements per lane per chunk in the look-back kernel
 };
 
 template <int MODE, typename TIn, typename TOut, int K, bool TMA>
 KernelEntry entry() {
     KernelEntry e;
+    constexpr int LBK = 16;  // the look-back kernel parks fp32 partial sums: 16 per lane for every type
     e.batched = reinterpret_cast<const void*>(&batched_scan_kernel<MODE, TIn, TOut, K, TMA>);
-    e.lookback = reinterpret_cast<const void*>(&lookback_scan_kernel<MODE, TIn, TOut, K, TMA>);
+    e.lookback = reinterpret_cast<const void*>(&lookback_scan_kernel<MODE, TIn, TOut, LBK, TMA>);
+    e.lb_K = LBK;
     e.K = K;
     e.warp_smem_per_stage = 2 * 32 * K * (int)sizeof(TIn);
     e.warp_smem_out = 2 * 32 * K * (int)sizeof(TOut);
-    e.lb_smem = [](int W) { return lb_total_smem_bytes<TIn, K>(W); };
+    e.lb_smem = [](int W, int S) { return lb_total_smem_bytes<TIn, LBK>(W, S); };
     return e;
 }
 
@@ -194,8 +197,9 @@ int choose_path(long long rows, const DeviceInfo& d) {
 
 size_t workspace_bytes_for(long long rows, long long n) {
     // sized for the smallest chunk so that it covers every type
-    const long long tiles = rows * lookback_tiles_per_row(n, kMinChunk, kLookbackMinWarps);
-    return sizeof(Header) + (size_t)tiles * 16;
+    const long long tpr = lookback_tiles_per_row(n, kMinChunk, kLookbackMinWarps);
+    const long long gpr = (tpr + kLbGroup - 1) / kLbGroup;
+    return sizeof(Header) + (size_t)(rows * (tpr + gpr)) * 16;
 }
 
 // cudaFuncSetAttribute and the occupancy query cost microseconds per call; remember what was set.
@@ -270,7 +274,8 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
 
     KernelEntry ke;
     if (!find_kernel(pr.mode, pr.din, pr.dout, tma, ke)) return HS_ERR_INVALID_ARG;
-    const int chunk = 32 * ke.K;
+    const int path = choose_path(p.rows, dev);
+    const int chunk = 32 * (path == HS_PATH_BATCHED ? ke.K : ke.lb_K);  // elements per warp per step
     p.nchunks = (int)((p.n + chunk - 1) / chunk);
     p.sign_vec_ok = (p.n % 16 == 0) && (!p.sign_a || aligned16(p.sign_a)) && (!p.sign_b || aligned16(p.sign_b)) &&
                     (!p.sign_x || aligned16(p.sign_x));
@@ -280,8 +285,7 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
     p.debug_flags = env_int("HEINSEN_SCAN_DEBUG_FLAGS", 0, 0, 255);
     p.ws = reinterpret_cast<Header*>(workspace);
 
-    const int path = choose_path(p.rows, dev);
-    int warps, stages, grid;
+    int warps, stages, grid, lb_smem = 0;
     const void* fn;
     if (path == HS_PATH_BATCHED) {
         // R rows per warp (32/R lanes per row): the largest R that still leaves about a dozen warps
@@ -305,16 +309,22 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         fn = ke.batched;
     } else {
         p.rows_per_warp = 1;
-        // W compute warps (as many as shared memory allows, at most the default) + 1 look-back warp
+        // S input stages per compute warp (phase 2 of a tile runs S-2 iterations after its phase 1),
+        // W compute warps (as many as shared memory allows, at most the default), NLB look-back warps
+        stages = env_int("HEINSEN_SCAN_LB_STAGES", 4, 3, kLbMaxStages);
+        const int nlb = env_int("HEINSEN_SCAN_LB_LOOKERS", 3, 1, 4);
         int W = env_int("HEINSEN_SCAN_LB_WARPS", kLookbackWarps, kLookbackMinWarps, kLbMaxWarps);
-        while (W > kLookbackMinWarps && ke.lb_smem(W) + 1024 > dev.max_smem_optin) --W;
-        warps = W + 1;
-        stages = kLbStages;
+        while (W > kLookbackMinWarps && ke.lb_smem(W, stages) + 1024 > dev.max_smem_optin) --W;
+        lb_smem = ke.lb_smem(W, stages) + 1024;
+        p.lb_warps = nlb;
+        warps = W + nlb;
         p.tiles_per_row = (int)lookback_tiles_per_row(p.n, chunk, W);
         p.num_tiles = p.rows * p.tiles_per_row;
-        const size_t need = sizeof(Header) + (size_t)p.num_tiles * 16;
+        p.groups_per_row = (p.tiles_per_row + kLbGroup - 1) / kLbGroup;
+        const size_t need = sizeof(Header) + ((size_t)p.num_tiles + (size_t)p.rows * p.groups_per_row) * 16;
         if (workspace_bytes < need) return HS_ERR_WORKSPACE_TOO_SMALL;
         p.desc = reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(workspace) + sizeof(Header));
+        p.gdesc = p.desc + p.num_tiles;
         fn = ke.lookback;
         grid = 0;  // set below from occupancy
     }
@@ -339,7 +349,7 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
     }
     p.stages = stages;
     const int smem = path == HS_PATH_LOOKBACK
-                         ? ke.lb_smem(warps - 1) + 1024
+                         ? lb_smem
                          : warps * (stages * ke.warp_smem_per_stage + ke.warp_smem_out) + warps * 8 * kMaxStages + 1024;
     if (smem > dev.max_smem_optin) return HS_ERR_INVALID_ARG;
     cudaError_t e = ensure_smem_attr(fn, smem);
@@ -358,7 +368,7 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         if (g > p.num_tiles) g = p.num_tiles;
         grid = (int)g;
         // every descriptor starts as "nothing yet"
-        e = cudaMemsetAsync(p.desc, 0, (size_t)p.num_tiles * 16, stream);
+        e = cudaMemsetAsync(p.desc, 0, ((size_t)p.num_tiles + (size_t)p.rows * p.groups_per_row) * 16, stream);
         if (e != cudaSuccess) return cuda_fail("cudaMemsetAsync", e);
         e = cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(warps * 32), args, smem, stream);
     } else {

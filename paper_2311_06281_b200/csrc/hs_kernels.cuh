@@ -57,6 +57,9 @@ struct Params {
     int tiles_per_row;
     long long num_tiles;
     uint4* desc;                // [num_tiles] tile descriptors, zeroed before the launch
+    uint4* gdesc;               // [rows * groups_per_row] group descriptors, zeroed before the launch
+    int groups_per_row;         // ceil(tiles_per_row / 32)
+    int lb_warps;               // look-back warps per CTA
     unsigned int spin_limit;    // bound on polls of predecessor flags
     long long mute_tile;        // test hook: this tile never publishes (-1: none)
     int debug_flags;            // timing experiments only (results are wrong when non-zero)
@@ -513,10 +516,10 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
 // pipelined so that the latency of the look-back never stalls the arithmetic:
 //
 //   compute warp, iteration i :  phase 1 of tile i   (inputs -> partial sums s_t parked in shared
-//                                                     memory, chunk aggregate handed to the
+//                                                     memory, chunk aggregate handed to a
 //                                                     look-back warp)
-//                                phase 2 of tile i-1 (whose entering value has arrived meanwhile:
-//                                                     outputs, TMA store)
+//                                phase 2 of tile i-D (whose entering value has arrived meanwhile:
+//                                                     outputs, TMA store), D = stages - 2
 //   look-back warp, tile i    :  scan of the W chunk aggregates, publish the tile aggregate,
 //                                assemble the value of x entering the tile from the descriptors
 //                                of the preceding tiles (aggregates until a tile whose value is
@@ -543,10 +546,17 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
-constexpr int kLookPerLane = 8;                     // predecessors polled by each lane per round
-constexpr int kLookWindow = 32 * kLookPerLane;      // tiles covered by one round
+constexpr int kLbGroup = 32;                        // tiles per group (one per lane)
 constexpr int kLbMaxWarps = 16;                     // compute warps per CTA, at most
 
+// Two levels of descriptors keep a look-back short however many tiles are in flight:
+//   tile level  : desc[T]   = aggregate of tile T (state 1), written right after its phase 1;
+//   group level : gdesc[g]  = aggregate of the 32 tiles of group g (state 1), written by the
+//                 look-back of the group's last tile as soon as it has seen the other 31, and
+//                 later replaced by the value of x after the group (state 2).
+// The value entering tile j = (value before its group, from group descriptors: aggregates back
+// to the nearest known value) composed with (the aggregates of the tiles of its own group before
+// it).  One round reads at most 31 + 32 descriptors, one or two per lane, all in flight at once.
 template <int MODE, typename TIn, typename TOut, int K>
 struct Lookback {
     using CE = ChunkEngine<MODE, TIn, TOut, K>;
@@ -572,92 +582,102 @@ struct Lookback {
     __device__ static __forceinline__ void publish_agg(const Params& p, long long T, const E& e) {
         st_desc(p.desc + T, pack(e, kAgg));
     }
-    __device__ static __forceinline__ void publish_inc(const Params& p, long long T, E e) {
-        e.A = neg_inf();
-        e.p = 0u;
-        st_desc(p.desc + T, pack(e, kInc));
+
+    // lane 0 holds the newest part, higher lanes older ones; returns their composition in every lane
+    __device__ static __forceinline__ E reduce_newest_first(E part, int lane) {
+#pragma unroll
+        for (int dd = 1; dd < 32; dd <<= 1) {
+            E other = shfl_down_elem(part, dd);
+            E c = compose(other, part);
+            if (lane + dd < 32) part = c;
+        }
+        return shfl_elem(part, 0);
+    }
+    __device__ static __forceinline__ bool give_up(const Params& p, unsigned int& polls) {
+        return ++polls >= p.spin_limit ||
+               ((polls & 255u) == 0u && *(volatile unsigned long long*)&p.ws->error_id == p.call_id);
     }
 
-    // Warp-collective.  Returns the value of x entering tile T (tile j of `row`), j >= 1.
-    // One round reads the descriptors of up to kLookWindow preceding tiles, all loads in flight
-    // at once; lane l looks at distances base + 8l .. base + 8l + 7, nearest first.
-    __device__ static __forceinline__ E run(const Params& p, long long T, int j, long long row, int lane, bool& failed,
-                                            unsigned int& total_polls) {
-        E acc = identity_elem<SIGNED>();
+    // Warp-collective.  Tile T is tile j of `row`; tile_total its aggregate.  Returns the value of
+    // x entering the tile and publishes the group descriptors this tile is responsible for.
+    __device__ static __forceinline__ E run(const Params& p, long long T, int j, long long row, int lane,
+                                            const E& tile_total, bool publish, bool& failed, unsigned int& total_polls) {
         failed = false;
-        const E x0e = CE::row_start(p, row);
-        for (int base = 1;; base += kLookWindow) {
-            Desc d[kLookPerLane];
-            bool complete = false, has_inc = false;
-            uint32_t inc_mask = 0u;
-            unsigned int polls = 0;
+        const int g = j / kLbGroup, k = j - g * kLbGroup;          // group, position in group
+        const long long gbase = row * p.groups_per_row;            // first group descriptor of the row
+        const bool closes_group = (k == kLbGroup - 1) || (j == p.tiles_per_row - 1);
+        unsigned int polls = 0;
+
+        // ---- tiles of the own group before this one: lane l looks at tile j-1-l (l < k)
+        E part = identity_elem<SIGNED>();
+        if (k > 0) {
+            Desc d;
+            d.lo = 0ull; d.hi = 0ull;
             while (true) {
-#pragma unroll
-                for (int q = 0; q < kLookPerLane; ++q) {
-                    const int dist = base + kLookPerLane * lane + q;
-                    if (j - dist >= 0) d[q] = ld_desc(p.desc + (T - dist));
-                    else { d[q].lo = 0ull; d[q].hi = 0ull; }
-                }
-                complete = true;
-                has_inc = false;
-#pragma unroll
-                for (int q = 0; q < kLookPerLane; ++q) {
-                    const int jj = j - (base + kLookPerLane * lane + q);
-                    const uint32_t s = (jj >= 0) ? state_of(d[q]) : (uint32_t)kInc;  // jj == -1: x_0; beyond: ignored
-                    if (!has_inc && complete) {  // ready prefix of this lane, up to its first known value
-                        if (s == kNotReady) complete = false;
-                        else if (s == kInc) has_inc = true;
-                    }
-                }
-                inc_mask = __ballot_sync(0xffffffffu, complete && has_inc);
-                const uint32_t ok_mask = __ballot_sync(0xffffffffu, complete);
+                if (lane < k) d = ld_desc(p.desc + (T - 1 - lane));
+                const bool ready = (lane >= k) || state_of(d) == kAgg;
+                ++total_polls;
+                if (__all_sync(0xffffffffu, ready)) break;
+                if (give_up(p, polls)) { failed = true; return part; }
+            }
+            if (lane < k) part = unpack(d);
+        }
+        const E before_in_group = reduce_newest_first(part, lane);
+        if (closes_group && publish && lane == 0 && k == kLbGroup - 1) {
+            // the other tiles need only this, not our own carry: publish it at once
+            st_desc(p.gdesc + gbase + g, pack(compose(before_in_group, tile_total), kAgg));
+        }
+
+        // ---- groups before the own one: lane l looks at group g-1-l; group -1 is x_0
+        E acc = identity_elem<SIGNED>();
+        const E x0e = CE::row_start(p, row);
+        for (int base = 1;; base += 32) {
+            const int gg = g - base - lane;
+            Desc d;
+            d.lo = 0ull; d.hi = 0ull;
+            uint32_t inc_mask = 0u;
+            while (true) {
+                if (gg >= 0) d = ld_desc(p.gdesc + gbase + gg);
+                const uint32_t s = (gg >= 0) ? state_of(d) : (uint32_t)kInc;  // gg == -1: x_0; beyond: ignored
+                inc_mask = __ballot_sync(0xffffffffu, s == kInc);
+                const uint32_t ok_mask = __ballot_sync(0xffffffffu, s != kNotReady);
                 const uint32_t need = inc_mask ? ((2u << (__ffs(inc_mask) - 1)) - 1u) : 0xffffffffu;
                 ++total_polls;
                 if ((ok_mask & need) == need) break;
-                if (++polls >= p.spin_limit ||
-                    ((polls & 255u) == 0u && *(volatile unsigned long long*)&p.ws->error_id == p.call_id)) {
-                    failed = true;
-                    return acc;
-                }
+                if (give_up(p, polls)) { failed = true; return acc; }
             }
             const int lstar = inc_mask ? (__ffs(inc_mask) - 1) : 31;
-            E part = identity_elem<SIGNED>();
-            bool stop = lane > lstar;
-#pragma unroll
-            for (int q = 0; q < kLookPerLane; ++q) {
-                const int jj = j - (base + kLookPerLane * lane + q);
-                if (!stop) {
-                    const E e = (jj >= 0) ? unpack(d[q]) : x0e;
-                    if (jj < 0 || state_of(d[q]) == kInc) stop = true;
-                    part = compose(e, part);  // e is older than everything folded so far
-                }
-            }
-            // ordered reduction: lane 0 holds the newest tiles, higher lanes older ones
-#pragma unroll
-            for (int dd = 1; dd < 32; dd <<= 1) {
-                E other = shfl_down_elem(part, dd);
-                E c = compose(other, part);
-                if (lane + dd < 32) part = c;
-            }
-            const E window = shfl_elem(part, 0);
-            acc = compose(window, acc);
-            if (inc_mask) return acc;
+            E gp = identity_elem<SIGNED>();
+            if (lane <= lstar) gp = (gg >= 0) ? unpack(d) : x0e;
+            acc = compose(reduce_newest_first(gp, lane), acc);
+            if (inc_mask) break;
         }
+        const E entering = compose(acc, before_in_group);
+        if (closes_group && publish && lane == 0) {
+            E after = compose(entering, tile_total);
+            renormalise(after);
+            after.A = neg_inf();
+            after.p = 0u;
+            st_desc(p.gdesc + gbase + g, pack(after, kInc));
+        }
+        return entering;
     }
 };
 
-// CTA-level exchange between the compute warps and the look-back warp (two tiles in flight).
+// CTA-level exchange between the compute warps and the look-back warps (a ring of tiles in flight).
+constexpr int kLbRing = 4;      // ring slots: tiles between "aggregate delivered" and "carry consumed"
+constexpr int kLbMaxStages = 5; // input stages per compute warp, at most
 struct alignas(16) Exchange {
-    float4 agg[2][kLbMaxWarps];    // per-warp aggregates of a tile
-    float4 wexcl[2][kLbMaxWarps];  // per-warp exclusive prefixes within the tile
-    float4 carry[2];               // value of x entering the tile (m, s)
-    unsigned long long agg_ready[2];    // mbarrier: all compute warps have delivered their aggregate
-    unsigned long long carry_ready[2];  // mbarrier: the look-back warp has delivered wexcl and carry
+    float4 agg[kLbRing][kLbMaxWarps];    // per-warp aggregates of a tile
+    float4 wexcl[kLbRing][kLbMaxWarps];  // per-warp exclusive prefixes within the tile
+    float4 carry[kLbRing];               // value of x entering the tile (m, s)
+    unsigned long long agg_ready[kLbRing];    // mbarrier: all compute warps have delivered their aggregate
+    unsigned long long carry_ready[kLbRing];  // mbarrier: a look-back warp has delivered wexcl and carry
     int abort;
     int pad[3];
 };
 
-// Per-lane state parked between the two phases of a chunk (structure of arrays, one per buffer).
+// Per-lane state parked between the two phases of a chunk (structure of arrays, one per stage).
 struct LanePark {
     float r[32];
     float A[32], m[32], s[32];
@@ -677,56 +697,56 @@ __device__ __forceinline__ Elem<SIGNED> unpack_elem(const float4 v) {
     return e;
 }
 
-constexpr int kLbStages = 3;  // input stages per compute warp: tile i-1 (awaiting phase 2), i, i+1 (in flight)
-
-template <int K>
-__host__ __device__ constexpr int lb_park_bytes() { return 32 * K * 4; }  // s_t as fp32; outputs reuse it
-
-// Chunk buffers of one compute warp of the look-back kernel (a multiple of 1024 bytes: the
-// swizzled layouts need 1024-byte aligned buffers); its two LanePark records live after the
-// chunk buffers of all warps.
+// One input stage of a compute warp: [a-tensor chunk][b-tensor chunk][park].  The partial sums
+// s_t (fp32) of phase 1 are parked over the b-tensor chunk when the input type is 4 bytes wide
+// (in place), else in a region of their own; the outputs of phase 2 are written over the parked
+// sums and stored from there.
 template <typename TIn, int K>
-__host__ __device__ constexpr int lb_warp_smem_bytes() {
-    return kLbStages * 2 * 32 * K * (int)sizeof(TIn) + 2 * lb_park_bytes<K>();
-}
-static_assert(lb_warp_smem_bytes<float, 16>() % 1024 == 0 && lb_warp_smem_bytes<__nv_bfloat16, 32>() % 1024 == 0, "");
-// total dynamic shared memory of the look-back kernel for W compute warps (without alignment slack)
+struct LbStage {
+    static constexpr int IN_BYTES = 32 * K * (int)sizeof(TIn);
+    static constexpr bool IN_PLACE = sizeof(TIn) == 4;
+    static constexpr int PARK_OFF = IN_PLACE ? IN_BYTES : 2 * IN_BYTES;
+    static constexpr int BYTES = IN_PLACE ? 2 * IN_BYTES : 2 * IN_BYTES + 32 * K * 4;
+    static_assert(BYTES % 1024 == 0 && PARK_OFF % 1024 == 0, "swizzled buffers need 1024-byte alignment");
+};
+// total dynamic shared memory of the look-back kernel for W compute warps and S stages (without alignment slack)
 template <typename TIn, int K>
-__host__ __device__ constexpr int lb_total_smem_bytes(int W) {
-    return W * (lb_warp_smem_bytes<TIn, K>() + 2 * (int)sizeof(LanePark)) + (int)sizeof(Exchange) + W * kLbStages * 8;
+__host__ __device__ constexpr int lb_total_smem_bytes(int W, int S) {
+    return W * S * (LbStage<TIn, K>::BYTES + (int)sizeof(LanePark)) + (int)sizeof(Exchange) + W * kLbMaxStages * 8;
 }
 
 template <int MODE, typename TIn, typename TOut, int K, bool TMA>
-__global__ void __launch_bounds__(544, 1)
+__global__ void __launch_bounds__(640, 1)
 lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                      const __grid_constant__ CUtensorMap tm_o) {
     using CE = ChunkEngine<MODE, TIn, TOut, K>;
     using LB = Lookback<MODE, TIn, TOut, K>;
     using R_ = Run<MODE, TIn, TOut, K>;
+    using ST = LbStage<TIn, K>;
     using E = typename CE::E;
     constexpr bool SIGNED = CE::SIGNED;
     constexpr int CHUNK = 32 * K;
-    constexpr int IN_BYTES = CHUNK * (int)sizeof(TIn);
-    constexpr int S = kLbStages;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align_1024(smem_raw);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int W = (blockDim.x >> 5) - 1;  // compute warps; warp W is the look-back warp
-    constexpr int per_warp = lb_warp_smem_bytes<TIn, K>();
+    const int NLB = p.lb_warps;                 // look-back warps (the last NLB warps of the CTA)
+    const int W = (blockDim.x >> 5) - NLB;      // compute warps
+    const int S = p.stages;                     // input stages per compute warp
+    const int D = S - 2;                        // phase 2 of a tile runs D iterations after its phase 1
 
-    uint8_t* tail = smem + W * per_warp;
-    LanePark* all_parks = reinterpret_cast<LanePark*>(tail);  // [W][2]
-    Exchange* xc = reinterpret_cast<Exchange*>(tail + W * 2 * sizeof(LanePark));
-    const uint32_t warp_bars = smem_u32(reinterpret_cast<uint8_t*>(xc) + sizeof(Exchange));  // W x S stage mbarriers
+    uint8_t* tail = smem + (size_t)W * S * ST::BYTES;
+    LanePark* all_parks = reinterpret_cast<LanePark*>(tail);  // [W][S]
+    Exchange* xc = reinterpret_cast<Exchange*>(tail + (size_t)W * S * sizeof(LanePark));
+    const uint32_t warp_bars = smem_u32(reinterpret_cast<uint8_t*>(xc) + sizeof(Exchange));  // [W][kLbMaxStages]
     const uint32_t agg_bar = smem_u32(&xc->agg_ready[0]), carry_bar = smem_u32(&xc->carry_ready[0]);
 
     if (threadIdx.x == 0) {
         xc->abort = 0;
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < kLbRing; ++b) {
             mbar_init(agg_bar + 8 * b, W);
             mbar_init(carry_bar + 8 * b, 1);
         }
-        for (int i = 0; i < W * S; ++i) mbar_init(warp_bars + 8 * i, 1);
+        for (int i = 0; i < W * kLbMaxStages; ++i) mbar_init(warp_bars + 8 * i, 1);
         fence_mbar_init();
         if (blockIdx.x == 0) p.ws->started_id = p.call_id;
     }
@@ -737,15 +757,17 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
     const long long first = blockIdx.x;
     const long long my_tiles = first < p.num_tiles ? (p.num_tiles - first + G - 1) / G : 0;
 
-    if (warp == W) {
-        // ------------------------------------------------------------------ look-back warp
-        for (long long i = 0; i < my_tiles; ++i) {
+    if (warp >= W) {
+        // ------------------------------------------------------------------ look-back warps
+        // Warp u of NLB takes the CTA's tiles u, u+NLB, u+2*NLB, ...: a tile's look-back lasts
+        // several L2 round trips, longer than a tile's arithmetic, so several are in flight.
+        for (long long i = warp - W; i < my_tiles; i += NLB) {
             const long long T = first + i * G;
             const long long row = T / tpr;
             const int j = (int)(T - row * tpr);
-            const int b = (int)(i & 1);
-            bool failed = !mbar_wait_bounded(agg_bar + 8 * b, (uint32_t)((i >> 1) & 1), kCopySpinLimit);
-            if (xc->abort) failed = true;
+            const int b = (int)(i % kLbRing);
+            bool failed = !mbar_wait_bounded(agg_bar + 8 * b, (uint32_t)((i / kLbRing) & 1), kCopySpinLimit);
+            if (*(volatile int*)&xc->abort) failed = true;
             unsigned long long t_agg = 0;
             unsigned int npolls = 0;
             if (p.debug_flags & 2) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_agg));
@@ -756,18 +778,9 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                 warp_scan(mine, lane, wex, tile_total);
                 if (lane < W) xc->wexcl[b][lane] = pack_elem<SIGNED>(wex);
                 const bool muted = (T == p.mute_tile);
-                if (j == 0) {
-                    carry = CE::row_start(p, row);
-                } else {
-                    if (lane == 0 && !muted) LB::publish_agg(p, T, tile_total);
-                    if (p.debug_flags & 1) carry = CE::row_start(p, row);
-                    else carry = LB::run(p, T, j, row, lane, failed, npolls);
-                }
-                if (!failed) {
-                    E incl = compose(carry, tile_total);
-                    renormalise(incl);
-                    if (lane == 0 && !muted) LB::publish_inc(p, T, incl);
-                }
+                if (lane == 0 && !muted) LB::publish_agg(p, T, tile_total);
+                if (p.debug_flags & 1) carry = CE::row_start(p, row);
+                else carry = LB::run(p, T, j, row, lane, tile_total, !muted, failed, npolls);
             }
             if (lane == 0) {
                 if (failed) {
@@ -779,7 +792,8 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
             if ((p.debug_flags & 2) && lane == 0) {
                 unsigned long long t_done;
                 asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_done));
-                reinterpret_cast<ulonglong2*>(p.desc + p.num_tiles)[T] = make_ulonglong2(t_agg, (t_done - t_agg) | ((unsigned long long)npolls << 32));
+                reinterpret_cast<ulonglong2*>(p.gdesc + p.rows * p.groups_per_row)[T] =
+                    make_ulonglong2(t_agg, (t_done - t_agg) | ((unsigned long long)npolls << 32));
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(carry_bar + 8 * b);  // releases wexcl, carry and abort to the CTA
@@ -796,16 +810,18 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
 #pragma unroll
     for (int jx = 0; jx < K / 4; ++jx) park_off[jx] = chunk_off(1, 0, (uint32_t)((lane * (K / 4) + jx) * 16));
 
-    WarpPipe<TIn, TOut, K> pipe;  // used for its TMA helpers; buffers are laid out here
-    uint8_t* wb = smem + warp * per_warp;
-    pipe.base = wb;
-    pipe.bars = warp_bars + warp * (8 * S);
-    pipe.stages = S;
-    pipe.lane = lane;
-    pipe.setup(1, p.flat_boxes != 0, p.n);
-    uint8_t* park_base = wb + S * 2 * IN_BYTES;
-    LanePark* lpark = all_parks + 2 * warp;
-    auto park_buf = [&](int b) { return park_base + b * lb_park_bytes<K>(); };
+    uint8_t* wb = smem + (size_t)warp * S * ST::BYTES;
+    auto st_a = [&](int st) { return wb + st * ST::BYTES; };
+    auto st_b = [&](int st) { return wb + st * ST::BYTES + ST::IN_BYTES; };
+    auto st_park = [&](int st) { return wb + st * ST::BYTES + ST::PARK_OFF; };
+    LanePark* lpark = all_parks + (size_t)warp * S;
+    const uint32_t bars = warp_bars + warp * (8 * kLbMaxStages);
+
+    // TMA helpers (same box geometry as WarpPipe, buffers laid out per stage here)
+    const bool flat = p.flat_boxes != 0;
+    constexpr int IN_PER_BOX = 128 / (int)sizeof(TIn), OUT_PER_BOX = 128 / (int)sizeof(TOut);
+    const int in_boxes = flat ? 1 : ST::IN_BYTES / 128;
+    const int out_boxes = flat ? 1 : (CHUNK * (int)sizeof(TOut)) / 128;
 
     auto tile_coords = [&](long long i, long long& row, long long& colbase) {
         const long long T = first + i * G;
@@ -818,7 +834,21 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
         if (issued < my_tiles) {
             long long r, cb;
             tile_coords(issued, r, cb);
-            pipe.issue(&tm_a, &tm_b, r, cb, (int)(issued % S));
+            const int st = (int)(issued % S);
+            const uint32_t bar = bars + 8 * st;
+            if (lane == 0) mbar_expect_tx(bar, 2 * ST::IN_BYTES);
+            __syncwarp();
+            if (flat) {
+                if (lane == 0) {
+                    const int line = (int)((r * p.n + cb) / IN_PER_BOX);
+                    tma_load_2d(smem_u32(st_a(st)), &tm_a, 0, line, bar);
+                    tma_load_2d(smem_u32(st_b(st)), &tm_b, 0, line, bar);
+                }
+            } else if (lane < in_boxes) {
+                const int x = (int)cb + lane * IN_PER_BOX;
+                tma_load_2d(smem_u32(st_a(st)) + lane * 128, &tm_a, x, (int)r, bar);
+                tma_load_2d(smem_u32(st_b(st)) + lane * 128, &tm_b, x, (int)r, bar);
+            }
             ++issued;
         }
     };
@@ -826,35 +856,39 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
 
     bool aborted = false;
     long long consumed = 0;
-    for (long long i = 0; i <= my_tiles && !aborted; ++i) {
+    for (long long i = 0; i < my_tiles + D && !aborted; ++i) {
         // ---- phase 1 of tile i
         if (i < my_tiles) {
             long long row, colbase;
             tile_coords(i, row, colbase);
-            const int st = (int)(i % S), b = (int)(i & 1);
+            const int st = (int)(i % S), b = (int)(i % kLbRing);
             if (TMA) {
-                issue_next();  // tile i+1 into the stage that tile i-2 left after its phase 2
-                if (!pipe.wait(st, (uint32_t)((i / S) & 1))) {
+                // tile i+1 goes into the stage whose tile finished phase 2 in the previous iteration;
+                // the store issued from it then has been read by now
+                if (lane < out_boxes) bulk_wait_read<0>();
+                __syncwarp();
+                issue_next();
+                if (!mbar_wait_bounded(bars + 8 * st, (uint32_t)((i / S) & 1), kCopySpinLimit)) {
                     if (lane == 0) { record_error(p, kErrCopyTimeout, first + i * G); xc->abort = 1; }
                     aborted = true;
                 } else {
                     ++consumed;
                 }
             } else {
-                CE::generic_load(p, pipe.in_a(st), pipe.in_b(st), lm, lane, row, colbase);
+                CE::generic_load(p, st_a(st), st_b(st), lm, lane, row, colbase);
                 __syncwarp();
             }
             if (!aborted) {
                 const long long col0 = colbase + lane * K;
                 typename CE::Pending pd;
                 E total;
-                CE::phase1(p, pipe.in_a(st), pipe.in_b(st), off, lm, lane, row, col0, pd, total);
-                // park what phase 2 needs; the store issued from this buffer two tiles ago has been read
-                if (TMA) { if (lane < pipe.out_boxes) bulk_wait_read<0>(); __syncwarp(); }
-                const uint32_t pb = smem_u32(park_buf(b));
+                CE::phase1(p, st_a(st), st_b(st), off, lm, lane, row, col0, pd, total);
+                LanePark& lp = lpark[st];
+                if (!pd.slow) {  // park the partial sums (a slow chunk keeps its inputs instead)
+                    const uint32_t pb = smem_u32(st_park(st));
 #pragma unroll
-                for (int jx = 0; jx < K / 4; ++jx) sts128(pb + park_off[jx], Storage<float>::pack(pd.run.s + 4 * jx));
-                LanePark& lp = lpark[b];
+                    for (int jx = 0; jx < K / 4; ++jx) sts128(pb + park_off[jx], Storage<float>::pack(pd.run.s + 4 * jx));
+                }
                 lp.r[lane] = pd.run.r;
                 lp.A[lane] = pd.excl.A; lp.m[lane] = pd.excl.m; lp.s[lane] = pd.excl.s;
                 if (SIGNED) lp.p[lane] = pd.excl.p;
@@ -866,16 +900,16 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                 if (lane == 0) mbar_arrive(agg_bar + 8 * b);
             }
         }
-        // ---- phase 2 of tile i-1
-        if (i >= 1 && !aborted) {
-            const long long ip = i - 1;
+        // ---- phase 2 of tile i-D
+        if (i >= D && !aborted) {
+            const long long ip = i - D;
             long long row, colbase;
             tile_coords(ip, row, colbase);
-            const int st = (int)(ip % S), b = (int)(ip & 1);
-            if (!mbar_wait_bounded(carry_bar + 8 * b, (uint32_t)((ip >> 1) & 1), kCopySpinLimit)) {
+            const int st = (int)(ip % S), b = (int)(ip % kLbRing);
+            if (!mbar_wait_bounded(carry_bar + 8 * b, (uint32_t)((ip / kLbRing) & 1), kCopySpinLimit)) {
                 if (lane == 0) { record_error(p, kErrLookbackTimeout, first + ip * G); xc->abort = 1; }
                 aborted = true;
-            } else if (xc->abort) {
+            } else if (*(volatile int*)&xc->abort) {
                 aborted = true;
             }
             if (!aborted) {
@@ -883,18 +917,18 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                 const long long left = p.n - col0;
                 E carry;
                 carry.A = neg_inf(); carry.m = xc->carry[b].x; carry.s = xc->carry[b].y; carry.p = 0u;
-                const LanePark& lp = lpark[b];
+                const LanePark& lp = lpark[st];
                 E excl;
                 excl.A = lp.A[lane]; excl.m = lp.m[lane]; excl.s = lp.s[lane]; excl.p = SIGNED ? lp.p[lane] : 0u;
                 const E entering = compose(compose(carry, unpack_elem<SIGNED>(xc->wexcl[b][warp])), excl);
-                const uint8_t* sm_a = pipe.in_a(st);
-                const uint8_t* sm_b = pipe.in_b(st);
-                uint8_t* sm_out = park_buf(b);
-                const uint32_t pb = smem_u32(sm_out);
+                uint8_t* sm_a = st_a(st);
+                uint8_t* sm_b = st_b(st);
+                const uint32_t pb = smem_u32(st_park(st));
                 float out_mag[K];
                 uint32_t out_sign[MODE == kLogSigned ? K : 1];
                 bool ok = false;
-                if (!lp.slow) {
+                const bool was_slow = lp.slow != 0;
+                if (!was_slow) {
                     // rebuild A_t (and the parity of a) from the inputs, fetch the parked s_t, apply
                     float va[K];
                     uint32_t sa[MODE == kLogSigned ? K : 1];
@@ -919,28 +953,48 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                         sts128(pb + off.out[jx], Storage<TOut>::pack(out_mag + jx * Storage<TOut>::kPerUnit));
                     if (MODE == kLogSigned) CE::store_signs(p.sign_x, row * p.n + col0, left, p.sign_vec_ok != 0, out_sign);
                 } else {
+                    if (!was_slow && ST::IN_PLACE) {
+                        // the parked sums replaced the b-tensor chunk: fetch the lane's b values again
+#pragma unroll
+                        for (int t = 0; t < K; ++t) {
+                            const float v = (t < left) ? Storage<TIn>::load(p.in_b, row * p.n + col0 + t) : neutral_b<MODE>();
+                            Storage<TIn>::to_smem(sm_b, chunk_off(1, 0, (uint32_t)((lane * K + t) * sizeof(TIn))), v);
+                        }
+                        __syncwarp();
+                    }
                     const typename CE::SlowOut so =
                         CE::slow_apply(entering, sm_a, sm_b, lm, MODE == kLogSigned ? p.sign_a : nullptr,
                                        MODE == kLogSigned ? p.sign_b : nullptr, row * p.n + col0, left);
+                    __syncwarp();
 #pragma unroll
                     for (int jx = 0; jx < CE::OUT_UNITS; ++jx)
                         sts128(pb + off.out[jx], Storage<TOut>::pack(so.vals + jx * Storage<TOut>::kPerUnit));
                     if (MODE == kLogSigned) CE::store_signs(p.sign_x, row * p.n + col0, left, p.sign_vec_ok != 0, so.sgn);
                 }
                 if (TMA) {
+                    fence_async_smem();
+                    __syncwarp();
                     // a chunk wholly beyond the row end has nothing to store (a flat box is not clipped per row)
-                    if (colbase < p.n) pipe.store_from(&tm_o, row, colbase, pb);
+                    if (lane < out_boxes && colbase < p.n) {
+                        if (flat) tma_store_2d(&tm_o, 0, (int)((row * p.n + colbase) / OUT_PER_BOX), pb);
+                        else tma_store_2d(&tm_o, (int)colbase + lane * OUT_PER_BOX, (int)row, pb + (uint32_t)(lane * 128));
+                        bulk_commit();
+                    }
                 } else {
                     __syncwarp();
-                    CE::generic_store(p, sm_out, lm, lane, row, colbase);
+                    CE::generic_store(p, st_park(st), lm, lane, row, colbase);
                 }
-                __syncwarp();  // every lane is done with this tile's input stage
+                __syncwarp();  // every lane is done with this tile's stage
             }
         }
     }
     if (TMA) {
-        if (aborted) pipe.drain_loads(consumed, issued);
-        pipe.drain();
+        if (aborted) {
+            for (long long c = consumed; c < issued; ++c)
+                (void)mbar_wait_bounded(bars + 8 * (int)(c % S), (uint32_t)((c / S) & 1), kCopySpinLimit);
+        }
+        if (lane < out_boxes) bulk_wait_all();
+        __syncwarp();
     }
 }
 
