@@ -25,11 +25,12 @@ std::atomic<unsigned int> g_spin_limit{hs::kLookbackSpinLimit};
 std::atomic<long long> g_mute_tile{-1};
 thread_local char g_cuda_msg[256] = "";
 
-constexpr long long kMaxTmaDim = (1ll << 31) - (1ll << 20);  // TMA coordinates are int32
+constexpr long long kMaxN = (1ll << 31) - (1ll << 20);  // column indices and TMA coordinates are int32
+constexpr long long kMaxTmaDim = kMaxN;
 constexpr int kBatchedMinRowsPerSm = 8;  // fewer rows per SM than this: look-back kernel
 constexpr int kBatchedMinWarpsPerSm = 12; // rows per warp are chosen to keep at least this many warps per SM
 constexpr int kLookbackMinWarps = 8;     // fewest compute warps (= chunks per tile) of the look-back kernel
-constexpr int kLookbackWarps = 12;       // default compute warps of the look-back kernel
+constexpr int kLookbackWarps = 16;       // default compute warps of the look-back kernel
 constexpr int kMinChunk = 512;           // smallest chunk (32 lanes x 16 elements)
 
 unsigned long long next_call_id() {
@@ -252,7 +253,7 @@ hs_status validate_common(const void* a, const void* b, const void* x0, const vo
     if (rows == 0 || n == 0) return HS_OK;
     if (!a || !b || !x0 || !out) return HS_ERR_INVALID_ARG;
     if (rows > 0x7fffffffll) return HS_ERR_INVALID_ARG;
-    if (n > (1ll << 40) || rows > (1ll << 62) / n) return HS_ERR_INVALID_ARG;
+    if (n > kMaxN || rows > (1ll << 62) / n) return HS_ERR_INVALID_ARG;
     return HS_OK;
 }
 
@@ -311,8 +312,8 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         p.rows_per_warp = 1;
         // S input stages per compute warp (phase 2 of a tile runs S-2 iterations after its phase 1),
         // W compute warps (as many as shared memory allows, at most the default), NLB look-back warps
-        stages = env_int("HEINSEN_SCAN_LB_STAGES", 4, 3, kLbMaxStages);
-        const int nlb = env_int("HEINSEN_SCAN_LB_LOOKERS", 3, 1, 4);
+        stages = env_int("HEINSEN_SCAN_LB_STAGES", 3, 3, kLbMaxStages);
+        const int nlb = env_int("HEINSEN_SCAN_LB_LOOKERS", 2, 1, 4);
         int W = env_int("HEINSEN_SCAN_LB_WARPS", kLookbackWarps, kLookbackMinWarps, kLbMaxWarps);
         while (W > kLookbackMinWarps && ke.lb_smem(W, stages) + 1024 > dev.max_smem_optin) --W;
         lb_smem = ke.lb_smem(W, stages) + 1024;
@@ -422,7 +423,7 @@ hs_status heinsen_scan_log(const void* log_a, const void* log_b, const void* log
 
 size_t heinsen_scan_workspace_bytes(int64_t rows, int64_t n) {
     if (rows <= 0 || n <= 0) return 0;
-    if (rows > 0x7fffffffll || n > (1ll << 40) || rows > (1ll << 62) / n) return 0;
+    if (rows > 0x7fffffffll || n > kMaxN || rows > (1ll << 62) / n) return 0;
     return workspace_bytes_for(rows, n);
 }
 

@@ -228,11 +228,14 @@ struct Storage<float> {
     }
     __device__ static __forceinline__ float load(const void* p, int64_t i) { return ((const float*)p)[i]; }
     __device__ static __forceinline__ void store(void* p, int64_t i, float v) { ((float*)p)[i] = v; }
-    __device__ static __forceinline__ float from_smem(const uint8_t* base, uint32_t off) {
-        return *(const float*)(base + off);
+    // addr: 32-bit shared-memory address
+    __device__ static __forceinline__ float from_smem(uint32_t addr) {
+        float v;
+        asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+        return v;
     }
-    __device__ static __forceinline__ void to_smem(uint8_t* base, uint32_t off, float v) {
-        *(float*)(base + off) = v;
+    __device__ static __forceinline__ void to_smem(uint32_t addr, float v) {
+        asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
     }
 };
 template <>
@@ -257,11 +260,14 @@ struct Storage<__nv_bfloat16> {
     __device__ static __forceinline__ void store(void* p, int64_t i, float v) {
         ((__nv_bfloat16*)p)[i] = __float2bfloat16_rn(v);
     }
-    __device__ static __forceinline__ float from_smem(const uint8_t* base, uint32_t off) {
-        return __bfloat162float(*(const __nv_bfloat16*)(base + off));
+    __device__ static __forceinline__ float from_smem(uint32_t addr) {
+        unsigned short h;
+        asm volatile("ld.shared.u16 %0, [%1];" : "=h"(h) : "r"(addr));
+        return __uint_as_float((uint32_t)h << 16);
     }
-    __device__ static __forceinline__ void to_smem(uint8_t* base, uint32_t off, float v) {
-        *(__nv_bfloat16*)(base + off) = __float2bfloat16_rn(v);
+    __device__ static __forceinline__ void to_smem(uint32_t addr, float v) {
+        const __nv_bfloat16 b = __float2bfloat16_rn(v);
+        asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(*reinterpret_cast<const unsigned short*>(&b)) : "memory");
     }
 };
 
@@ -342,9 +348,8 @@ struct Run {
 
     // Load the lane's K inputs of both tensors from the swizzled chunk; `off` holds the lane's
     // IN_UNITS unit offsets (chunk_off), computed once per kernel.
-    __device__ __forceinline__ static void load(const uint8_t* sm_a, const uint8_t* sm_b, const uint32_t* off, float* va,
+    __device__ __forceinline__ static void load(uint32_t base_a, uint32_t base_b, const uint32_t* off, float* va,
                                                 float* vb) {
-        const uint32_t base_a = smem_u32(sm_a), base_b = smem_u32(sm_b);
 #pragma unroll
         for (int j = 0; j < IN_UNITS; ++j) {
             Storage<TIn>::unpack(lds128(base_a + off[j]), va + j * Storage<TIn>::kPerUnit);
@@ -352,8 +357,7 @@ struct Run {
         }
     }
 
-    __device__ __forceinline__ static void load_a(const uint8_t* sm_a, const uint32_t* off, float* va) {
-        const uint32_t base_a = smem_u32(sm_a);
+    __device__ __forceinline__ static void load_a(uint32_t base_a, const uint32_t* off, float* va) {
 #pragma unroll
         for (int j = 0; j < IN_UNITS; ++j) Storage<TIn>::unpack(lds128(base_a + off[j]), va + j * Storage<TIn>::kPerUnit);
     }

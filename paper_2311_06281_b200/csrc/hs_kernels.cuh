@@ -155,7 +155,7 @@ struct ChunkEngine {
 
     // Tracked form, pass 1: the lane's run as one part, every step with its own reference.
     // idx0/left as above (`left` <= 0: the run lies wholly beyond the row).
-    __device__ static __noinline__ E slow_pass1(const uint8_t* sm_a, const uint8_t* sm_b, LaneMap lm, const uint8_t* gsa,
+    __device__ static __noinline__ E slow_pass1(uint32_t sm_a, uint32_t sm_b, LaneMap lm, const uint8_t* gsa,
                                                 const uint8_t* gsb, long long idx0, long long left) {
         E e = identity_elem<SIGNED>();
         for (int t = 0; t < K; ++t) {
@@ -163,7 +163,7 @@ struct ChunkEngine {
                 const uint32_t off = chunk_off(lm.R, lm.g, (uint32_t)((lm.i * K + t) * sizeof(TIn)));
                 const uint32_t sa = gsa ? (((uint32_t)gsa[idx0 + t] & 1u) << 31) : 0u;
                 const uint32_t sb = gsb ? (((uint32_t)gsb[idx0 + t] & 1u) << 31) : 0u;
-                e = compose(e, Leaf<MODE, TIn>::get(Storage<TIn>::from_smem(sm_a, off), Storage<TIn>::from_smem(sm_b, off),
+                e = compose(e, Leaf<MODE, TIn>::get(Storage<TIn>::from_smem(sm_a + off), Storage<TIn>::from_smem(sm_b + off),
                                                     sa, sb));
             }
         }
@@ -174,7 +174,7 @@ struct ChunkEngine {
         uint32_t sgn[MODE == kLogSigned ? K : 1];
     };
     // Tracked form, pass 2: step the value through the lane's run; returns outputs (and signs).
-    __device__ static __noinline__ SlowOut slow_apply(E st, const uint8_t* sm_a, const uint8_t* sm_b, LaneMap lm,
+    __device__ static __noinline__ SlowOut slow_apply(E st, uint32_t sm_a, uint32_t sm_b, LaneMap lm,
                                                       const uint8_t* gsa, const uint8_t* gsb, long long idx0,
                                                       long long left) {
         SlowOut so;
@@ -185,7 +185,7 @@ struct ChunkEngine {
                 const uint32_t off = chunk_off(lm.R, lm.g, (uint32_t)((lm.i * K + t) * sizeof(TIn)));
                 const uint32_t sa = gsa ? (((uint32_t)gsa[idx0 + t] & 1u) << 31) : 0u;
                 const uint32_t sb = gsb ? (((uint32_t)gsb[idx0 + t] & 1u) << 31) : 0u;
-                st = compose(st, Leaf<MODE, TIn>::get(Storage<TIn>::from_smem(sm_a, off), Storage<TIn>::from_smem(sm_b, off),
+                st = compose(st, Leaf<MODE, TIn>::get(Storage<TIn>::from_smem(sm_a + off), Storage<TIn>::from_smem(sm_b + off),
                                                      sa, sb));
                 renormalise(st);
                 if (MODE == kLinear) {
@@ -210,14 +210,16 @@ struct ChunkEngine {
 
     // Phase 1: inputs from shared memory, the lane's run, the scan over the lanes of the row.
     // `row` is the lane's row (may be >= rows for a padded group), col0 its first column.
-    __device__ static __forceinline__ void phase1(const Params& p, const uint8_t* sm_a, const uint8_t* sm_b,
+    // `ragged` (warp-uniform): the chunk reaches beyond the row end or the warp's group beyond the
+    // last row, so some lanes must pad their run with neutral elements.
+    __device__ static __forceinline__ void phase1(const Params& p, uint32_t sm_a, uint32_t sm_b,
                                                   const Offsets& off, const LaneMap& lm, int lane, long long row,
-                                                  long long col0, Pending& pd, E& total) {
+                                                  long long col0, bool ragged, Pending& pd, E& total) {
         float va[K], vb[K];
         uint32_t sa[MODE == kLogSigned ? K : 1], sb[MODE == kLogSigned ? K : 1];
         R_::load(sm_a, sm_b, off.in, va, vb);
         const long long left = (row < p.rows) ? p.n - col0 : 0;
-        if (left < K) {
+        if (ragged) {
 #pragma unroll
             for (int t = 0; t < K; ++t) {
                 if (t >= left) { va[t] = neutral_a<MODE>(); vb[t] = neutral_b<MODE>(); }
@@ -237,12 +239,12 @@ struct ChunkEngine {
     }
 
     // Phase 2: `entering_row` is the value of x entering this row's piece of the chunk.
-    __device__ static __forceinline__ void phase2(const Params& p, const uint8_t* sm_a, const uint8_t* sm_b,
-                                                  uint8_t* sm_out, const Offsets& off, const LaneMap& lm, long long row,
+    __device__ static __forceinline__ void phase2(const Params& p, uint32_t sm_a, uint32_t sm_b,
+                                                  uint32_t sm_out, const Offsets& off, const LaneMap& lm, long long row,
                                                   long long col0, const Pending& pd, const E& entering_row) {
         const E entering = compose(entering_row, pd.excl);
         const long long left = (row < p.rows) ? p.n - col0 : 0;
-        const uint32_t ob = smem_u32(sm_out);
+        const uint32_t ob = sm_out;
         float out_mag[K];
         uint32_t out_sign[MODE == kLogSigned ? K : 1];
         bool ok = false;
@@ -263,37 +265,46 @@ struct ChunkEngine {
         }
     }
 
-    // Value of x_0 of a row as the element that starts the second scan (Eq. 7's cat(log x_0, .)).
-    __device__ static __forceinline__ E row_start(const Params& p, long long row) {
-        if (row >= p.rows) return state_elem<SIGNED>(neg_inf(), 0u);
-        const float v = Storage<TIn>::load(p.x0, row);
-        if (MODE == kLinear) return state_elem<SIGNED>(log_abs_accurate(v), __float_as_uint(v) & kSignBit);
-        uint32_t sg = 0u;
-        if (MODE == kLogSigned && p.sign_x0) sg = ((uint32_t)p.sign_x0[row] & 1u) << 31;
-        return state_elem<SIGNED>(v, sg);
+    // x_0 of a row as stored (value, sign mask); rows beyond the last one are empty (x_0 = 0).
+    struct RawX0 { float v; uint32_t sg; };
+    __device__ static __forceinline__ RawX0 load_x0(const Params& p, long long row) {
+        RawX0 r;
+        r.v = MODE == kLinear ? 0.0f : neg_inf();
+        r.sg = 0u;
+        if (row < p.rows) {
+            r.v = Storage<TIn>::load(p.x0, row);
+            if (MODE == kLogSigned && p.sign_x0) r.sg = ((uint32_t)p.sign_x0[row] & 1u) << 31;
+        }
+        return r;
     }
+    // ... and as the element that starts the second scan (Eq. 7's cat(log x_0, .)).
+    __device__ static __forceinline__ E x0_elem(const RawX0& r) {
+        if (MODE == kLinear) return state_elem<SIGNED>(log_abs_accurate(r.v), __float_as_uint(r.v) & kSignBit);
+        return state_elem<SIGNED>(r.v, r.sg);
+    }
+    __device__ static __forceinline__ E row_start(const Params& p, long long row) { return x0_elem(load_x0(p, row)); }
 
     // Plain-load staging for rows that TMA cannot address (unaligned base or row pitch).
     // row0: first row of the warp's group, colbase: first column of the chunk.
-    __device__ static __forceinline__ void generic_load(const Params& p, uint8_t* sm_a, uint8_t* sm_b, const LaneMap& lm,
+    __device__ static __forceinline__ void generic_load(const Params& p, uint32_t sm_a, uint32_t sm_b, const LaneMap& lm,
                                                         int lane, long long row0, long long colbase) {
         for (int e = lane; e < 32 * K; e += 32) {
             const int rg = e / lm.W, c = e - rg * lm.W;
             const long long row = row0 + rg, col = colbase + c;
             const bool in = row < p.rows && col < p.n;
             const uint32_t off = chunk_off(lm.R, rg, (uint32_t)(c * sizeof(TIn)));
-            Storage<TIn>::to_smem(sm_a, off, in ? Storage<TIn>::load(p.in_a, row * p.n + col) : neutral_a<MODE>());
-            Storage<TIn>::to_smem(sm_b, off, in ? Storage<TIn>::load(p.in_b, row * p.n + col) : neutral_b<MODE>());
+            Storage<TIn>::to_smem(sm_a + off, in ? Storage<TIn>::load(p.in_a, row * p.n + col) : neutral_a<MODE>());
+            Storage<TIn>::to_smem(sm_b + off, in ? Storage<TIn>::load(p.in_b, row * p.n + col) : neutral_b<MODE>());
         }
     }
-    __device__ static __forceinline__ void generic_store(const Params& p, const uint8_t* sm_out, const LaneMap& lm, int lane,
+    __device__ static __forceinline__ void generic_store(const Params& p, uint32_t sm_out, const LaneMap& lm, int lane,
                                                          long long row0, long long colbase) {
         for (int e = lane; e < 32 * K; e += 32) {
             const int rg = e / lm.W, c = e - rg * lm.W;
             const long long row = row0 + rg, col = colbase + c;
             if (row < p.rows && col < p.n) {
                 const uint32_t off = chunk_off(lm.R, rg, (uint32_t)(c * sizeof(TOut)));
-                Storage<TOut>::store(p.out, row * p.n + col, Storage<TOut>::from_smem(sm_out, off));
+                Storage<TOut>::store(p.out, row * p.n + col, Storage<TOut>::from_smem(sm_out + off));
             }
         }
     }
@@ -317,7 +328,7 @@ struct WarpPipe {
     static constexpr int OUT_BYTES = 32 * K * (int)sizeof(TOut);
     static constexpr int IN_PER_BOX = 128 / (int)sizeof(TIn);    // elements of a row in one box
     static constexpr int OUT_PER_BOX = 128 / (int)sizeof(TOut);
-    uint8_t* base;   // this warp's shared memory
+    uint32_t base;   // this warp's shared memory (32-bit shared address)
     uint32_t bars;   // shared address of this warp's mbarriers
     int stages;
     int lane;
@@ -325,18 +336,16 @@ struct WarpPipe {
     int in_boxes;    // boxes per tensor per chunk, input / output
     int out_boxes;
     bool flat;       // one box per chunk, addressed by line number (see Params::flat_boxes)
-    long long n;     // row length, for line numbers
 
-    __device__ __forceinline__ void setup(int rows_per_warp, bool flat_boxes = false, long long row_len = 0) {
+    __device__ __forceinline__ void setup(int rows_per_warp, bool flat_boxes = false) {
         R = rows_per_warp;
         flat = flat_boxes;
-        n = row_len;
         in_boxes = flat ? 1 : IN_BYTES / (128 * R);
         out_boxes = flat ? 1 : OUT_BYTES / (128 * R);
     }
-    __device__ __forceinline__ uint8_t* in_a(int s) const { return base + s * 2 * IN_BYTES; }
-    __device__ __forceinline__ uint8_t* in_b(int s) const { return base + s * 2 * IN_BYTES + IN_BYTES; }
-    __device__ __forceinline__ uint8_t* out(int o) const { return base + stages * 2 * IN_BYTES + o * OUT_BYTES; }
+    __device__ __forceinline__ uint32_t in_a(int s) const { return base + s * 2 * IN_BYTES; }
+    __device__ __forceinline__ uint32_t in_b(int s) const { return base + s * 2 * IN_BYTES + IN_BYTES; }
+    __device__ __forceinline__ uint32_t out(int o) const { return base + stages * 2 * IN_BYTES + o * OUT_BYTES; }
 
     __device__ __forceinline__ void init() {
         if (lane == 0) {
@@ -345,23 +354,23 @@ struct WarpPipe {
         }
         __syncwarp();
     }
-    // row0: first row of the group; colbase: first column of the chunk
-    __device__ __forceinline__ void issue(const CUtensorMap* tm_a, const CUtensorMap* tm_b, long long row0, long long colbase,
+    // colbase: first column of the chunk, row0: first row of the group; `line` (flat boxes only):
+    // index of the chunk's first 128-byte line in the flat view
+    __device__ __forceinline__ void issue(const CUtensorMap* tm_a, const CUtensorMap* tm_b, int row0, int colbase, int line,
                                           int s) {
         const uint32_t bar = bars + 8 * s;
         if (lane == 0) mbar_expect_tx(bar, 2 * IN_BYTES);
         __syncwarp();
         if (flat) {
             if (lane == 0) {
-                const int line = (int)((row0 * n + colbase) / IN_PER_BOX);
-                tma_load_2d(smem_u32(in_a(s)), tm_a, 0, line, bar);
-                tma_load_2d(smem_u32(in_b(s)), tm_b, 0, line, bar);
+                tma_load_2d(in_a(s), tm_a, 0, line, bar);
+                tma_load_2d(in_b(s), tm_b, 0, line, bar);
             }
         } else if (lane < in_boxes) {
-            const int x = (int)colbase + lane * IN_PER_BOX;
+            const int x = colbase + lane * IN_PER_BOX;
             const uint32_t dst = (uint32_t)(lane * R * 128);
-            tma_load_2d(smem_u32(in_a(s)) + dst, tm_a, x, (int)row0, bar);
-            tma_load_2d(smem_u32(in_b(s)) + dst, tm_b, x, (int)row0, bar);
+            tma_load_2d(in_a(s) + dst, tm_a, x, row0, bar);
+            tma_load_2d(in_b(s) + dst, tm_b, x, row0, bar);
         }
     }
     __device__ __forceinline__ bool wait(int s, uint32_t parity) const {
@@ -372,22 +381,19 @@ struct WarpPipe {
         if (lane < out_boxes) bulk_wait_read<1>();
         __syncwarp();
     }
-    // store the chunk held in shared memory at `src`
-    __device__ __forceinline__ void store_from(const CUtensorMap* tm_o, long long row0, long long colbase, uint32_t src) const {
+    // store the chunk held in shared memory at `src`; `line`: as for issue(), in output lines
+    __device__ __forceinline__ void store_from(const CUtensorMap* tm_o, int row0, int colbase, int line, uint32_t src) const {
         fence_async_smem();
         __syncwarp();
         if (lane < out_boxes) {
             if (flat) {
-                tma_store_2d(tm_o, 0, (int)((row0 * n + colbase) / OUT_PER_BOX), src);
+                tma_store_2d(tm_o, 0, line, src);
             } else {
-                const int x = (int)colbase + lane * OUT_PER_BOX;
-                tma_store_2d(tm_o, x, (int)row0, src + (uint32_t)(lane * R * 128));
+                const int x = colbase + lane * OUT_PER_BOX;
+                tma_store_2d(tm_o, x, row0, src + (uint32_t)(lane * R * 128));
             }
             bulk_commit();
         }
-    }
-    __device__ __forceinline__ void store(const CUtensorMap* tm_o, long long row0, long long colbase, int o) const {
-        store_from(tm_o, row0, colbase, smem_u32(out(o)));
     }
     __device__ __forceinline__ void drain() const {
         if (lane < out_boxes) bulk_wait_all();
@@ -398,6 +404,8 @@ struct WarpPipe {
     __device__ __forceinline__ void drain_loads(long long consumed, long long issued) const {
         for (long long c = consumed; c < issued; ++c) (void)wait((int)(c % stages), (uint32_t)((c / stages) & 1));
     }
+    static constexpr int IN_LINES = IN_BYTES / 128;    // 128-byte lines of one tensor's chunk
+    static constexpr int OUT_LINES = OUT_BYTES / 128;
 };
 
 // ------------------------------------------------------------------------------------------
@@ -424,83 +432,101 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
     lm.W = (32 / R) * K;
     const typename CE::Offsets off = CE::offsets(lm);
 
-    WarpPipe<TIn, TOut, K> pipe;
-    pipe.base = smem + warp * per_warp;
+    using Pipe = WarpPipe<TIn, TOut, K>;
+    Pipe pipe;
+    pipe.base = smem_u32(smem) + warp * per_warp;
     pipe.bars = smem_u32(smem + nwarps * per_warp) + warp * (8 * kMaxStages);
     pipe.stages = S;
     pipe.lane = lane;
-    pipe.setup(R, p.flat_boxes != 0, p.n);
+    pipe.setup(R, p.flat_boxes != 0);
     if (TMA) pipe.init();
 
     if (blockIdx.x == 0 && threadIdx.x == 0) p.ws->started_id = p.call_id;
 
-    const long long gw = (long long)blockIdx.x * nwarps + warp;
-    const long long GW = (long long)gridDim.x * nwarps;
-    const long long groups = (p.rows + R - 1) / R;
+    // All hot-loop indices are 32-bit and advance incrementally (rows < 2^31; with TMA also n < 2^31);
+    // 64-bit products appear once per row only.
+    const int gw = blockIdx.x * nwarps + warp;
+    const int GW = gridDim.x * nwarps;
+    const int groups = (int)((p.rows + R - 1) / R);
     if (gw >= groups) return;
-    const long long my_groups = (groups - gw + GW - 1) / GW;
-    const long long items = my_groups * p.nchunks;
+    const int my_groups = (groups - gw + GW - 1) / GW;
+    const long long items = (long long)my_groups * p.nchunks;
+    const int nchunks = p.nchunks;
+    const bool tail_ragged = (p.n % lm.W) != 0;  // the last chunk of a row is partial
+    auto first_line = [&](int grp, int per_box) { return (int)(((long long)grp * R * p.n) / per_box); };
 
-    // producer cursor
-    long long pgroup = gw;
-    int pchunk = 0;
+    // producer cursor (TMA loads run S-1 chunks ahead)
+    int pgroup = gw, pchunk = 0, pstage = 0;
+    int pline = pipe.flat ? first_line(pgroup, Pipe::IN_PER_BOX) : 0;
     long long issued = 0;
-    if (TMA) {
-        for (; issued < S - 1 && issued < items; ++issued) {
-            pipe.issue(&tm_a, &tm_b, pgroup * R, (long long)pchunk * lm.W, (int)(issued % S));
-            if (++pchunk == p.nchunks) { pchunk = 0; pgroup += GW; }
+    auto issue_next = [&]() {
+        pipe.issue(&tm_a, &tm_b, pgroup * R, pchunk * lm.W, pline, pstage);
+        ++issued;
+        pline += Pipe::IN_LINES;
+        if (++pstage == S) pstage = 0;
+        if (++pchunk == nchunks) {
+            pchunk = 0;
+            pgroup += GW;
+            if (pipe.flat && pgroup < groups) pline = first_line(pgroup, Pipe::IN_PER_BOX);
         }
+    };
+    if (TMA) {
+        for (int s = 0; s < S - 1 && issued < items; ++s) issue_next();
     }
 
-    long long group = gw;
-    int chunk = 0;
-    long long row = group * R + lm.g;
+    int group = gw, chunk = 0, colbase = 0;
+    int oline = pipe.flat ? first_line(group, Pipe::OUT_PER_BOX) : 0;
+    long long row = (long long)group * R + lm.g;
+    bool group_ragged = (group + 1) * (long long)R > p.rows;
     E state = CE::row_start(p, row);
+    typename CE::RawX0 x0_next = CE::load_x0(p, row + (long long)GW * R);  // in flight during this row
     int stage = 0;
     uint32_t parity = 0;
     for (long long q = 0; q < items; ++q) {
-        const long long colbase = (long long)chunk * lm.W;
         if (TMA) {
-            if (issued < items) {
-                pipe.issue(&tm_a, &tm_b, pgroup * R, (long long)pchunk * lm.W, (int)(issued % S));
-                ++issued;
-                if (++pchunk == p.nchunks) { pchunk = 0; pgroup += GW; }
-            }
+            if (issued < items) issue_next();
             if (!pipe.wait(stage, parity)) {
                 if (lane == 0) record_error(p, kErrCopyTimeout, row);
                 pipe.drain_loads(q + 1, issued);
                 break;
             }
         } else {
-            CE::generic_load(p, pipe.in_a(0), pipe.in_b(0), lm, lane, group * R, colbase);
+            CE::generic_load(p, pipe.in_a(0), pipe.in_b(0), lm, lane, (long long)group * R, colbase);
             __syncwarp();
         }
-        const uint8_t* sm_a = pipe.in_a(stage);
-        const uint8_t* sm_b = pipe.in_b(stage);
-        uint8_t* sm_out = pipe.out((int)(q & 1));
-        const long long col0 = colbase + lm.i * K;
+        const uint32_t sm_a = pipe.in_a(stage);
+        const uint32_t sm_b = pipe.in_b(stage);
+        const uint32_t sm_out = pipe.out((int)(q & 1));
+        const int col0 = colbase + lm.i * K;
+        const bool ragged = group_ragged || (tail_ragged && chunk == nchunks - 1);
 
         typename CE::Pending pd;
         E total;
-        CE::phase1(p, sm_a, sm_b, off, lm, lane, row, col0, pd, total);
+        CE::phase1(p, sm_a, sm_b, off, lm, lane, row, col0, ragged, pd, total);
         if (TMA) pipe.acquire_out();
         CE::phase2(p, sm_a, sm_b, sm_out, off, lm, row, col0, pd, state);
         state = compose(state, total);
         renormalise(state);
 
         if (TMA) {
-            pipe.store(&tm_o, group * R, colbase, (int)(q & 1));
+            pipe.store_from(&tm_o, group * R, colbase, oline, sm_out);
         } else {
             __syncwarp();
-            CE::generic_store(p, sm_out, lm, lane, group * R, colbase);
+            CE::generic_store(p, sm_out, lm, lane, (long long)group * R, colbase);
         }
         __syncwarp();  // every lane is done with this input stage
 
-        if (++chunk == p.nchunks) {
+        colbase += lm.W;
+        oline += Pipe::OUT_LINES;
+        if (++chunk == nchunks) {
             chunk = 0;
+            colbase = 0;
             group += GW;
-            row = group * R + lm.g;
-            if (group < groups) state = CE::row_start(p, row);
+            row = (long long)group * R + lm.g;
+            group_ragged = (group + 1) * (long long)R > p.rows;
+            state = CE::x0_elem(x0_next);
+            x0_next = CE::load_x0(p, row + (long long)GW * R);
+            if (pipe.flat && group < groups) oline = first_line(group, Pipe::OUT_PER_BOX);
         }
         if (++stage == S) { stage = 0; parity ^= 1u; }
     }
@@ -715,6 +741,24 @@ __host__ __device__ constexpr int lb_total_smem_bytes(int W, int S) {
     return W * S * (LbStage<TIn, K>::BYTES + (int)sizeof(LanePark)) + (int)sizeof(Exchange) + W * kLbMaxStages * 8;
 }
 
+// Position of a CTA's tile sequence: tile T = tile j of row `row`; advances by a fixed stride
+// without divisions (the stride is split once into whole rows and a remainder).
+struct TileCursor {
+    long long T;
+    int row, j;
+    __device__ __forceinline__ void init(long long t, int tiles_per_row) {
+        T = t;
+        row = (int)(t / tiles_per_row);
+        j = (int)(t - (long long)row * tiles_per_row);
+    }
+    __device__ __forceinline__ void advance(int stride, int stride_rows, int stride_rem, int tiles_per_row) {
+        T += stride;
+        row += stride_rows;
+        j += stride_rem;
+        if (j >= tiles_per_row) { j -= tiles_per_row; ++row; }
+    }
+};
+
 template <int MODE, typename TIn, typename TOut, int K, bool TMA>
 __global__ void __launch_bounds__(640, 1)
 lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
@@ -761,10 +805,14 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
         // ------------------------------------------------------------------ look-back warps
         // Warp u of NLB takes the CTA's tiles u, u+NLB, u+2*NLB, ...: a tile's look-back lasts
         // several L2 round trips, longer than a tile's arithmetic, so several are in flight.
-        for (long long i = warp - W; i < my_tiles; i += NLB) {
-            const long long T = first + i * G;
-            const long long row = T / tpr;
-            const int j = (int)(T - row * tpr);
+        TileCursor cur;
+        cur.init(first + (long long)(warp - W) * G, tpr);
+        const int lb_stride = NLB * (int)G;
+        const int lb_rows = lb_stride / tpr, lb_rem = lb_stride % tpr;
+        for (long long i = warp - W; i < my_tiles; i += NLB, cur.advance(lb_stride, lb_rows, lb_rem, tpr)) {
+            const long long T = cur.T;
+            const long long row = cur.row;
+            const int j = cur.j;
             const int b = (int)(i % kLbRing);
             bool failed = !mbar_wait_bounded(agg_bar + 8 * b, (uint32_t)((i / kLbRing) & 1), kCopySpinLimit);
             if (*(volatile int*)&xc->abort) failed = true;
@@ -810,7 +858,7 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
 #pragma unroll
     for (int jx = 0; jx < K / 4; ++jx) park_off[jx] = chunk_off(1, 0, (uint32_t)((lane * (K / 4) + jx) * 16));
 
-    uint8_t* wb = smem + (size_t)warp * S * ST::BYTES;
+    const uint32_t wb = smem_u32(smem) + (uint32_t)(warp * S * ST::BYTES);
     auto st_a = [&](int st) { return wb + st * ST::BYTES; };
     auto st_b = [&](int st) { return wb + st * ST::BYTES + ST::IN_BYTES; };
     auto st_park = [&](int st) { return wb + st * ST::BYTES + ST::PARK_OFF; };
@@ -823,53 +871,58 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
     const int in_boxes = flat ? 1 : ST::IN_BYTES / 128;
     const int out_boxes = flat ? 1 : (CHUNK * (int)sizeof(TOut)) / 128;
 
-    auto tile_coords = [&](long long i, long long& row, long long& colbase) {
-        const long long T = first + i * G;
-        row = T / tpr;
-        const int j = (int)(T - row * tpr);
-        colbase = ((long long)j * W + warp) * CHUNK;
-    };
+    const int g_rows = (int)G / tpr, g_rem = (int)G % tpr;
+    TileCursor ci, c1, c2;  // tiles being loaded, in phase 1, in phase 2
+    ci.init(first, tpr);
+    c1 = ci;
+    c2 = ci;
+    auto colbase_of = [&](const TileCursor& c) { return (c.j * W + warp) * CHUNK; };
     long long issued = 0;
+    int istage = 0;
     auto issue_next = [&]() {
         if (issued < my_tiles) {
-            long long r, cb;
-            tile_coords(issued, r, cb);
-            const int st = (int)(issued % S);
-            const uint32_t bar = bars + 8 * st;
+            const int cb = colbase_of(ci);
+            const uint32_t bar = bars + 8 * istage;
             if (lane == 0) mbar_expect_tx(bar, 2 * ST::IN_BYTES);
             __syncwarp();
             if (flat) {
                 if (lane == 0) {
-                    const int line = (int)((r * p.n + cb) / IN_PER_BOX);
-                    tma_load_2d(smem_u32(st_a(st)), &tm_a, 0, line, bar);
-                    tma_load_2d(smem_u32(st_b(st)), &tm_b, 0, line, bar);
+                    const int line = (int)(((long long)ci.row * p.n + cb) / IN_PER_BOX);
+                    tma_load_2d(st_a(istage), &tm_a, 0, line, bar);
+                    tma_load_2d(st_b(istage), &tm_b, 0, line, bar);
                 }
             } else if (lane < in_boxes) {
-                const int x = (int)cb + lane * IN_PER_BOX;
-                tma_load_2d(smem_u32(st_a(st)) + lane * 128, &tm_a, x, (int)r, bar);
-                tma_load_2d(smem_u32(st_b(st)) + lane * 128, &tm_b, x, (int)r, bar);
+                const int x = cb + lane * IN_PER_BOX;
+                tma_load_2d(st_a(istage) + lane * 128, &tm_a, x, ci.row, bar);
+                tma_load_2d(st_b(istage) + lane * 128, &tm_b, x, ci.row, bar);
             }
             ++issued;
+            if (++istage == S) istage = 0;
+            ci.advance((int)G, g_rows, g_rem, tpr);
         }
     };
     if (TMA) issue_next();
 
     bool aborted = false;
     long long consumed = 0;
+    int st1 = 0, st2 = 0;          // stages of the tiles in phase 1 / phase 2
+    uint32_t par1 = 0;             // parity of stage st1's mbarrier
+    int b1 = 0, b2 = 0;            // ring slots of those tiles
+    uint32_t parb2 = 0;            // parity of ring slot b2's carry mbarrier
     for (long long i = 0; i < my_tiles + D && !aborted; ++i) {
         // ---- phase 1 of tile i
         if (i < my_tiles) {
-            long long row, colbase;
-            tile_coords(i, row, colbase);
-            const int st = (int)(i % S), b = (int)(i % kLbRing);
+            const long long row = c1.row;
+            const int colbase = colbase_of(c1);
+            const int st = st1, b = b1;
             if (TMA) {
                 // tile i+1 goes into the stage whose tile finished phase 2 in the previous iteration;
                 // the store issued from it then has been read by now
                 if (lane < out_boxes) bulk_wait_read<0>();
                 __syncwarp();
                 issue_next();
-                if (!mbar_wait_bounded(bars + 8 * st, (uint32_t)((i / S) & 1), kCopySpinLimit)) {
-                    if (lane == 0) { record_error(p, kErrCopyTimeout, first + i * G); xc->abort = 1; }
+                if (!mbar_wait_bounded(bars + 8 * st, par1, kCopySpinLimit)) {
+                    if (lane == 0) { record_error(p, kErrCopyTimeout, c1.T); xc->abort = 1; }
                     aborted = true;
                 } else {
                     ++consumed;
@@ -882,10 +935,10 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                 const long long col0 = colbase + lane * K;
                 typename CE::Pending pd;
                 E total;
-                CE::phase1(p, st_a(st), st_b(st), off, lm, lane, row, col0, pd, total);
+                CE::phase1(p, st_a(st), st_b(st), off, lm, lane, row, col0, colbase + CHUNK > p.n, pd, total);
                 LanePark& lp = lpark[st];
                 if (!pd.slow) {  // park the partial sums (a slow chunk keeps its inputs instead)
-                    const uint32_t pb = smem_u32(st_park(st));
+                    const uint32_t pb = st_park(st);
 #pragma unroll
                     for (int jx = 0; jx < K / 4; ++jx) sts128(pb + park_off[jx], Storage<float>::pack(pd.run.s + 4 * jx));
                 }
@@ -899,15 +952,17 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                 __syncwarp();
                 if (lane == 0) mbar_arrive(agg_bar + 8 * b);
             }
+            c1.advance((int)G, g_rows, g_rem, tpr);
+            if (++st1 == S) { st1 = 0; par1 ^= 1u; }
+            if (++b1 == kLbRing) b1 = 0;
         }
         // ---- phase 2 of tile i-D
         if (i >= D && !aborted) {
-            const long long ip = i - D;
-            long long row, colbase;
-            tile_coords(ip, row, colbase);
-            const int st = (int)(ip % S), b = (int)(ip % kLbRing);
-            if (!mbar_wait_bounded(carry_bar + 8 * b, (uint32_t)((ip / kLbRing) & 1), kCopySpinLimit)) {
-                if (lane == 0) { record_error(p, kErrLookbackTimeout, first + ip * G); xc->abort = 1; }
+            const long long row = c2.row;
+            const int colbase = colbase_of(c2);
+            const int st = st2, b = b2;
+            if (!mbar_wait_bounded(carry_bar + 8 * b, parb2, kCopySpinLimit)) {
+                if (lane == 0) { record_error(p, kErrLookbackTimeout, c2.T); xc->abort = 1; }
                 aborted = true;
             } else if (*(volatile int*)&xc->abort) {
                 aborted = true;
@@ -921,9 +976,9 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                 E excl;
                 excl.A = lp.A[lane]; excl.m = lp.m[lane]; excl.s = lp.s[lane]; excl.p = SIGNED ? lp.p[lane] : 0u;
                 const E entering = compose(compose(carry, unpack_elem<SIGNED>(xc->wexcl[b][warp])), excl);
-                uint8_t* sm_a = st_a(st);
-                uint8_t* sm_b = st_b(st);
-                const uint32_t pb = smem_u32(st_park(st));
+                uint32_t sm_a = st_a(st);
+                uint32_t sm_b = st_b(st);
+                const uint32_t pb = st_park(st);
                 float out_mag[K];
                 uint32_t out_sign[MODE == kLogSigned ? K : 1];
                 bool ok = false;
@@ -933,7 +988,7 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                     float va[K];
                     uint32_t sa[MODE == kLogSigned ? K : 1];
                     R_::load_a(sm_a, off.in, va);
-                    if (left < K) {
+                    if (colbase + CHUNK > p.n) {
 #pragma unroll
                         for (int t = 0; t < K; ++t)
                             if (t >= left) va[t] = neutral_a<MODE>();
@@ -958,7 +1013,7 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
 #pragma unroll
                         for (int t = 0; t < K; ++t) {
                             const float v = (t < left) ? Storage<TIn>::load(p.in_b, row * p.n + col0 + t) : neutral_b<MODE>();
-                            Storage<TIn>::to_smem(sm_b, chunk_off(1, 0, (uint32_t)((lane * K + t) * sizeof(TIn))), v);
+                            Storage<TIn>::to_smem(sm_b + chunk_off(1, 0, (uint32_t)((lane * K + t) * sizeof(TIn))), v);
                         }
                         __syncwarp();
                     }
@@ -986,6 +1041,9 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                 }
                 __syncwarp();  // every lane is done with this tile's stage
             }
+            c2.advance((int)G, g_rows, g_rem, tpr);
+            if (++st2 == S) st2 = 0;
+            if (++b2 == kLbRing) { b2 = 0; parb2 ^= 1u; }
         }
     }
     if (TMA) {
