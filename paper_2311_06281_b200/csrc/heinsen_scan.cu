@@ -30,7 +30,7 @@ constexpr long long kMaxTmaDim = kMaxN;
 constexpr int kBatchedMinRowsPerSm = 8;  // fewer rows per SM than this: look-back kernel
 constexpr int kBatchedMinWarpsPerSm = 12; // rows per warp are chosen to keep at least this many warps per SM
 constexpr int kLookbackMinWarps = 8;     // fewest compute warps (= chunks per tile) of the look-back kernel
-constexpr int kLookbackWarps = 16;       // default compute warps of the look-back kernel
+constexpr int kLookbackWarps = 12;       // default compute warps of the look-back kernel
 constexpr int kMinChunk = 512;           // smallest chunk (32 lanes x 16 elements)
 
 unsigned long long next_call_id() {
@@ -199,7 +199,7 @@ int choose_path(long long rows, const DeviceInfo& d) {
 size_t workspace_bytes_for(long long rows, long long n) {
     // sized for the smallest chunk so that it covers every type
     const long long tpr = lookback_tiles_per_row(n, kMinChunk, kLookbackMinWarps);
-    const long long gpr = (tpr + kLbGroup - 1) / kLbGroup;
+    const long long gpr = (tpr + 1) / 2;  // groups hold at least 2 tiles
     return sizeof(Header) + (size_t)(rows * (tpr + gpr)) * 16;
 }
 
@@ -312,7 +312,7 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         p.rows_per_warp = 1;
         // S input stages per compute warp (phase 2 of a tile runs S-2 iterations after its phase 1),
         // W compute warps (as many as shared memory allows, at most the default), NLB look-back warps
-        stages = env_int("HEINSEN_SCAN_LB_STAGES", 3, 3, kLbMaxStages);
+        stages = env_int("HEINSEN_SCAN_LB_STAGES", 4, 3, kLbMaxStages);
         const int nlb = env_int("HEINSEN_SCAN_LB_LOOKERS", 2, 1, 4);
         int W = env_int("HEINSEN_SCAN_LB_WARPS", kLookbackWarps, kLookbackMinWarps, kLbMaxWarps);
         while (W > kLookbackMinWarps && ke.lb_smem(W, stages) + 1024 > dev.max_smem_optin) --W;
@@ -321,7 +321,10 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         warps = W + nlb;
         p.tiles_per_row = (int)lookback_tiles_per_row(p.n, chunk, W);
         p.num_tiles = p.rows * p.tiles_per_row;
-        p.groups_per_row = (p.tiles_per_row + kLbGroup - 1) / kLbGroup;
+        // group = the tiles one wave of CTAs processes (the grid is sm_count CTAs: one per SM)
+        p.lb_group = dev.sm_count < kLbMaxGroup ? dev.sm_count : kLbMaxGroup;
+        p.lb_group = env_int("HEINSEN_SCAN_LB_GROUP", p.lb_group, 2, kLbMaxGroup);
+        p.groups_per_row = (p.tiles_per_row + p.lb_group - 1) / p.lb_group;
         const size_t need = sizeof(Header) + ((size_t)p.num_tiles + (size_t)p.rows * p.groups_per_row) * 16;
         if (workspace_bytes < need) return HS_ERR_WORKSPACE_TOO_SMALL;
         p.desc = reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(workspace) + sizeof(Header));

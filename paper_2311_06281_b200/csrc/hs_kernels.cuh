@@ -58,7 +58,8 @@ struct Params {
     long long num_tiles;
     uint4* desc;                // [num_tiles] tile descriptors, zeroed before the launch
     uint4* gdesc;               // [rows * groups_per_row] group descriptors, zeroed before the launch
-    int groups_per_row;         // ceil(tiles_per_row / 32)
+    int groups_per_row;         // ceil(tiles_per_row / lb_group)
+    int lb_group;               // tiles per group: the CTAs of the launch, at most kLbMaxGroup
     int lb_warps;               // look-back warps per CTA
     unsigned int spin_limit;    // bound on polls of predecessor flags
     long long mute_tile;        // test hook: this tile never publishes (-1: none)
@@ -572,17 +573,20 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
-constexpr int kLbGroup = 32;                        // tiles per group (one per lane)
+constexpr int kLbPerLane = 5;                       // tile descriptors polled by each lane per round
+constexpr int kLbMaxGroup = 32 * kLbPerLane;        // tiles per group, at most
 constexpr int kLbMaxWarps = 16;                     // compute warps per CTA, at most
 
-// Two levels of descriptors keep a look-back short however many tiles are in flight:
+// Two levels of descriptors keep a look-back to one round trip however long the row is:
 //   tile level  : desc[T]   = aggregate of tile T (state 1), written right after its phase 1;
-//   group level : gdesc[g]  = aggregate of the 32 tiles of group g (state 1), written by the
-//                 look-back of the group's last tile as soon as it has seen the other 31, and
+//   group level : gdesc[g]  = aggregate of the tiles of group g (state 1), written by the
+//                 look-back of the group's last tile as soon as it has seen the others, and
 //                 later replaced by the value of x after the group (state 2).
-// The value entering tile j = (value before its group, from group descriptors: aggregates back
-// to the nearest known value) composed with (the aggregates of the tiles of its own group before
-// it).  One round reads at most 31 + 32 descriptors, one or two per lane, all in flight at once.
+// A group is p.lb_group consecutive tiles of a row -- the tiles that the resident CTAs process at
+// the same time -- so the group descriptors a tile needs are those of earlier waves, already
+// visible when it looks.  The value entering tile j = (value before its group: group aggregates
+// back to the nearest known value) composed with (the aggregates of the tiles of its own group
+// before it).  Both levels are polled together, every load of a round in flight at once.
 template <int MODE, typename TIn, typename TOut, int K>
 struct Lookback {
     using CE = ChunkEngine<MODE, TIn, TOut, K>;
@@ -627,56 +631,82 @@ struct Lookback {
     // Warp-collective.  Tile T is tile j of `row`; tile_total its aggregate.  Returns the value of
     // x entering the tile and publishes the group descriptors this tile is responsible for.
     __device__ static __forceinline__ E run(const Params& p, long long T, int j, long long row, int lane,
-                                            const E& tile_total, bool publish, bool& failed, unsigned int& total_polls) {
+                                            const E& tile_total, bool publish, bool& failed, unsigned int& total_polls,
+                                            unsigned long long* stamps = nullptr) {
         failed = false;
-        const int g = j / kLbGroup, k = j - g * kLbGroup;          // group, position in group
+        const int gsz = p.lb_group;
+        const int g = j / gsz, k = j - g * gsz;                    // group, position in group
         const long long gbase = row * p.groups_per_row;            // first group descriptor of the row
-        const bool closes_group = (k == kLbGroup - 1) || (j == p.tiles_per_row - 1);
+        const bool closes_group = (k == gsz - 1) || (j == p.tiles_per_row - 1);
+        const bool full_group = (k == gsz - 1);
         unsigned int polls = 0;
-
-        // ---- tiles of the own group before this one: lane l looks at tile j-1-l (l < k)
-        E part = identity_elem<SIGNED>();
-        if (k > 0) {
-            Desc d;
-            d.lo = 0ull; d.hi = 0ull;
-            while (true) {
-                if (lane < k) d = ld_desc(p.desc + (T - 1 - lane));
-                const bool ready = (lane >= k) || state_of(d) == kAgg;
-                ++total_polls;
-                if (__all_sync(0xffffffffu, ready)) break;
-                if (give_up(p, polls)) { failed = true; return part; }
-            }
-            if (lane < k) part = unpack(d);
-        }
-        const E before_in_group = reduce_newest_first(part, lane);
-        if (closes_group && publish && lane == 0 && k == kLbGroup - 1) {
-            // the other tiles need only this, not our own carry: publish it at once
-            st_desc(p.gdesc + gbase + g, pack(compose(before_in_group, tile_total), kAgg));
-        }
-
-        // ---- groups before the own one: lane l looks at group g-1-l; group -1 is x_0
-        E acc = identity_elem<SIGNED>();
         const E x0e = CE::row_start(p, row);
-        for (int base = 1;; base += 32) {
-            const int gg = g - base - lane;
-            Desc d;
-            d.lo = 0ull; d.hi = 0ull;
-            uint32_t inc_mask = 0u;
-            while (true) {
-                if (gg >= 0) d = ld_desc(p.gdesc + gbase + gg);
-                const uint32_t s = (gg >= 0) ? state_of(d) : (uint32_t)kInc;  // gg == -1: x_0; beyond: ignored
-                inc_mask = __ballot_sync(0xffffffffu, s == kInc);
+
+        // tiles of the own group before this one: lane l looks at tiles j-1-5l .. j-5-5l (dist <= k);
+        // groups before the own one: lane l looks at group g-1-l; group -1 is x_0
+        Desc td[kLbPerLane];
+#pragma unroll
+        for (int q = 0; q < kLbPerLane; ++q) { td[q].lo = 0ull; td[q].hi = 0ull; }
+        Desc gd;
+        gd.lo = 0ull; gd.hi = 0ull;
+        bool tiles_done = (k == 0), groups_done = false, group_agg_sent = false;
+        E before_in_group = identity_elem<SIGNED>();
+        E acc = identity_elem<SIGNED>();
+        int gwin = 1;  // distance of the nearest group of the current group window
+        while (true) {
+            if (!tiles_done) {
+#pragma unroll
+                for (int q = 0; q < kLbPerLane; ++q) {
+                    const int dist = kLbPerLane * lane + q + 1;
+                    if (dist <= k) td[q] = ld_desc(p.desc + (T - dist));
+                }
+            }
+            const int gg = g - gwin - lane;
+            if (!groups_done && gg >= 0) gd = ld_desc(p.gdesc + gbase + gg);
+            ++total_polls;
+
+            if (!tiles_done) {
+                bool ready = true;
+#pragma unroll
+                for (int q = 0; q < kLbPerLane; ++q) {
+                    const int dist = kLbPerLane * lane + q + 1;
+                    if (dist <= k && state_of(td[q]) != kAgg) ready = false;
+                }
+                if (__all_sync(0xffffffffu, ready)) {
+                    E part = identity_elem<SIGNED>();
+#pragma unroll
+                    for (int q = 0; q < kLbPerLane; ++q) {
+                        const int dist = kLbPerLane * lane + q + 1;
+                        if (dist <= k) part = compose(unpack(td[q]), part);  // older first
+                    }
+                    before_in_group = reduce_newest_first(part, lane);
+                    tiles_done = true;
+                    if (stamps) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(stamps[0]));
+                }
+            }
+            if (tiles_done && full_group && publish && !group_agg_sent) {
+                // later groups need only this, not our own carry: publish it at once
+                if (lane == 0) st_desc(p.gdesc + gbase + g, pack(compose(before_in_group, tile_total), kAgg));
+                group_agg_sent = true;
+            }
+            if (!groups_done) {
+                const uint32_t s = (gg >= 0) ? state_of(gd) : (uint32_t)kInc;  // gg == -1: x_0; beyond: ignored
+                const uint32_t inc_mask = __ballot_sync(0xffffffffu, s == kInc);
                 const uint32_t ok_mask = __ballot_sync(0xffffffffu, s != kNotReady);
                 const uint32_t need = inc_mask ? ((2u << (__ffs(inc_mask) - 1)) - 1u) : 0xffffffffu;
-                ++total_polls;
-                if ((ok_mask & need) == need) break;
-                if (give_up(p, polls)) { failed = true; return acc; }
+                if ((ok_mask & need) == need) {
+                    const int lstar = inc_mask ? (__ffs(inc_mask) - 1) : 31;
+                    E gp = identity_elem<SIGNED>();
+                    if (lane <= lstar) gp = (gg >= 0) ? unpack(gd) : x0e;
+                    acc = compose(reduce_newest_first(gp, lane), acc);
+                    if (inc_mask) {
+                        groups_done = true;
+                        if (stamps) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(stamps[1]));
+                    } else gwin += 32;  // every group of this window is an aggregate: look further back
+                }
             }
-            const int lstar = inc_mask ? (__ffs(inc_mask) - 1) : 31;
-            E gp = identity_elem<SIGNED>();
-            if (lane <= lstar) gp = (gg >= 0) ? unpack(d) : x0e;
-            acc = compose(reduce_newest_first(gp, lane), acc);
-            if (inc_mask) break;
+            if (tiles_done && groups_done) break;
+            if (give_up(p, polls)) { failed = true; return acc; }
         }
         const E entering = compose(acc, before_in_group);
         if (closes_group && publish && lane == 0) {
@@ -816,7 +846,7 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
             const int b = (int)(i % kLbRing);
             bool failed = !mbar_wait_bounded(agg_bar + 8 * b, (uint32_t)((i / kLbRing) & 1), kCopySpinLimit);
             if (*(volatile int*)&xc->abort) failed = true;
-            unsigned long long t_agg = 0;
+            unsigned long long t_agg = 0, t_pub = 0, stamps[2] = {0, 0};
             unsigned int npolls = 0;
             if (p.debug_flags & 2) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_agg));
             E carry = identity_elem<SIGNED>();
@@ -827,8 +857,9 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                 if (lane < W) xc->wexcl[b][lane] = pack_elem<SIGNED>(wex);
                 const bool muted = (T == p.mute_tile);
                 if (lane == 0 && !muted) LB::publish_agg(p, T, tile_total);
+                if (p.debug_flags & 2) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_pub));
                 if (p.debug_flags & 1) carry = CE::row_start(p, row);
-                else carry = LB::run(p, T, j, row, lane, tile_total, !muted, failed, npolls);
+                else carry = LB::run(p, T, j, row, lane, tile_total, !muted, failed, npolls, (p.debug_flags & 2) ? stamps : nullptr);
             }
             if (lane == 0) {
                 if (failed) {
@@ -840,8 +871,9 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
             if ((p.debug_flags & 2) && lane == 0) {
                 unsigned long long t_done;
                 asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_done));
+                auto d16 = [&](unsigned long long t) { return (unsigned long long)(t > t_agg ? ((t - t_agg) >> 5) & 0xffff : 0); };
                 reinterpret_cast<ulonglong2*>(p.gdesc + p.rows * p.groups_per_row)[T] =
-                    make_ulonglong2(t_agg, (t_done - t_agg) | ((unsigned long long)npolls << 32));
+                    make_ulonglong2(t_agg, d16(t_pub) | (d16(stamps[0]) << 16) | (d16(stamps[1]) << 32) | (d16(t_done) << 48));
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(carry_bar + 8 * b);  // releases wexcl, carry and abort to the CTA
