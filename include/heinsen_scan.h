@@ -144,6 +144,42 @@ hs_status heinsen_scan_log_host(const void* log_a, const void* log_b, const void
 size_t heinsen_scan_host_scratch_bytes(int64_t rows, int64_t n, hs_dtype dtype_in, hs_dtype dtype_out,
                                        int with_signs);
 
+/*
+ * Allocation-free variant of heinsen_scan_log (the paper has no counterpart: this is a service
+ * to callers, not a step of the method).
+ *
+ * Who needs it: code that runs where device memory cannot be requested -- a plug-in called from
+ * another framework's execution callback under a fixed memory plan, a service that forbids
+ * allocation after start-up because cudaMalloc synchronises the device and may fail under
+ * fragmentation, or a host that simply has no allocator to hand this library a workspace.  Such
+ * callers still own their inputs and outputs; what they cannot provide is the scratch that the
+ * single-pass look-back kernel needs for its per-tile descriptors.
+ *
+ * What it does: the same computation as heinsen_scan_log with fp32 storage and no sign tensors
+ * (log_a, log_b: [rows,n]; log_x0: [rows]; log_x: [rows,n]; all DEVICE pointers), always through
+ * the look-back kernel, with the scratch taken from a fixed 1 MiB array that is part of the
+ * library image.  Every GPU that loads the library carries that array until the process exits.
+ * The call performs no cudaMalloc, cudaFree or other allocating call.
+ *
+ * Limits and rules:
+ *   - rows and n must be small enough that heinsen_scan_workspace_bytes(rows, n) <= 1 MiB
+ *     (one row: up to heinsen_scan_static_max_elements() elements, about 1.7e8); larger problems return
+ *     HS_ERR_WORKSPACE_TOO_SMALL and launch nothing.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call outside any stream capture.
+ *   - All calls share the one array and it keeps what the previous call wrote.  The entry point
+ *     clears the part it uses on `stream` before launching, so calls issued one after another on
+ *     one stream are safe; calls that can overlap on the GPU (different streams, or different
+ *     host threads without ordering) race on the array and give undefined results.
+ *   - Device-side errors of the last call are read with heinsen_scan_check_static(stream).
+ */
+hs_status heinsen_scan_log_static(const void* log_a, const void* log_b, const void* log_x0, void* log_x,
+                                  int64_t rows, int64_t n, void* stream);
+/* Synchronises `stream` and returns the device-side status of the last heinsen_scan_log_static call. */
+hs_status heinsen_scan_check_static(void* stream);
+/* Largest n that heinsen_scan_log_static accepts for a single row. */
+size_t heinsen_scan_static_max_elements(void);
+
 /* Process-wide kernel selection (default HS_PATH_AUTO); for tests and benchmarks. */
 hs_status heinsen_scan_set_path(hs_path path);
 /*

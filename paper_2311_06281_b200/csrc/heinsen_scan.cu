@@ -257,7 +257,7 @@ hs_status validate_common(const void* a, const void* b, const void* x0, const vo
     return HS_OK;
 }
 
-hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t stream) {
+hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t stream, int force_path = 0) {
     Params& p = pr.p;
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HS_ERR_INVALID_ARG;
     if (workspace_bytes < sizeof(Header)) return HS_ERR_WORKSPACE_TOO_SMALL;
@@ -275,7 +275,7 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
 
     KernelEntry ke;
     if (!find_kernel(pr.mode, pr.din, pr.dout, tma, ke)) return HS_ERR_INVALID_ARG;
-    const int path = choose_path(p.rows, dev);
+    const int path = force_path ? force_path : choose_path(p.rows, dev);
     const int chunk = 32 * (path == HS_PATH_BATCHED ? ke.K : ke.lb_K);  // elements per warp per step
     p.nchunks = (int)((p.n + chunk - 1) / chunk);
     p.sign_vec_ok = (p.n % 16 == 0) && (!p.sign_a || aligned16(p.sign_a)) && (!p.sign_b || aligned16(p.sign_b)) &&
@@ -384,6 +384,31 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
     return HS_OK;
 }
 
+// Scratch of heinsen_scan_log_static(): lives in the library image, so every GPU that loads the
+// library holds these bytes until the process exits.  In host code `g_static_scratch` is only a
+// handle for the runtime; the device address comes from cudaGetSymbolAddress().
+constexpr size_t kStaticScratchBytes = 1u << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// Device address of g_static_scratch on the current device, looked up once per device.
+hs_status static_scratch_address(void** out) {
+    static std::mutex mu;
+    static void* addr[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail("cudaGetDevice", e);
+    if (dev < 0 || dev >= 64) return HS_ERR_UNSUPPORTED_DEVICE;
+    std::lock_guard<std::mutex> lk(mu);
+    if (!addr[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess) return cuda_fail("cudaGetSymbolAddress", e);
+        addr[dev] = p;
+    }
+    *out = addr[dev];
+    return HS_OK;
+}
+
 }  // namespace
 
 // =============================================================================================
@@ -422,6 +447,44 @@ hs_status heinsen_scan_log(const void* log_a, const void* log_b, const void* log
     if (is_signed) { pr.p.sign_a = sign_a; pr.p.sign_b = sign_b; pr.p.sign_x0 = sign_x0; pr.p.sign_x = sign_x; }
     pr.p.rows = rows; pr.p.n = n;
     return run(pr, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
+}
+
+hs_status heinsen_scan_log_static(const void* log_a, const void* log_b, const void* log_x0, void* log_x, int64_t rows,
+                                  int64_t n, void* stream) {
+    hs_status st = validate_common(log_a, log_b, log_x0, log_x, rows, n);
+    if (st != HS_OK || rows == 0 || n == 0) return st;
+    // the descriptors of every tile of the problem must fit the fixed array
+    if (workspace_bytes_for(rows, n) > kStaticScratchBytes) return HS_ERR_WORKSPACE_TOO_SMALL;
+    void* scratch = nullptr;
+    st = static_scratch_address(&scratch);
+    if (st != HS_OK) return st;
+    Problem pr;
+    std::memset(&pr, 0, sizeof pr);
+    pr.mode = kLogUnsigned;
+    pr.din = pr.dout = HS_F32;
+    pr.p.in_a = log_a; pr.p.in_b = log_b; pr.p.x0 = log_x0; pr.p.out = log_x;
+    pr.p.rows = rows; pr.p.n = n;
+    // run() clears the descriptors it is about to use (cudaMemsetAsync on `stream`), so what the
+    // previous call left in the array does not matter
+    return run(pr, scratch, kStaticScratchBytes, static_cast<cudaStream_t>(stream), HS_PATH_LOOKBACK);
+}
+
+hs_status heinsen_scan_check_static(void* stream) {
+    void* scratch = nullptr;
+    hs_status st = static_scratch_address(&scratch);
+    if (st != HS_OK) return st;
+    return heinsen_scan_check(scratch, stream);
+}
+
+size_t heinsen_scan_static_max_elements(void) {
+    // workspace_bytes_for() grows with rows * ceil(n / 4096); this is the single-row capacity
+    size_t lo = 0, hi = (size_t)1 << 31;
+    while (hi - lo > 1) {
+        const size_t mid = lo + (hi - lo) / 2;
+        if (mid <= (size_t)kMaxN && workspace_bytes_for(1, (long long)mid) <= kStaticScratchBytes) lo = mid;
+        else hi = mid;
+    }
+    return lo;
 }
 
 size_t heinsen_scan_workspace_bytes(int64_t rows, int64_t n) {

@@ -26,6 +26,7 @@ EXPORTS = [
     "heinsen_scan_linear_host", "heinsen_scan_log_host", "heinsen_scan_host_scratch_bytes",
     "heinsen_scan_set_path", "heinsen_scan_debug_config", "heinsen_scan_last_path",
     "heinsen_scan_launch_count", "heinsen_scan_strerror",
+    "heinsen_scan_log_static", "heinsen_scan_check_static", "heinsen_scan_static_max_elements",
 ]
 
 
@@ -68,6 +69,11 @@ def lib() -> ctypes.CDLL:
         L.heinsen_scan_debug_config.restype = ci
         L.heinsen_scan_last_path.restype = ci
         L.heinsen_scan_launch_count.restype = i64
+        L.heinsen_scan_log_static.argtypes = [vp, vp, vp, vp, i64, i64, vp]
+        L.heinsen_scan_log_static.restype = ci
+        L.heinsen_scan_check_static.argtypes = [vp]
+        L.heinsen_scan_check_static.restype = ci
+        L.heinsen_scan_static_max_elements.restype = sz
         L.heinsen_scan_strerror.argtypes = [ci]
         L.heinsen_scan_strerror.restype = ctypes.c_char_p
         _lib = L
@@ -211,6 +217,38 @@ def scan_log(log_a: torch.Tensor, log_b: torch.Tensor, log_x0: torch.Tensor, log
                                       _dtype_code(log_x), _ptr(workspace), workspace.numel(),
                                       _stream_ptr(log_a.device)))
     return (log_x, sign_x) if signed else log_x
+
+
+def scan_log_static(log_a: torch.Tensor, log_b: torch.Tensor, log_x0: torch.Tensor,
+                    log_x: torch.Tensor | None = None) -> torch.Tensor:
+    """heinsen_scan_log_static: float32 log-domain scan that takes its scratch from a fixed array inside
+    the library instead of a caller-provided workspace, for callers that cannot allocate device memory
+    (they still pass inputs and the output).  Problems whose descriptors do not fit that array raise
+    HeinsenScanError(HS_ERR_WORKSPACE_TOO_SMALL).  Calls must not overlap on the GPU.  Asynchronous."""
+    rows, n = log_a.shape
+    _require(log_a, (rows, n), "log_a"); _require(log_b, (rows, n), "log_b"); _require(log_x0, (rows,), "log_x0")
+    if not (log_a.dtype == log_b.dtype == log_x0.dtype == torch.float32):
+        raise TypeError("scan_log_static takes float32 tensors")
+    if log_x is None:
+        log_x = torch.empty_like(log_a)
+    _require(log_x, (rows, n), "log_x")
+    if log_x.dtype != torch.float32:
+        raise TypeError("scan_log_static writes float32")
+    with _on_device(log_a.device):
+        _check(lib().heinsen_scan_log_static(_ptr(log_a), _ptr(log_b), _ptr(log_x0), _ptr(log_x), rows, n,
+                                             _stream_ptr(log_a.device)))
+    return log_x
+
+
+def check_static(device):
+    """Synchronise the current stream of `device` and raise if the last scan_log_static call failed on the device."""
+    device = torch.device(device)
+    with _on_device(device):
+        _check(lib().heinsen_scan_check_static(_stream_ptr(device)))
+
+
+def static_max_elements() -> int:
+    return int(lib().heinsen_scan_static_max_elements())
 
 
 def host_scratch_bytes(rows: int, n: int, dtype_in: torch.dtype, dtype_out: torch.dtype, with_signs: bool) -> int:
