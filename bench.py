@@ -30,7 +30,7 @@ UNIT = "elements/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (None until a capture of that workload exists).
-NCU_TRAFFIC_BYTES = {2: None, 3: None, 4: None, 5: None}
+NCU_TRAFFIC_BYTES = {2: 356.2e6, 3: 662.4e6, 4: None, 5: None}  # cfg3: 2^24 capture scaled by 4 (see profiles/)
 
 HBM_FALLBACK_GBS = 6650.0  # used only when MEASURED_PEAKS.json is absent
 
@@ -42,6 +42,8 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", type=int, default=2, choices=[2, 3, 4, 5])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--rows", type=int, default=None, help="override the workload's rows (profiling of small cases)")
+    ap.add_argument("--n", type=int, default=None, help="override the workload's n (profiling of small cases)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -179,7 +181,7 @@ def run_ours(args):
 
     cid = args.workload
     # weak scaling: every rank runs its own full batch, seeded by its rank
-    w = workloads.make(cid, seed=rank)
+    w = workloads.make(cid, rows=args.rows, n=args.n, seed=rank)
     t = w.tensors
     rows, n = w.rows, w.n
     keys = ("a", "b", "x0") if w.kind == "linear" else ("log_a", "log_b", "log_x0")
@@ -305,7 +307,7 @@ def run_ours(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
-            "config": {"workload": workload_name(cid, w), "rows_per_gpu": rows, "n": n, "storage": w.storage,
+            "config": {"workload": workload_name(cid, w) + ("" if args.rows is None and args.n is None else " [reduced size]"), "rows_per_gpu": rows, "n": n, "storage": w.storage,
                        "entry_point": "heinsen_scan_linear" if w.kind == "linear" else "heinsen_scan_log",
                        "l2": f"{nsets} rotating buffer sets of {alg_bytes / 1e6:.0f} MB each (every set exceeds the 126 MB L2)",
                        "parallelism": f"rows sharded, {world} rank(s), no data-path collective"},

@@ -534,16 +534,55 @@ const char* heinsen_scan_strerror(hs_status status) {
 
 // ---------------------------------------------------------------------------------------------
 // Host-buffer variants: copy in, run, copy out, on `stream`; synchronise before returning.
+constexpr int kHostBlocks = 8;  // row blocks of the host-buffer entry points (copy/compute overlap)
+
+static int host_blocks(int64_t rows) { return rows < kHostBlocks ? (int)rows : kHostBlocks; }
+static size_t up256(size_t v) { return (v + 255) & ~size_t(255); }
+
 size_t heinsen_scan_host_scratch_bytes(int64_t rows, int64_t n, hs_dtype dtype_in, hs_dtype dtype_out, int with_signs) {
     if (rows <= 0 || n <= 0) return 0;
     const size_t es_in = dtype_in == HS_F32 ? 4 : 2, es_out = dtype_out == HS_F32 ? 4 : 2;
-    auto up = [](size_t v) { return (v + 255) & ~size_t(255); };
     const size_t cnt = (size_t)rows * (size_t)n;
-    size_t total = up(workspace_bytes_for(rows, n));
-    total += 2 * up(cnt * es_in) + up((size_t)rows * es_in) + up(cnt * es_out);
-    if (with_signs) total += 3 * up(cnt) + up((size_t)rows);
+    const int nblk = host_blocks(rows);
+    const int64_t rows_blk = (rows + nblk - 1) / nblk;
+    size_t total = (size_t)nblk * up256(workspace_bytes_for(rows_blk, n));
+    total += 2 * up256(cnt * es_in) + up256((size_t)rows * es_in) + up256(cnt * es_out);
+    if (with_signs) total += 3 * up256(cnt) + up256((size_t)rows);
     return total;
 }
+
+namespace {
+// Two side streams per device so that the host->device copy of one row block overlaps the
+// device->host copy of the previous one (PCIe is full duplex) and the kernels in between.
+struct HostLanes {
+    cudaStream_t side[2] = {nullptr, nullptr};
+    cudaEvent_t start = nullptr, done[2] = {nullptr, nullptr};
+    bool ok = false;
+};
+hs_status host_lanes(HostLanes** out) {
+    static std::mutex mu;
+    static HostLanes lanes[64];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail("cudaGetDevice", e);
+    if (dev < 0 || dev >= 64) return HS_ERR_UNSUPPORTED_DEVICE;
+    std::lock_guard<std::mutex> lk(mu);
+    HostLanes& h = lanes[dev];
+    if (!h.ok) {
+        for (int i = 0; i < 2; ++i) {
+            if ((e = cudaStreamCreateWithFlags(&h.side[i], cudaStreamNonBlocking)) != cudaSuccess)
+                return cuda_fail("cudaStreamCreateWithFlags", e);
+            if ((e = cudaEventCreateWithFlags(&h.done[i], cudaEventDisableTiming)) != cudaSuccess)
+                return cuda_fail("cudaEventCreateWithFlags", e);
+        }
+        if ((e = cudaEventCreateWithFlags(&h.start, cudaEventDisableTiming)) != cudaSuccess)
+            return cuda_fail("cudaEventCreateWithFlags", e);
+        h.ok = true;
+    }
+    *out = &h;
+    return HS_OK;
+}
+}  // namespace
 
 static hs_status host_run(int linear, const void* a, const void* b, const void* x0, void* x, const uint8_t* sa,
                           const uint8_t* sb, const uint8_t* sx0, uint8_t* sx, int64_t rows, int64_t n, hs_dtype din,
@@ -555,45 +594,75 @@ static hs_status host_run(int linear, const void* a, const void* b, const void* 
     if (!scratch || (reinterpret_cast<uintptr_t>(scratch) & 255u)) return HS_ERR_INVALID_ARG;
     if (scratch_bytes < heinsen_scan_host_scratch_bytes(rows, n, din, dout, with_signs)) return HS_ERR_WORKSPACE_TOO_SMALL;
     const size_t es_in = din == HS_F32 ? 4 : 2, es_out = dout == HS_F32 ? 4 : 2;
-    auto up = [](size_t v) { return (v + 255) & ~size_t(255); };
     const size_t cnt = (size_t)rows * (size_t)n;
+    const int nblk = host_blocks(rows);
+    const int64_t rows_blk = (rows + nblk - 1) / nblk;
+    const size_t ws_bytes = workspace_bytes_for(rows_blk, n);
+
     uint8_t* w = static_cast<uint8_t*>(scratch);
-    void* ws = w;                 w += up(workspace_bytes_for(rows, n));
-    void* d_a = w;                w += up(cnt * es_in);
-    void* d_b = w;                w += up(cnt * es_in);
-    void* d_x0 = w;               w += up((size_t)rows * es_in);
-    void* d_x = w;                w += up(cnt * es_out);
+    uint8_t* ws0 = w;             w += (size_t)nblk * up256(ws_bytes);
+    uint8_t* d_a = w;             w += up256(cnt * es_in);
+    uint8_t* d_b = w;             w += up256(cnt * es_in);
+    uint8_t* d_x0 = w;            w += up256((size_t)rows * es_in);
+    uint8_t* d_x = w;             w += up256(cnt * es_out);
     uint8_t *d_sa = nullptr, *d_sb = nullptr, *d_sx0 = nullptr, *d_sx = nullptr;
     if (with_signs) {
-        d_sa = w; w += up(cnt);
-        d_sb = w; w += up(cnt);
-        d_sx = w; w += up(cnt);
-        d_sx0 = w; w += up((size_t)rows);
+        d_sa = w; w += up256(cnt);
+        d_sb = w; w += up256(cnt);
+        d_sx = w; w += up256(cnt);
+        d_sx0 = w; w += up256((size_t)rows);
     }
-    cudaError_t e;
-#define HS_CP(dst, src, bytes, kind)                                        \
-    do {                                                                    \
-        e = cudaMemcpyAsync(dst, src, bytes, kind, stream);                 \
-        if (e != cudaSuccess) return cuda_fail("cudaMemcpyAsync", e);       \
-    } while (0)
-    HS_CP(d_a, a, cnt * es_in, cudaMemcpyHostToDevice);
-    HS_CP(d_b, b, cnt * es_in, cudaMemcpyHostToDevice);
-    HS_CP(d_x0, x0, (size_t)rows * es_in, cudaMemcpyHostToDevice);
-    if (with_signs) {
-        if (sa) HS_CP(d_sa, sa, cnt, cudaMemcpyHostToDevice);
-        if (sb) HS_CP(d_sb, sb, cnt, cudaMemcpyHostToDevice);
-        if (sx0) HS_CP(d_sx0, sx0, (size_t)rows, cudaMemcpyHostToDevice);
-    }
-    if (linear)
-        st = heinsen_scan_linear(d_a, d_b, d_x0, d_x, rows, n, din, ws, workspace_bytes_for(rows, n), stream);
-    else
-        st = heinsen_scan_log(d_a, d_b, d_x0, d_x, sa ? d_sa : nullptr, sb ? d_sb : nullptr, sx0 ? d_sx0 : nullptr,
-                              with_signs ? d_sx : nullptr, rows, n, din, dout, ws, workspace_bytes_for(rows, n), stream);
+    HostLanes* hl = nullptr;
+    st = host_lanes(&hl);
     if (st != HS_OK) return st;
-    HS_CP(x, d_x, cnt * es_out, cudaMemcpyDeviceToHost);
-    if (with_signs) HS_CP(sx, d_sx, cnt, cudaMemcpyDeviceToHost);
-#undef HS_CP
-    return heinsen_scan_check(ws, stream);
+    cudaError_t e;
+#define HS_TRY(call)                                          \
+    do {                                                      \
+        e = (call);                                           \
+        if (e != cudaSuccess) return cuda_fail(#call, e);     \
+    } while (0)
+    // the side streams start after everything already queued on the caller's stream
+    HS_TRY(cudaEventRecord(hl->start, stream));
+    HS_TRY(cudaStreamWaitEvent(hl->side[0], hl->start, 0));
+    HS_TRY(cudaStreamWaitEvent(hl->side[1], hl->start, 0));
+    const uint8_t *ha = static_cast<const uint8_t*>(a), *hb = static_cast<const uint8_t*>(b),
+                  *hx0 = static_cast<const uint8_t*>(x0);
+    uint8_t* hx = static_cast<uint8_t*>(x);
+    for (int k = 0; k < nblk; ++k) {
+        const int64_t r0 = (int64_t)k * rows_blk;
+        const int64_t rb = rows - r0 < rows_blk ? rows - r0 : rows_blk;
+        if (rb <= 0) break;
+        cudaStream_t s = hl->side[k & 1];
+        const size_t e0 = (size_t)r0 * (size_t)n, ec = (size_t)rb * (size_t)n;
+        HS_TRY(cudaMemcpyAsync(d_a + e0 * es_in, ha + e0 * es_in, ec * es_in, cudaMemcpyHostToDevice, s));
+        HS_TRY(cudaMemcpyAsync(d_b + e0 * es_in, hb + e0 * es_in, ec * es_in, cudaMemcpyHostToDevice, s));
+        HS_TRY(cudaMemcpyAsync(d_x0 + (size_t)r0 * es_in, hx0 + (size_t)r0 * es_in, (size_t)rb * es_in,
+                               cudaMemcpyHostToDevice, s));
+        if (sa) HS_TRY(cudaMemcpyAsync(d_sa + e0, sa + e0, ec, cudaMemcpyHostToDevice, s));
+        if (sb) HS_TRY(cudaMemcpyAsync(d_sb + e0, sb + e0, ec, cudaMemcpyHostToDevice, s));
+        if (sx0) HS_TRY(cudaMemcpyAsync(d_sx0 + r0, sx0 + r0, (size_t)rb, cudaMemcpyHostToDevice, s));
+        void* ws = ws0 + (size_t)k * up256(ws_bytes);
+        if (linear)
+            st = heinsen_scan_linear(d_a + e0 * es_in, d_b + e0 * es_in, d_x0 + (size_t)r0 * es_in, d_x + e0 * es_out, rb, n,
+                                     din, ws, ws_bytes, s);
+        else
+            st = heinsen_scan_log(d_a + e0 * es_in, d_b + e0 * es_in, d_x0 + (size_t)r0 * es_in, d_x + e0 * es_out,
+                                  sa ? d_sa + e0 : nullptr, sb ? d_sb + e0 : nullptr, sx0 ? d_sx0 + r0 : nullptr,
+                                  with_signs ? d_sx + e0 : nullptr, rb, n, din, dout, ws, ws_bytes, s);
+        if (st != HS_OK) return st;
+        HS_TRY(cudaMemcpyAsync(hx + e0 * es_out, d_x + e0 * es_out, ec * es_out, cudaMemcpyDeviceToHost, s));
+        if (with_signs) HS_TRY(cudaMemcpyAsync(sx + e0, d_sx + e0, ec, cudaMemcpyDeviceToHost, s));
+    }
+    for (int i = 0; i < 2; ++i) {
+        HS_TRY(cudaEventRecord(hl->done[i], hl->side[i]));
+        HS_TRY(cudaStreamWaitEvent(stream, hl->done[i], 0));
+    }
+#undef HS_TRY
+    for (int k = 0; k < nblk; ++k) {
+        st = heinsen_scan_check(ws0 + (size_t)k * up256(ws_bytes), stream);
+        if (st != HS_OK) return st;
+    }
+    return HS_OK;
 }
 
 hs_status heinsen_scan_linear_host(const void* a, const void* b, const void* x0, void* x, int64_t rows, int64_t n,
