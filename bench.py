@@ -243,7 +243,7 @@ def run_ours(args):
     alg_bytes = elements * bpe + rows * (4 if w.storage == "f32" else 2)
     achieved = alg_bytes / (ms_local / args.steps * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": NCU_TRAFFIC_BYTES.get(cid), "peak_source": f"{peak_kind} (MEASURED_PEAKS.json hbm_gbs)"
+                "traffic": NCU_TRAFFIC_BYTES.get(cid) if args.rows is None and args.n is None else None, "peak_source": f"{peak_kind} (MEASURED_PEAKS.json hbm_gbs)"
                 if peak_kind == "measured" else "fallback (no MEASURED_PEAKS.json)",
                 "algorithmic_bytes_per_launch": alg_bytes, "bytes_per_element": bpe,
                 "kernel": "batched_scan_kernel" if hs.last_path() == hs.PATH_BATCHED else "lookback_scan_kernel",

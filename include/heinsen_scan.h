@@ -38,7 +38,8 @@
  *   - rows == 0 or n == 0: HS_OK, nothing is launched.
  *   - log 0 = -inf is a legal input.  +inf and NaN inputs give unspecified values in
  *     their own row from that element on and never affect other rows.
- *   - Errors found on the host (null pointer, negative size, overflow of rows*n,
+ *   - Limits: rows < 2^31, n < 2^31 - 2^20.
+ *   - Errors found on the host (null pointer, negative size, size beyond the limits,
  *     unsupported type, bad workspace) return before any CUDA call.
  *   - Errors found on the device (a bounded wait that ran out) are written to a
  *     status word in `workspace` and are read back by heinsen_scan_check().
@@ -112,7 +113,7 @@ hs_status heinsen_scan_log(const void* log_a, const void* log_b, const void* log
 
 /*
  * Scratch size in bytes for a problem of this shape (any path, any type): a 256-byte
- * header (status word, tile ticket) plus one descriptor per tile of the look-back
+ * header (status words) plus 16 bytes per tile and per group of tiles of the look-back
  * kernel -- the carry between parts that the associativity of prefix sums allows
  * (Summary, footnote on associativity).  Returns 0 only for invalid sizes.
  */
