@@ -1,0 +1,83 @@
+"""The C-ABI library builds, loads, and exports every function that include/heinsen_scan.h declares;
+the argument checks that run before any CUDA call behave as documented.  No GPU needed."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2311_06281_b200 import build_ext, heinsen_scan
+    build_ext.build()
+    return heinsen_scan.lib()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "heinsen_scan.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(heinsen_scan_\w+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    from paper_2311_06281_b200 import heinsen_scan
+    names = declared_functions()
+    assert len(names) >= 12
+    for name in names:
+        assert hasattr(lib, name), f"{name} is declared in the header but not exported"
+    assert sorted(heinsen_scan.EXPORTS) == names, "the Python binding's export list and the header disagree"
+
+
+def test_host_side_validation_needs_no_gpu(lib):
+    buf = np.zeros(64, dtype=np.float32)
+    p = buf.ctypes.data
+    OK, INVALID, TOO_SMALL = 0, 1, 3
+    # empty problems succeed without touching CUDA
+    assert lib.heinsen_scan_log(p, p, p, p, None, None, None, None, 0, 8, 0, 0, None, 0, None) == OK
+    assert lib.heinsen_scan_linear(p, p, p, p, 4, 0, 0, None, 0, None) == OK
+    # null pointers, negative and oversized shapes, unsupported types, missing sign output
+    assert lib.heinsen_scan_log(None, p, p, p, None, None, None, None, 2, 8, 0, 0, p, 4096, None) == INVALID
+    assert lib.heinsen_scan_log(p, p, p, p, None, None, None, None, -2, 8, 0, 0, p, 4096, None) == INVALID
+    assert lib.heinsen_scan_log(p, p, p, p, None, None, None, None, 2, 1 << 31, 0, 0, p, 4096, None) == INVALID
+    assert lib.heinsen_scan_log(p, p, p, p, None, None, None, None, 1 << 31, 8, 0, 0, p, 4096, None) == INVALID
+    assert lib.heinsen_scan_log(p, p, p, p, None, None, None, None, 2, 8, 7, 0, p, 4096, None) == INVALID
+    assert lib.heinsen_scan_log(p, p, p, p, None, None, None, None, 2, 8, 1, 0, p, 4096, None) == INVALID   # bf16 -> f32
+    assert lib.heinsen_scan_log(p, p, p, p, p, None, None, None, 2, 8, 0, 0, p, 4096, None) == INVALID      # no sign_x
+    assert lib.heinsen_scan_linear(p, p, p, p, 2, 8, 1, p, 4096, None) == INVALID                           # bf16 linear
+    # workspace: null, misaligned, too small
+    assert lib.heinsen_scan_log(p, p, p, p, None, None, None, None, 2, 8, 0, 0, None, 4096, None) == INVALID
+    assert lib.heinsen_scan_log(p, p, p, p, None, None, None, None, 2, 8, 0, 0, p + 4, 4096, None) == INVALID
+    aligned = (p + 255) & ~255
+    assert lib.heinsen_scan_log(p, p, p, p, None, None, None, None, 2, 8, 0, 0, aligned, 16, None) == TOO_SMALL
+    assert lib.heinsen_scan_log_static(p, p, p, p, 1 << 20, 4096, None) == TOO_SMALL
+    assert lib.heinsen_scan_set_path(7) == INVALID and lib.heinsen_scan_set_path(0) == OK
+
+
+def test_workspace_sizes_and_messages(lib):
+    assert lib.heinsen_scan_workspace_bytes(0, 8) == 0 and lib.heinsen_scan_workspace_bytes(8, -1) == 0
+    small, big = lib.heinsen_scan_workspace_bytes(1, 4096), lib.heinsen_scan_workspace_bytes(1, 1 << 26)
+    assert 256 <= small <= 512 and small < big <= 1 << 20
+    assert lib.heinsen_scan_workspace_bytes(16384, 2048) < 1 << 20
+    assert lib.heinsen_scan_host_scratch_bytes(16, 1024, 0, 0, 0) >= 3 * 16 * 1024 * 4
+    for code in range(7):
+        msg = lib.heinsen_scan_strerror(code)
+        assert isinstance(msg, bytes) and len(msg) > 1
+    assert lib.heinsen_scan_strerror(99) == b"unknown status"
+    assert lib.heinsen_scan_launch_count() >= 0 and lib.heinsen_scan_last_path() in (0, 1, 2)
+
+
+def test_without_a_gpu_the_product_path_fails_loudly(lib):
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    buf = np.zeros(4096, dtype=np.float32)
+    p = (buf.ctypes.data + 255) & ~255
+    status = lib.heinsen_scan_log(p, p, p, p, None, None, None, None, 2, 8, 0, 0, p, 4096, None)
+    assert status in (2, 4)   # unsupported device / CUDA error: never a silent CPU result
+    from paper_2311_06281_b200 import heinsen_scan
+    with pytest.raises(ValueError):
+        heinsen_scan.scan_log(torch.zeros(2, 8), torch.zeros(2, 8), torch.zeros(2))
