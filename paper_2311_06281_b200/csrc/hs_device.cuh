@@ -72,6 +72,26 @@ __device__ __forceinline__ float log_abs_accurate(float v) {
     return zero ? neg_inf() : fmaf((float)e + bias, kLn2, lm);
 }
 
+// log|v| for the hot path of the linear entry point, about half the cost of log_abs_accurate:
+// near 1 (|v| in (0.875, 1.125)) the Taylor series of log(1+f) in f = |v| - 1 (exact in fp32),
+// relative error <= 1.3e-7; elsewhere lg2.approx, whose absolute error of 2^-22 is there a relative
+// error <= 1.4e-6 of log|v| (inside the 2e-6 |a*_t| term of the tolerance even if it never cancelled).
+// |v| = 0 and denormals give -inf.
+__device__ __forceinline__ float log_abs_fast(float v) {
+    const float av = fabsf(v);
+    const float f = av - 1.0f;
+    float p = fmaf(f, -1.0f / 8.0f, 1.0f / 7.0f);
+    p = fmaf(p, f, -1.0f / 6.0f);
+    p = fmaf(p, f, 1.0f / 5.0f);
+    p = fmaf(p, f, -1.0f / 4.0f);
+    p = fmaf(p, f, 1.0f / 3.0f);
+    p = fmaf(p, f, -0.5f);
+    p = fmaf(p, f, 1.0f);
+    const float near_one = p * f;
+    const float far = lg2(av) * kLn2;
+    return (fabsf(f) < 0.125f) ? near_one : far;
+}
+
 // ------------------------------------------------------------------------------------------
 // The associative element.
 template <bool SIGNED>
@@ -372,7 +392,7 @@ struct Run {
         for (int t = 0; t < K; ++t) {
             float la, lbr;
             if (MODE == kLinear) {
-                la = log_abs_accurate(va[t]);
+                la = log_abs_fast(va[t]);
                 par ^= __float_as_uint(va[t]) & kSignBit;
                 lbr = lg2(fabsf(vb[t])) * kLn2;  // rough: only seeds the reference
             } else {
@@ -421,7 +441,7 @@ struct Run {
 #pragma unroll
         for (int t = 0; t < K; ++t) {
             if (MODE == kLinear) {
-                acc += log_abs_accurate(va[t]);
+                acc += log_abs_fast(va[t]);
                 par ^= __float_as_uint(va[t]) & kSignBit;
             } else {
                 acc += va[t];
