@@ -313,12 +313,14 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         // S input stages per compute warp (phase 2 of a tile runs S-2 iterations after its phase 1),
         // W compute warps (as many as shared memory allows, at most the default), NLB look-back warps
         stages = env_int("HEINSEN_SCAN_LB_STAGES", 4, 3, kLbMaxStages);
-        const int nlb = env_int("HEINSEN_SCAN_LB_LOOKERS", 2, 1, 4);
+        const int nlb = env_int("HEINSEN_SCAN_LB_LOOKERS", 1, 1, 4);
         int W = env_int("HEINSEN_SCAN_LB_WARPS", kLookbackWarps, kLookbackMinWarps, kLbMaxWarps);
         while (W > kLookbackMinWarps && ke.lb_smem(W, stages) + 1024 > dev.max_smem_optin) --W;
         lb_smem = ke.lb_smem(W, stages) + 1024;
         p.lb_warps = nlb;
-        warps = W + nlb;
+        p.lb_sleep_idle = (unsigned)env_int("HEINSEN_SCAN_LB_SLEEP_IDLE", 1000, 0, 100000);
+        p.lb_sleep_ready = (unsigned)env_int("HEINSEN_SCAN_LB_SLEEP_READY", 500, 0, 100000);
+        warps = W + nlb + 1;  // + the publisher warp
         p.tiles_per_row = (int)lookback_tiles_per_row(p.n, chunk, W);
         p.num_tiles = p.rows * p.tiles_per_row;
         // group = the tiles one wave of CTAs processes (the grid is sm_count CTAs: one per SM)

@@ -61,6 +61,8 @@ struct Params {
     int groups_per_row;         // ceil(tiles_per_row / lb_group)
     int lb_group;               // tiles per group: the CTAs of the launch, at most kLbMaxGroup
     int lb_warps;               // look-back warps per CTA
+    unsigned int lb_sleep_idle;   // ns between polls while the tile's own aggregate is not in yet
+    unsigned int lb_sleep_ready;  // ns between polls afterwards
     unsigned int spin_limit;    // bound on polls of predecessor flags
     long long mute_tile;        // test hook: this tile never publishes (-1: none)
     int debug_flags;            // timing experiments only (results are wrong when non-zero)
@@ -569,8 +571,30 @@ __device__ __forceinline__ void st_desc(void* p, Desc d) {
     asm volatile("{\n\t.reg .b128 q;\n\tmov.b128 q, {%1, %2};\n\tst.relaxed.gpu.global.b128 [%0], q;\n\t}"
                  ::"l"(p), "l"(d.lo), "l"(d.hi) : "memory");
 }
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {  // non-blocking
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+template <bool SIGNED>
+__device__ __forceinline__ float4 pack_elem(const Elem<SIGNED>& e) {
+    return make_float4(e.A, e.m, e.s, __uint_as_float(e.p));
+}
+template <bool SIGNED>
+__device__ __forceinline__ Elem<SIGNED> unpack_elem(const float4 v) {
+    Elem<SIGNED> e;
+    e.A = v.x; e.m = v.y; e.s = v.z; e.p = SIGNED ? __float_as_uint(v.w) : 0u;
+    return e;
 }
 
 constexpr int kLbPerLane = 5;                       // tile descriptors polled by each lane per round
@@ -628,17 +652,22 @@ struct Lookback {
                ((polls & 255u) == 0u && *(volatile unsigned long long*)&p.ws->error_id == p.call_id);
     }
 
-    // Warp-collective.  Tile T is tile j of `row`; tile_total its aggregate.  Returns the value of
-    // x entering the tile and publishes the group descriptors this tile is responsible for.
+    // Warp-collective: everything a look-back warp does for tile T (tile j of `row`).  It starts
+    // reading the predecessors' descriptors at once and in the same loop watches for the tile's own
+    // aggregate (mbarrier `agg_bar`, value at `total_src`; the compute warps have already published
+    // it); once both are there it returns the value of x entering the tile.  Publishes the group
+    // descriptors the tile is responsible for.
     __device__ static __forceinline__ E run(const Params& p, long long T, int j, long long row, int lane,
-                                            const E& tile_total, bool publish, bool& failed, unsigned int& total_polls,
-                                            unsigned long long* stamps = nullptr) {
+                                            uint32_t agg_bar, uint32_t agg_parity, const float4* total_src,
+                                            const volatile int* abort_flag, bool& failed,
+                                            unsigned int& total_polls, unsigned long long* stamps = nullptr) {
         failed = false;
         const int gsz = p.lb_group;
         const int g = j / gsz, k = j - g * gsz;                    // group, position in group
         const long long gbase = row * p.groups_per_row;            // first group descriptor of the row
         const bool closes_group = (k == gsz - 1) || (j == p.tiles_per_row - 1);
         const bool full_group = (k == gsz - 1);
+        const bool publish = (T != p.mute_tile);
         unsigned int polls = 0;
         const E x0e = CE::row_start(p, row);
 
@@ -649,9 +678,11 @@ struct Lookback {
         for (int q = 0; q < kLbPerLane; ++q) { td[q].lo = 0ull; td[q].hi = 0ull; }
         Desc gd;
         gd.lo = 0ull; gd.hi = 0ull;
-        bool tiles_done = (k == 0), groups_done = false, group_agg_sent = false;
+        bool own_ready = false, tiles_done = (k == 0), groups_done = (p.debug_flags & 1) != 0, group_agg_sent = false;
+        E tile_total = identity_elem<SIGNED>();
         E before_in_group = identity_elem<SIGNED>();
-        E acc = identity_elem<SIGNED>();
+        E acc = (p.debug_flags & 1) ? x0e : identity_elem<SIGNED>();
+        if (p.debug_flags & 1) tiles_done = true;
         int gwin = 1;  // distance of the nearest group of the current group window
         while (true) {
             if (!tiles_done) {
@@ -665,6 +696,11 @@ struct Lookback {
             if (!groups_done && gg >= 0) gd = ld_desc(p.gdesc + gbase + gg);
             ++total_polls;
 
+            if (!own_ready && mbar_test(agg_bar, agg_parity)) {
+                own_ready = true;
+                if (stamps) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(stamps[2]));
+                tile_total = unpack_elem<SIGNED>(*total_src);  // scanned and published by the compute warps
+            }
             if (!tiles_done) {
                 bool ready = true;
 #pragma unroll
@@ -684,7 +720,7 @@ struct Lookback {
                     if (stamps) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(stamps[0]));
                 }
             }
-            if (tiles_done && full_group && publish && !group_agg_sent) {
+            if (own_ready && tiles_done && full_group && publish && !group_agg_sent) {
                 // later groups need only this, not our own carry: publish it at once
                 if (lane == 0) st_desc(p.gdesc + gbase + g, pack(compose(before_in_group, tile_total), kAgg));
                 group_agg_sent = true;
@@ -705,8 +741,9 @@ struct Lookback {
                     } else gwin += 32;  // every group of this window is an aggregate: look further back
                 }
             }
-            if (tiles_done && groups_done) break;
-            if (give_up(p, polls)) { failed = true; return acc; }
+            if (own_ready && tiles_done && groups_done) break;
+            if (*abort_flag || give_up(p, polls)) { failed = true; return acc; }
+            __nanosleep(own_ready ? p.lb_sleep_ready : p.lb_sleep_idle);  // polls cost L2 bandwidth and issue slots
         }
         const E entering = compose(acc, before_in_group);
         if (closes_group && publish && lane == 0) {
@@ -726,7 +763,9 @@ constexpr int kLbMaxStages = 5; // input stages per compute warp, at most
 struct alignas(16) Exchange {
     float4 agg[kLbRing][kLbMaxWarps];    // per-warp aggregates of a tile
     float4 wexcl[kLbRing][kLbMaxWarps];  // per-warp exclusive prefixes within the tile
+    float4 total[kLbRing];               // the tile's aggregate (written by the last compute warp to finish phase 1)
     float4 carry[kLbRing];               // value of x entering the tile (m, s)
+    unsigned long long total_ready[kLbRing];  // mbarrier: the publisher warp has written total and wexcl
     unsigned long long agg_ready[kLbRing];    // mbarrier: all compute warps have delivered their aggregate
     unsigned long long carry_ready[kLbRing];  // mbarrier: a look-back warp has delivered wexcl and carry
     int abort;
@@ -741,17 +780,6 @@ struct LanePark {
     int slow;
     int pad[3];
 };
-
-template <bool SIGNED>
-__device__ __forceinline__ float4 pack_elem(const Elem<SIGNED>& e) {
-    return make_float4(e.A, e.m, e.s, __uint_as_float(e.p));
-}
-template <bool SIGNED>
-__device__ __forceinline__ Elem<SIGNED> unpack_elem(const float4 v) {
-    Elem<SIGNED> e;
-    e.A = v.x; e.m = v.y; e.s = v.z; e.p = SIGNED ? __float_as_uint(v.w) : 0u;
-    return e;
-}
 
 // One input stage of a compute warp: [a-tensor chunk][b-tensor chunk][park].  The partial sums
 // s_t (fp32) of phase 1 are parked over the b-tensor chunk when the input type is 4 bytes wide
@@ -803,8 +831,8 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align_1024(smem_raw);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int NLB = p.lb_warps;                 // look-back warps (the last NLB warps of the CTA)
-    const int W = (blockDim.x >> 5) - NLB;      // compute warps
+    const int NLB = p.lb_warps;                 // look-back warps; after them comes one publisher warp
+    const int W = (blockDim.x >> 5) - NLB - 1;  // compute warps
     const int S = p.stages;                     // input stages per compute warp
     const int D = S - 2;                        // phase 2 of a tile runs D iterations after its phase 1
 
@@ -813,11 +841,13 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
     Exchange* xc = reinterpret_cast<Exchange*>(tail + (size_t)W * S * sizeof(LanePark));
     const uint32_t warp_bars = smem_u32(reinterpret_cast<uint8_t*>(xc) + sizeof(Exchange));  // [W][kLbMaxStages]
     const uint32_t agg_bar = smem_u32(&xc->agg_ready[0]), carry_bar = smem_u32(&xc->carry_ready[0]);
+    const uint32_t total_bar = smem_u32(&xc->total_ready[0]);
 
     if (threadIdx.x == 0) {
         xc->abort = 0;
         for (int b = 0; b < kLbRing; ++b) {
             mbar_init(agg_bar + 8 * b, W);
+            mbar_init(total_bar + 8 * b, 1);
             mbar_init(carry_bar + 8 * b, 1);
         }
         for (int i = 0; i < W * kLbMaxStages; ++i) mbar_init(warp_bars + 8 * i, 1);
@@ -831,10 +861,38 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
     const long long first = blockIdx.x;
     const long long my_tiles = first < p.num_tiles ? (p.num_tiles - first + G - 1) / G : 0;
 
+    if (warp == W + NLB) {
+        // ------------------------------------------------------------------ publisher warp
+        // Blocks on each tile's chunk aggregates in turn, folds them (per-warp exclusive prefixes
+        // for phase 2, the tile's aggregate for everyone else) and publishes the tile's descriptor
+        // at once: the tiles after this one are waiting for it.
+        TileCursor cur;
+        cur.init(first, tpr);
+        const int g_rows_p = (int)G / tpr, g_rem_p = (int)G % tpr;
+        for (long long i = 0; i < my_tiles; ++i, cur.advance((int)G, g_rows_p, g_rem_p, tpr)) {
+            const int b = (int)(i % kLbRing);
+            if (!mbar_wait_bounded(agg_bar + 8 * b, (uint32_t)((i / kLbRing) & 1), kCopySpinLimit) ||
+                *(volatile int*)&xc->abort) {
+                if (lane == 0) { record_error(p, kErrCopyTimeout, cur.T); xc->abort = 1; }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(total_bar + 8 * b);
+                break;
+            }
+            E mine = (lane < W) ? unpack_elem<SIGNED>(xc->agg[b][lane]) : identity_elem<SIGNED>();
+            E wex, tile_total;
+            warp_scan(mine, lane, wex, tile_total);
+            if (lane < W) xc->wexcl[b][lane] = pack_elem<SIGNED>(wex);
+            if (lane == 0) {
+                if (cur.T != p.mute_tile) LB::publish_agg(p, cur.T, tile_total);
+                xc->total[b] = pack_elem<SIGNED>(tile_total);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(total_bar + 8 * b);
+        }
+        return;
+    }
     if (warp >= W) {
         // ------------------------------------------------------------------ look-back warps
-        // Warp u of NLB takes the CTA's tiles u, u+NLB, u+2*NLB, ...: a tile's look-back lasts
-        // several L2 round trips, longer than a tile's arithmetic, so several are in flight.
         TileCursor cur;
         cur.init(first + (long long)(warp - W) * G, tpr);
         const int lb_stride = NLB * (int)G;
@@ -844,23 +902,12 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
             const long long row = cur.row;
             const int j = cur.j;
             const int b = (int)(i % kLbRing);
-            bool failed = !mbar_wait_bounded(agg_bar + 8 * b, (uint32_t)((i / kLbRing) & 1), kCopySpinLimit);
-            if (*(volatile int*)&xc->abort) failed = true;
-            unsigned long long t_agg = 0, t_pub = 0, stamps[2] = {0, 0};
+            bool failed = false;
+            unsigned long long stamps[3] = {0, 0, 0}, t_start = 0;
             unsigned int npolls = 0;
-            if (p.debug_flags & 2) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_agg));
-            E carry = identity_elem<SIGNED>();
-            if (!failed) {
-                E mine = (lane < W) ? unpack_elem<SIGNED>(xc->agg[b][lane]) : identity_elem<SIGNED>();
-                E wex, tile_total;
-                warp_scan(mine, lane, wex, tile_total);
-                if (lane < W) xc->wexcl[b][lane] = pack_elem<SIGNED>(wex);
-                const bool muted = (T == p.mute_tile);
-                if (lane == 0 && !muted) LB::publish_agg(p, T, tile_total);
-                if (p.debug_flags & 2) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_pub));
-                if (p.debug_flags & 1) carry = CE::row_start(p, row);
-                else carry = LB::run(p, T, j, row, lane, tile_total, !muted, failed, npolls, (p.debug_flags & 2) ? stamps : nullptr);
-            }
+            if (p.debug_flags & 2) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_start));
+            const E carry = LB::run(p, T, j, row, lane, total_bar + 8 * b, (uint32_t)((i / kLbRing) & 1), &xc->total[b],
+                                    &xc->abort, failed, npolls, (p.debug_flags & 2) ? stamps : nullptr);
             if (lane == 0) {
                 if (failed) {
                     record_error(p, kErrLookbackTimeout, T);
@@ -871,9 +918,10 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
             if ((p.debug_flags & 2) && lane == 0) {
                 unsigned long long t_done;
                 asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_done));
+                const unsigned long long t_agg = stamps[2];
                 auto d16 = [&](unsigned long long t) { return (unsigned long long)(t > t_agg ? ((t - t_agg) >> 5) & 0xffff : 0); };
                 reinterpret_cast<ulonglong2*>(p.gdesc + p.rows * p.groups_per_row)[T] =
-                    make_ulonglong2(t_agg, d16(t_pub) | (d16(stamps[0]) << 16) | (d16(stamps[1]) << 32) | (d16(t_done) << 48));
+                    make_ulonglong2(t_agg, d16(t_start) | (d16(stamps[0]) << 16) | (d16(stamps[1]) << 32) | (d16(t_done) << 48));
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(carry_bar + 8 * b);  // releases wexcl, carry and abort to the CTA
@@ -993,7 +1041,15 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
             const long long row = c2.row;
             const int colbase = colbase_of(c2);
             const int st = st2, b = b2;
-            if (!mbar_wait_bounded(carry_bar + 8 * b, parb2, kCopySpinLimit)) {
+            unsigned long long tw0 = 0;
+            if ((p.debug_flags & 2) && warp == 0 && lane == 0) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tw0));
+            const bool carry_ok = mbar_wait_bounded(carry_bar + 8 * b, parb2, kCopySpinLimit);
+            if ((p.debug_flags & 2) && warp == 0 && lane == 0) {
+                unsigned long long tw1;
+                asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tw1));
+                reinterpret_cast<ulonglong2*>(p.gdesc + p.rows * p.groups_per_row)[p.num_tiles + c2.T] = make_ulonglong2(tw0, tw1 - tw0);
+            }
+            if (!carry_ok) {
                 if (lane == 0) { record_error(p, kErrLookbackTimeout, c2.T); xc->abort = 1; }
                 aborted = true;
             } else if (*(volatile int*)&xc->abort) {
