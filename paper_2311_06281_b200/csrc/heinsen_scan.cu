@@ -30,7 +30,7 @@ constexpr long long kMaxTmaDim = kMaxN;
 constexpr int kBatchedMinRowsPerSm = 8;  // fewer rows per SM than this: look-back kernel
 constexpr int kBatchedMinWarpsPerSm = 12; // rows per warp are chosen to keep at least this many warps per SM
 constexpr int kLookbackMinWarps = 8;     // fewest compute warps (= chunks per tile) of the look-back kernel
-constexpr int kLookbackWarps = 12;       // default compute warps of the look-back kernel
+constexpr int kLookbackWarps = 14;       // default compute warps of the look-back kernel
 constexpr int kMinChunk = 512;           // smallest chunk (32 lanes x 16 elements)
 
 unsigned long long next_call_id() {
@@ -315,7 +315,8 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         stages = env_int("HEINSEN_SCAN_LB_STAGES", 4, 3, kLbMaxStages);
         const int nlb = env_int("HEINSEN_SCAN_LB_LOOKERS", 1, 1, 4);
         int W = env_int("HEINSEN_SCAN_LB_WARPS", kLookbackWarps, kLookbackMinWarps, kLbMaxWarps);
-        while (W > kLookbackMinWarps && ke.lb_smem(W, stages) + 1024 > dev.max_smem_optin) --W;
+        if (stages > 5) stages = 5;
+        while (W > kLookbackMinWarps && (ke.lb_smem(W, stages) + 1024 > dev.max_smem_optin || W + nlb + 1 > 16)) --W;
         lb_smem = ke.lb_smem(W, stages) + 1024;
         p.lb_warps = nlb;
         p.lb_sleep_idle = (unsigned)env_int("HEINSEN_SCAN_LB_SLEEP_IDLE", 1000, 0, 100000);

@@ -761,8 +761,8 @@ struct Lookback {
 constexpr int kLbRing = 4;      // ring slots: tiles between "aggregate delivered" and "carry consumed"
 constexpr int kLbMaxStages = 5; // input stages per compute warp, at most
 struct alignas(16) Exchange {
-    float4 agg[kLbRing][kLbMaxWarps];    // per-warp aggregates of a tile
-    float4 wexcl[kLbRing][kLbMaxWarps];  // per-warp exclusive prefixes within the tile
+    float4 agg[kLbRing][kLbMaxWarps];    // per-warp aggregates of a tile; the publisher warp replaces them in
+                                         // place by the per-warp exclusive prefixes within the tile
     float4 total[kLbRing];               // the tile's aggregate (written by the last compute warp to finish phase 1)
     float4 carry[kLbRing];               // value of x entering the tile (m, s)
     unsigned long long total_ready[kLbRing];  // mbarrier: the publisher warp has written total and wexcl
@@ -772,13 +772,13 @@ struct alignas(16) Exchange {
     int pad[3];
 };
 
-// Per-lane state parked between the two phases of a chunk (structure of arrays, one per stage).
+// Per-lane state carried from phase 1 to phase 2 of a chunk.  It stays in registers: the compute
+// warps keep the records of the last four tiles and shift them by one every iteration.
+template <bool SIGNED>
 struct LanePark {
-    float r[32];
-    float A[32], m[32], s[32];
-    uint32_t p[32];
-    int slow;
-    int pad[3];
+    float r;              // reference of the lane's run
+    Elem<SIGNED> excl;    // parts of the chunk before the lane's run
+    bool slow;            // the chunk took the tracked form in phase 1 (warp-uniform)
 };
 
 // One input stage of a compute warp: [a-tensor chunk][b-tensor chunk][park].  The partial sums
@@ -796,7 +796,7 @@ struct LbStage {
 // total dynamic shared memory of the look-back kernel for W compute warps and S stages (without alignment slack)
 template <typename TIn, int K>
 __host__ __device__ constexpr int lb_total_smem_bytes(int W, int S) {
-    return W * S * (LbStage<TIn, K>::BYTES + (int)sizeof(LanePark)) + (int)sizeof(Exchange) + W * kLbMaxStages * 8;
+    return W * S * LbStage<TIn, K>::BYTES + (int)sizeof(Exchange) + W * kLbMaxStages * 8;
 }
 
 // Position of a CTA's tile sequence: tile T = tile j of row `row`; advances by a fixed stride
@@ -818,7 +818,7 @@ struct TileCursor {
 };
 
 template <int MODE, typename TIn, typename TOut, int K, bool TMA>
-__global__ void __launch_bounds__(640, 1)
+__global__ void __launch_bounds__(512, 1)
 lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                      const __grid_constant__ CUtensorMap tm_o) {
     using CE = ChunkEngine<MODE, TIn, TOut, K>;
@@ -837,8 +837,7 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
     const int D = S - 2;                        // phase 2 of a tile runs D iterations after its phase 1
 
     uint8_t* tail = smem + (size_t)W * S * ST::BYTES;
-    LanePark* all_parks = reinterpret_cast<LanePark*>(tail);  // [W][S]
-    Exchange* xc = reinterpret_cast<Exchange*>(tail + (size_t)W * S * sizeof(LanePark));
+    Exchange* xc = reinterpret_cast<Exchange*>(tail);
     const uint32_t warp_bars = smem_u32(reinterpret_cast<uint8_t*>(xc) + sizeof(Exchange));  // [W][kLbMaxStages]
     const uint32_t agg_bar = smem_u32(&xc->agg_ready[0]), carry_bar = smem_u32(&xc->carry_ready[0]);
     const uint32_t total_bar = smem_u32(&xc->total_ready[0]);
@@ -881,7 +880,7 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
             E mine = (lane < W) ? unpack_elem<SIGNED>(xc->agg[b][lane]) : identity_elem<SIGNED>();
             E wex, tile_total;
             warp_scan(mine, lane, wex, tile_total);
-            if (lane < W) xc->wexcl[b][lane] = pack_elem<SIGNED>(wex);
+            if (lane < W) xc->agg[b][lane] = pack_elem<SIGNED>(wex);  // every lane has read its aggregate by now
             if (lane == 0) {
                 if (cur.T != p.mute_tile) LB::publish_agg(p, cur.T, tile_total);
                 xc->total[b] = pack_elem<SIGNED>(tile_total);
@@ -942,7 +941,9 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
     auto st_a = [&](int st) { return wb + st * ST::BYTES; };
     auto st_b = [&](int st) { return wb + st * ST::BYTES + ST::IN_BYTES; };
     auto st_park = [&](int st) { return wb + st * ST::BYTES + ST::PARK_OFF; };
-    LanePark* lpark = all_parks + (size_t)warp * S;
+    LanePark<SIGNED> lp[4];  // lp[d]: the tile that went through phase 1 d iterations ago
+#pragma unroll
+    for (int d = 0; d < 4; ++d) { lp[d].r = neg_inf(); lp[d].excl = identity_elem<SIGNED>(); lp[d].slow = false; }
     const uint32_t bars = warp_bars + warp * (8 * kLbMaxStages);
 
     // TMA helpers (same box geometry as WarpPipe, buffers laid out per stage here)
@@ -990,6 +991,7 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
     int b1 = 0, b2 = 0;            // ring slots of those tiles
     uint32_t parb2 = 0;            // parity of ring slot b2's carry mbarrier
     for (long long i = 0; i < my_tiles + D && !aborted; ++i) {
+        lp[3] = lp[2]; lp[2] = lp[1]; lp[1] = lp[0];
         // ---- phase 1 of tile i
         if (i < my_tiles) {
             const long long row = c1.row;
@@ -1016,19 +1018,15 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                 typename CE::Pending pd;
                 E total;
                 CE::phase1(p, st_a(st), st_b(st), off, lm, lane, row, col0, colbase + CHUNK > p.n, pd, total);
-                LanePark& lp = lpark[st];
                 if (!pd.slow) {  // park the partial sums (a slow chunk keeps its inputs instead)
                     const uint32_t pb = st_park(st);
 #pragma unroll
                     for (int jx = 0; jx < K / 4; ++jx) sts128(pb + park_off[jx], Storage<float>::pack(pd.run.s + 4 * jx));
                 }
-                lp.r[lane] = pd.run.r;
-                lp.A[lane] = pd.excl.A; lp.m[lane] = pd.excl.m; lp.s[lane] = pd.excl.s;
-                if (SIGNED) lp.p[lane] = pd.excl.p;
-                if (lane == 0) {
-                    lp.slow = pd.slow ? 1 : 0;
-                    xc->agg[b][warp] = pack_elem<SIGNED>(total);
-                }
+                lp[0].r = pd.run.r;
+                lp[0].excl = pd.excl;
+                lp[0].slow = pd.slow;
+                if (lane == 0) xc->agg[b][warp] = pack_elem<SIGNED>(total);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(agg_bar + 8 * b);
             }
@@ -1060,17 +1058,16 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                 const long long left = p.n - col0;
                 E carry;
                 carry.A = neg_inf(); carry.m = xc->carry[b].x; carry.s = xc->carry[b].y; carry.p = 0u;
-                const LanePark& lp = lpark[st];
-                E excl;
-                excl.A = lp.A[lane]; excl.m = lp.m[lane]; excl.s = lp.s[lane]; excl.p = SIGNED ? lp.p[lane] : 0u;
-                const E entering = compose(compose(carry, unpack_elem<SIGNED>(xc->wexcl[b][warp])), excl);
+                const LanePark<SIGNED> mine = (D == 1) ? lp[1] : (D == 2) ? lp[2] : lp[3];
+                const E excl = mine.excl;
+                const E entering = compose(compose(carry, unpack_elem<SIGNED>(xc->agg[b][warp])), excl);
                 uint32_t sm_a = st_a(st);
                 uint32_t sm_b = st_b(st);
                 const uint32_t pb = st_park(st);
                 float out_mag[K];
                 uint32_t out_sign[MODE == kLogSigned ? K : 1];
                 bool ok = false;
-                const bool was_slow = lp.slow != 0;
+                const bool was_slow = mine.slow;
                 if (!was_slow) {
                     // rebuild A_t (and the parity of a) from the inputs, fetch the parked s_t, apply
                     float va[K];
@@ -1084,7 +1081,7 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                     if (MODE == kLogSigned) CE::load_signs(p.sign_a, row * p.n + col0, left, p.sign_vec_ok != 0, sa);
                     R_ run;
                     run.rebuild(va, sa);
-                    run.r = lp.r[lane];
+                    run.r = mine.r;
 #pragma unroll
                     for (int jx = 0; jx < K / 4; ++jx) Storage<float>::unpack(lds128(pb + park_off[jx]), run.s + 4 * jx);
                     ok = run.apply(entering, out_mag, out_sign);
