@@ -319,8 +319,8 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         while (W > kLookbackMinWarps && (ke.lb_smem(W, stages) + 1024 > dev.max_smem_optin || W + nlb + 1 > 16)) --W;
         lb_smem = ke.lb_smem(W, stages) + 1024;
         p.lb_warps = nlb;
-        p.lb_sleep_idle = (unsigned)env_int("HEINSEN_SCAN_LB_SLEEP_IDLE", 1000, 0, 100000);
-        p.lb_sleep_ready = (unsigned)env_int("HEINSEN_SCAN_LB_SLEEP_READY", 500, 0, 100000);
+        p.lb_sleep_idle = (unsigned)env_int("HEINSEN_SCAN_LB_SLEEP_IDLE", 200, 0, 100000);
+        p.lb_sleep_ready = (unsigned)env_int("HEINSEN_SCAN_LB_SLEEP_READY", 0, 0, 100000);
         warps = W + nlb + 1;  // + the publisher warp
         p.tiles_per_row = (int)lookback_tiles_per_row(p.n, chunk, W);
         p.num_tiles = p.rows * p.tiles_per_row;
