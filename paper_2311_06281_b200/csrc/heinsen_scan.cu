@@ -293,8 +293,10 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         // per SM, so that rows with many steps use few scan steps and few rows still fill the GPU.
         int R = 8;
         while (R > 1 && (p.rows + R - 1) / R < (long long)kBatchedMinWarpsPerSm * dev.sm_count) R >>= 1;
-        // whole chunks and enough rows: one row per warp, each chunk one contiguous 2 KB box
-        if (tma && p.n % chunk == 0 && p.rows >= (long long)kBatchedMinWarpsPerSm * dev.sm_count) R = 1;
+        // rows that start on 128-byte lines, and enough of them: one row per warp, each chunk one contiguous box
+        if (tma && (p.n * es_in) % 128 == 0 && (p.n * es_out) % 128 == 0 &&
+            p.rows >= (long long)kBatchedMinWarpsPerSm * dev.sm_count)
+            R = 1;
         R = env_int("HEINSEN_SCAN_ROWS_PER_WARP", R, 1, 8);
         while (R & (R - 1)) R &= R - 1;  // power of two
         p.rows_per_warp = R;
@@ -336,20 +338,22 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         grid = 0;  // set below from occupancy
     }
 
-    CUtensorMap tm_a, tm_b, tm_o;
+    CUtensorMap tm_a, tm_b, tm_o, tm_o1;
+    std::memset(&tm_o1, 0, sizeof tm_o1);
     std::memset(&tm_a, 0, sizeof tm_a);
     std::memset(&tm_b, 0, sizeof tm_b);
     std::memset(&tm_o, 0, sizeof tm_o);
     if (tma) {
         // one row per warp and whole chunks only: move a chunk as a single box of consecutive lines
-        const bool flat = p.rows_per_warp == 1 && p.n % chunk == 0 && p.rows * p.n * es_in / 128 < (1ll << 31) &&
-                          !env_int("HEINSEN_SCAN_NO_FLAT", 0, 0, 1);
+        const bool flat = p.rows_per_warp == 1 && (p.n * es_in) % 128 == 0 && (p.n * es_out) % 128 == 0 &&
+                          p.rows * p.n * es_in / 128 < (1ll << 31) && !env_int("HEINSEN_SCAN_NO_FLAT", 0, 0, 1);
         p.flat_boxes = flat ? 1 : 0;
         const int br_in = flat ? chunk * es_in / 128 : p.rows_per_warp;
         const int br_out = flat ? chunk * es_out / 128 : p.rows_per_warp;
         if (!make_tmap(&tm_a, p.in_a, pr.din, p.rows, p.n, br_in, flat) ||
             !make_tmap(&tm_b, p.in_b, pr.din, p.rows, p.n, br_in, flat) ||
-            !make_tmap(&tm_o, p.out, pr.dout, p.rows, p.n, br_out, flat)) {
+            !make_tmap(&tm_o, p.out, pr.dout, p.rows, p.n, br_out, flat) ||
+            (flat && !make_tmap(&tm_o1, p.out, pr.dout, p.rows, p.n, 1, true))) {
             snprintf(g_cuda_msg, sizeof g_cuda_msg, "cuTensorMapEncodeTiled failed");
             return HS_ERR_CUDA;
         }
@@ -362,7 +366,7 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
     cudaError_t e = ensure_smem_attr(fn, smem);
     if (e != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", e);
 
-    void* args[] = {&p, &tm_a, &tm_b, &tm_o};
+    void* args[] = {&p, &tm_a, &tm_b, &tm_o, &tm_o1};
     if (path == HS_PATH_LOOKBACK) {
         // Tiles wait for their predecessors, so every CTA must be resident: size the grid from the
         // occupancy of this kernel and launch cooperatively (the launch fails rather than deadlocks).

@@ -49,8 +49,9 @@ struct Params {
     int stages;         // input stages per warp (2..kMaxStages)
     int sign_vec_ok;    // sign tensors may be accessed with 16-byte vectors
     int rows_per_warp;  // R: rows held by one warp of the batched kernel (1, 2, 4, 8); look-back: 1
-    int flat_boxes;     // R == 1 and n a multiple of the chunk: a chunk moves as ONE box of consecutive
+    int flat_boxes;     // R == 1 and rows start on 128-byte lines: a chunk moves as ONE box of consecutive
                         // 128-byte lines of the flat [rows*n/line, line] view instead of one box per line
+                        // (the partial last chunk of a row is stored line by line so as not to touch the next row)
     unsigned long long call_id;
     Header* ws;
     // look-back kernel only
@@ -344,7 +345,7 @@ struct WarpPipe {
         R = rows_per_warp;
         flat = flat_boxes;
         in_boxes = flat ? 1 : IN_BYTES / (128 * R);
-        out_boxes = flat ? 1 : OUT_BYTES / (128 * R);
+        out_boxes = flat ? OUT_BYTES / 128 : OUT_BYTES / (128 * R);  // lanes that issue (or may issue) stores
     }
     __device__ __forceinline__ uint32_t in_a(int s) const { return base + s * 2 * IN_BYTES; }
     __device__ __forceinline__ uint32_t in_b(int s) const { return base + s * 2 * IN_BYTES + IN_BYTES; }
@@ -384,17 +385,23 @@ struct WarpPipe {
         if (lane < out_boxes) bulk_wait_read<1>();
         __syncwarp();
     }
-    // store the chunk held in shared memory at `src`; `line`: as for issue(), in output lines
-    __device__ __forceinline__ void store_from(const CUtensorMap* tm_o, int row0, int colbase, int line, uint32_t src) const {
+    // store the chunk held in shared memory at `src`; `line`: as for issue(), in output lines;
+    // flat boxes: `valid_lines` < OUT_LINES for the partial last chunk of a row, which goes out as
+    // single lines through `tm_o1` (same view, one-line box)
+    __device__ __forceinline__ void store_from(const CUtensorMap* tm_o, const CUtensorMap* tm_o1, int row0, int colbase,
+                                               int line, uint32_t src, int valid_lines) const {
         fence_async_smem();
         __syncwarp();
-        if (lane < out_boxes) {
-            if (flat) {
-                tma_store_2d(tm_o, 0, line, src);
-            } else {
-                const int x = colbase + lane * OUT_PER_BOX;
-                tma_store_2d(tm_o, x, row0, src + (uint32_t)(lane * R * 128));
+        if (flat) {
+            if (valid_lines >= OUT_BYTES / 128) {
+                if (lane == 0) tma_store_2d(tm_o, 0, line, src);
+            } else if (lane < valid_lines) {
+                tma_store_2d(tm_o1, 0, line + lane, src + (uint32_t)(lane * 128));
             }
+            if (lane < out_boxes) bulk_commit();  // every lane that may ever store keeps its group count in step
+        } else if (lane < out_boxes) {
+            const int x = colbase + lane * OUT_PER_BOX;
+            tma_store_2d(tm_o, x, row0, src + (uint32_t)(lane * R * 128));
             bulk_commit();
         }
     }
@@ -418,7 +425,7 @@ struct WarpPipe {
 template <int MODE, typename TIn, typename TOut, int K, bool TMA>
 __global__ void __launch_bounds__(512, 1)
 batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-                    const __grid_constant__ CUtensorMap tm_o) {
+                    const __grid_constant__ CUtensorMap tm_o, const __grid_constant__ CUtensorMap tm_o1) {
     using CE = ChunkEngine<MODE, TIn, TOut, K>;
     using E = typename CE::E;
     extern __shared__ uint8_t smem_raw[];
@@ -512,7 +519,8 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
         renormalise(state);
 
         if (TMA) {
-            pipe.store_from(&tm_o, group * R, colbase, oline, sm_out);
+            pipe.store_from(&tm_o, &tm_o1, group * R, colbase, oline, sm_out,
+                            ragged ? (int)((p.n - colbase) / Pipe::OUT_PER_BOX) : Pipe::OUT_LINES);
         } else {
             __syncwarp();
             CE::generic_store(p, sm_out, lm, lane, (long long)group * R, colbase);
@@ -820,7 +828,7 @@ struct TileCursor {
 template <int MODE, typename TIn, typename TOut, int K, bool TMA>
 __global__ void __launch_bounds__(512, 1)
 lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-                     const __grid_constant__ CUtensorMap tm_o) {
+                     const __grid_constant__ CUtensorMap tm_o, const __grid_constant__ CUtensorMap tm_o1) {
     using CE = ChunkEngine<MODE, TIn, TOut, K>;
     using LB = Lookback<MODE, TIn, TOut, K>;
     using R_ = Run<MODE, TIn, TOut, K>;
@@ -950,7 +958,8 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
     const bool flat = p.flat_boxes != 0;
     constexpr int IN_PER_BOX = 128 / (int)sizeof(TIn), OUT_PER_BOX = 128 / (int)sizeof(TOut);
     const int in_boxes = flat ? 1 : ST::IN_BYTES / 128;
-    const int out_boxes = flat ? 1 : (CHUNK * (int)sizeof(TOut)) / 128;
+    constexpr int OUT_LINES = (CHUNK * (int)sizeof(TOut)) / 128;
+    const int out_boxes = OUT_LINES;  // lanes that issue (or may issue) stores
 
     const int g_rows = (int)G / tpr, g_rem = (int)G % tpr;
     TileCursor ci, c1, c2;  // tiles being loaded, in phase 1, in phase 2
@@ -1114,10 +1123,20 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                 if (TMA) {
                     fence_async_smem();
                     __syncwarp();
-                    // a chunk wholly beyond the row end has nothing to store (a flat box is not clipped per row)
-                    if (lane < out_boxes && colbase < p.n) {
-                        if (flat) tma_store_2d(&tm_o, 0, (int)((row * p.n + colbase) / OUT_PER_BOX), pb);
-                        else tma_store_2d(&tm_o, (int)colbase + lane * OUT_PER_BOX, (int)row, pb + (uint32_t)(lane * 128));
+                    // a flat box is not clipped per row: a chunk wholly beyond the row end stores nothing, the
+                    // partial last chunk of a row goes out line by line
+                    if (flat) {
+                        const long long rem = p.n - colbase;
+                        const int valid = rem >= CHUNK ? OUT_LINES : (rem > 0 ? (int)(rem / OUT_PER_BOX) : 0);
+                        const int line = (int)((row * p.n + colbase) / OUT_PER_BOX);
+                        if (valid >= OUT_LINES) {
+                            if (lane == 0) tma_store_2d(&tm_o, 0, line, pb);
+                        } else if (lane < valid) {
+                            tma_store_2d(&tm_o1, 0, line + lane, pb + (uint32_t)(lane * 128));
+                        }
+                        if (lane < OUT_LINES) bulk_commit();
+                    } else if (lane < out_boxes) {
+                        tma_store_2d(&tm_o, colbase + lane * OUT_PER_BOX, (int)row, pb + (uint32_t)(lane * 128));
                         bulk_commit();
                     }
                 } else {

@@ -141,6 +141,30 @@ def test_odd_shapes_signed_linear(hs, oracle, n):
         run_linear(hs, oracle, w.tensors, path=path, signed=True, what=f"signed 5x{n}/{path}")
 
 
+@pytest.mark.parametrize("rows,n,cid", [(1800, 1056, 2), (1800, 544, 2), (2, 5 * 512 + 96, 2), (1900, 1088, 5), (3, 7 * 512 + 64, 5)])
+def test_rows_on_128_byte_lines_with_partial_last_chunk(hs, oracle, rows, n, cid):
+    """Rows that start on 128-byte lines move as single contiguous boxes even when n is not a multiple of
+    the chunk; the partial last chunk of every row must not spill into the next row (canaries around the
+    output, exact parity inside)."""
+    w = workloads.make(cid, rows=rows, n=n)
+    t = w.tensors
+    la, lb, lx0 = to_dev(t["log_a"]), to_dev(t["log_b"]), to_dev(t["log_x0"])
+    ref, _ = oracle.scan_log(t["log_a"], t["log_b"], t["log_x0"])
+    tol = tol_positive(storage_f64(t["log_a"]), ref)
+    if cid == 5:
+        tol = tol + 1e-2 * np.abs(ref)
+    pad = 4096
+    buf = torch.zeros(rows * n + 2 * pad, dtype=la.dtype, device="cuda")
+    buf[:pad] = 12345.0
+    buf[-pad:] = 12345.0
+    out = buf[pad:pad + rows * n].view(rows, n)
+    ws = hs.new_workspace(rows, n, "cuda")
+    hs.scan_log(la, lb, lx0, log_x=out, workspace=ws)
+    hs.check(ws)
+    assert_log_close(to_f64(out), ref, tol, f"{rows}x{n}")
+    assert (buf[:pad] == 12345.0).all() and (buf[-pad:] == 12345.0).all()
+
+
 def test_unaligned_base_pointer(hs, oracle):
     w = workloads.make(2, rows=9, n=1000)
     t = w.tensors
