@@ -44,6 +44,9 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--rows", type=int, default=None, help="override the workload's rows (profiling of small cases)")
     ap.add_argument("--n", type=int, default=None, help="override the workload's n (profiling of small cases)")
+    ap.add_argument("--fig1", action="store_true",
+                    help="the paper's only experiment: sequential (CPU oracle, one core) over parallel (this library) "
+                         "time for one sequence of n = 2^10..2^28 elements, means of 30 runs; prints one JSON object")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -319,8 +322,60 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_fig1(args):
+    """Figure 1 of the paper: time to compute n elements sequentially relative to the parallel evaluation,
+    each point the mean of 30 runs.  Sequential = the float64 oracle loop on one host core; parallel =
+    heinsen_scan_linear on one B200 with the inputs resident on the device (single sequence, look-back path)."""
+    import math
+
+    import numpy as np
+    import torch
+
+    from oracle import heinsen_oracle
+    from paper_2311_06281_b200 import build_ext, heinsen_scan as hs, workloads
+
+    build_ext.build()
+    heinsen_oracle.build()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    points = []
+    for e in range(10, 29, 2):
+        n = 1 << e
+        t = workloads.make(1, rows=1, n=n).tensors
+        a, b, x0 = (torch.from_numpy(t[k]).to(dev) for k in ("a", "b", "x0"))
+        x = torch.empty_like(a)
+        ws = hs.new_workspace(1, n, dev)
+        for _ in range(5):
+            hs.scan_linear(a, b, x0, x=x, workspace=ws)
+        torch.cuda.synchronize()
+        gpu = []
+        for _ in range(30):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            hs.scan_linear(a, b, x0, x=x, workspace=ws)
+            e1.record()
+            torch.cuda.synchronize()
+            gpu.append(e0.elapsed_time(e1) * 1e-3)
+        hs.check(ws)
+        reps = 30 if n <= (1 << 24) else 5   # bounded: the largest sizes take ~1 s per sequential run
+        cpu = []
+        for _ in range(reps):
+            t0 = time.perf_counter()
+            heinsen_oracle.scan_linear(t["a"], t["b"], t["x0"], nthreads=1)
+            cpu.append(time.perf_counter() - t0)
+        points.append({"n": n, "sequential_s": float(np.mean(cpu)), "sequential_runs": reps,
+                       "parallel_s": float(np.mean(gpu)), "parallel_runs": 30,
+                       "ratio": float(np.mean(cpu) / np.mean(gpu)), "n_over_log2n": n / math.log2(n)})
+        del a, b, x, ws
+    print(json.dumps({"fig1": points, "sequential": "float64 oracle loop, 1 host core", "parallel": "heinsen_scan_linear, 1x B200, "
+                      "device-resident inputs, wall time of one call incl. launch"}), flush=True)
+
+
 def main():
     args = parse_args()
+    if args.fig1:
+        run_fig1(args)
+        return
     if args.impl == "reference":
         run_reference(args)
     else:

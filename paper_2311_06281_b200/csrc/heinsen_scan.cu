@@ -378,10 +378,16 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         long long g = (long long)per_sm * dev.sm_count;
         if (g > p.num_tiles) g = p.num_tiles;
         grid = (int)g;
-        // every descriptor starts as "nothing yet"
-        e = cudaMemsetAsync(p.desc, 0, ((size_t)p.num_tiles + (size_t)p.rows * p.groups_per_row) * 16, stream);
-        if (e != cudaSuccess) return cuda_fail("cudaMemsetAsync", e);
-        e = cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(warps * 32), args, smem, stream);
+        if (p.tiles_per_row == 1) {
+            // every row is a single tile: no tile waits for another, so neither the descriptors nor the
+            // co-residency guarantee of a cooperative launch are needed
+            e = cudaLaunchKernel(fn, dim3(grid), dim3(warps * 32), args, smem, stream);
+        } else {
+            // every descriptor starts as "nothing yet"
+            e = cudaMemsetAsync(p.desc, 0, ((size_t)p.num_tiles + (size_t)p.rows * p.groups_per_row) * 16, stream);
+            if (e != cudaSuccess) return cuda_fail("cudaMemsetAsync", e);
+            e = cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(warps * 32), args, smem, stream);
+        }
     } else {
         e = cudaLaunchKernel(fn, dim3(grid), dim3(warps * 32), args, smem, stream);
     }
