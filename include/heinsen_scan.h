@@ -181,6 +181,20 @@ hs_status heinsen_scan_check_static(void* stream);
 /* Largest n that heinsen_scan_log_static accepts for a single row. */
 size_t heinsen_scan_static_max_elements(void);
 
+/*
+ * The two calls in their shortest form: fp32 storage, legacy default stream, automatic kernel
+ * selection, scratch from the library's fixed 1 MiB array (the rules of heinsen_scan_log_static
+ * apply: problems whose look-back descriptors do not fit return HS_ERR_WORKSPACE_TOO_SMALL; calls
+ * must not overlap on the GPU).  scan_linear: Eq. 3 / Eq. 7 on linear inputs, as
+ * heinsen_scan_linear.  scan_log: Eq. 7 on log inputs with optional sign tensors (NULL = all
+ * positive; sign_x required iff any sign input is given), as heinsen_scan_log.  Device pointers.
+ * Device-side errors are read with heinsen_scan_check_static(NULL).
+ */
+hs_status scan_linear(const void* a, const void* b, const void* x0, void* x, int64_t rows, int64_t n);
+hs_status scan_log(const void* log_a, const void* log_b, const void* log_x0, void* log_x,
+                   const uint8_t* sign_a, const uint8_t* sign_b, const uint8_t* sign_x0, uint8_t* sign_x,
+                   int64_t rows, int64_t n);
+
 /* Process-wide kernel selection (default HS_PATH_AUTO); for tests and benchmarks. */
 hs_status heinsen_scan_set_path(hs_path path);
 /*

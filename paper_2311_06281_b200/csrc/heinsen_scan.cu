@@ -482,6 +482,27 @@ hs_status heinsen_scan_log_static(const void* log_a, const void* log_b, const vo
     return run(pr, scratch, kStaticScratchBytes, static_cast<cudaStream_t>(stream), HS_PATH_LOOKBACK);
 }
 
+hs_status scan_linear(const void* a, const void* b, const void* x0, void* x, int64_t rows, int64_t n) {
+    hs_status st = validate_common(a, b, x0, x, rows, n);
+    if (st != HS_OK || rows == 0 || n == 0) return st;
+    void* scratch = nullptr;
+    st = static_scratch_address(&scratch);
+    if (st != HS_OK) return st;
+    return heinsen_scan_linear(a, b, x0, x, rows, n, HS_F32, scratch, kStaticScratchBytes, nullptr);
+}
+
+hs_status scan_log(const void* log_a, const void* log_b, const void* log_x0, void* log_x, const uint8_t* sign_a,
+                   const uint8_t* sign_b, const uint8_t* sign_x0, uint8_t* sign_x, int64_t rows, int64_t n) {
+    hs_status st = validate_common(log_a, log_b, log_x0, log_x, rows, n);
+    if (st != HS_OK || rows == 0 || n == 0) return st;
+    if ((sign_a || sign_b || sign_x0) && !sign_x) return HS_ERR_INVALID_ARG;
+    void* scratch = nullptr;
+    st = static_scratch_address(&scratch);
+    if (st != HS_OK) return st;
+    return heinsen_scan_log(log_a, log_b, log_x0, log_x, sign_a, sign_b, sign_x0, sign_x, rows, n, HS_F32, HS_F32, scratch,
+                            kStaticScratchBytes, nullptr);
+}
+
 hs_status heinsen_scan_check_static(void* stream) {
     void* scratch = nullptr;
     hs_status st = static_scratch_address(&scratch);

@@ -28,6 +28,7 @@ EXPORTS = [
     "heinsen_scan_launch_count", "heinsen_scan_strerror",
     "heinsen_scan_log_static", "heinsen_scan_check_static", "heinsen_scan_static_max_elements",
 ]
+SHORT_EXPORTS = ["scan_linear", "scan_log"]  # the six/ten-argument forms of the two calls
 
 
 class HeinsenScanError(RuntimeError):
@@ -74,6 +75,10 @@ def lib() -> ctypes.CDLL:
         L.heinsen_scan_check_static.argtypes = [vp]
         L.heinsen_scan_check_static.restype = ci
         L.heinsen_scan_static_max_elements.restype = sz
+        L.scan_linear.argtypes = [vp, vp, vp, vp, i64, i64]
+        L.scan_linear.restype = ci
+        L.scan_log.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i64, i64]
+        L.scan_log.restype = ci
         L.heinsen_scan_strerror.argtypes = [ci]
         L.heinsen_scan_strerror.restype = ctypes.c_char_p
         _lib = L

@@ -20,7 +20,7 @@ def lib():
 def declared_functions():
     text = open(os.path.join(ROOT, "include", "heinsen_scan.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(heinsen_scan_\w+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(heinsen_scan_\w+|scan_linear|scan_log)\s*\(", text)))
 
 
 def test_every_declared_symbol_is_exported(lib):
@@ -29,7 +29,7 @@ def test_every_declared_symbol_is_exported(lib):
     assert len(names) >= 12
     for name in names:
         assert hasattr(lib, name), f"{name} is declared in the header but not exported"
-    assert sorted(heinsen_scan.EXPORTS) == names, "the Python binding's export list and the header disagree"
+    assert sorted(heinsen_scan.EXPORTS + heinsen_scan.SHORT_EXPORTS) == names, "binding export list and header disagree"
 
 
 def test_host_side_validation_needs_no_gpu(lib):
@@ -54,6 +54,8 @@ def test_host_side_validation_needs_no_gpu(lib):
     aligned = (p + 255) & ~255
     assert lib.heinsen_scan_log(p, p, p, p, None, None, None, None, 2, 8, 0, 0, aligned, 16, None) == TOO_SMALL
     assert lib.heinsen_scan_log_static(p, p, p, p, 1 << 20, 4096, None) == TOO_SMALL
+    assert lib.scan_linear(None, p, p, p, 2, 8) == INVALID and lib.scan_linear(p, p, p, p, 0, 8) == OK
+    assert lib.scan_log(p, p, p, p, p, None, None, None, 2, 8) == INVALID and lib.scan_log(p, p, p, p, None, None, None, None, 2, 0) == OK
     assert lib.heinsen_scan_set_path(7) == INVALID and lib.heinsen_scan_set_path(0) == OK
 
 

@@ -325,6 +325,26 @@ def test_host_buffer_entry_point(hs, oracle):
     assert_log_close(out.double().numpy(), ref, tol_positive(t["log_a"].astype(np.float64), ref), "host entry")
 
 
+def test_short_forms_of_the_two_calls(hs, oracle):
+    """scan_linear(a, b, x0, x, rows, n) and scan_log(..., rows, n): fp32, default stream, library scratch."""
+    L = hs.lib()
+    w = workloads.make(4, rows=1300, n=1024)
+    a, b, x0 = (to_dev(w.tensors[k]) for k in ("a", "b", "x0"))
+    x = torch.empty_like(a)
+    torch.cuda.synchronize()
+    assert L.scan_linear(a.data_ptr(), b.data_ptr(), x0.data_ptr(), x.data_ptr(), 1300, 1024) == 0
+    hs.check_static("cuda")
+    assert_signed_close(to_f64(x), oracle.scan_linear(w.tensors["a"], w.tensors["b"], w.tensors["x0"]), "scan_linear short form")
+    w = workloads.make(3, rows=1, n=1 << 20)
+    la, lb, lx0 = (to_dev(w.tensors[k]) for k in ("log_a", "log_b", "log_x0"))
+    out = torch.empty_like(la)
+    torch.cuda.synchronize()
+    assert L.scan_log(la.data_ptr(), lb.data_ptr(), lx0.data_ptr(), out.data_ptr(), None, None, None, None, 1, 1 << 20) == 0
+    hs.check_static("cuda")
+    ref, _ = oracle.scan_log(w.tensors["log_a"], w.tensors["log_b"], w.tensors["log_x0"])
+    assert_log_close(to_f64(out), ref, tol_positive(w.tensors["log_a"].astype(np.float64), ref), "scan_log short form")
+
+
 def test_repeatability(hs):
     w = workloads.make(3, rows=1, n=1 << 21)
     la, lb, lx0 = (to_dev(w.tensors[k]) for k in ("log_a", "log_b", "log_x0"))
