@@ -325,6 +325,20 @@ def test_host_buffer_entry_point(hs, oracle):
     assert_log_close(out.double().numpy(), ref, tol_positive(t["log_a"].astype(np.float64), ref), "host entry")
 
 
+def test_lookback_several_rows_several_groups(hs, oracle):
+    """Look-back path with a few rows, each several descriptor groups long (a group is one wave of tiles),
+    plus a ragged last tile: exercises group aggregates, group values and the row start inside a launch."""
+    rows, n = 3, 2_650_112 + 40
+    w = workloads.make(3, rows=rows, n=n)
+    t = w.tensors
+    hs.set_path(hs.PATH_LOOKBACK)
+    ws = hs.new_workspace(rows, n, "cuda")
+    out = hs.scan_log(to_dev(t["log_a"]), to_dev(t["log_b"]), to_dev(t["log_x0"]), workspace=ws)
+    hs.check(ws)
+    ref, _ = oracle.scan_log(t["log_a"], t["log_b"], t["log_x0"])
+    assert_log_close(to_f64(out), ref, tol_positive(t["log_a"].astype(np.float64), ref), "3 rows x 2.65M")
+
+
 def test_short_forms_of_the_two_calls(hs, oracle):
     """scan_linear(a, b, x0, x, rows, n) and scan_log(..., rows, n): fp32, default stream, library scratch."""
     L = hs.lib()
