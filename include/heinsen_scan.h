@@ -182,6 +182,23 @@ hs_status heinsen_scan_check_static(void* stream);
 size_t heinsen_scan_static_max_elements(void);
 
 /*
+ * Complex-logarithm form of heinsen_scan_log (Summary, last paragraph: with negative a_t, b_t
+ * or x_0 the interim logarithms are complex while x_t stays real).  Every value is one complex64
+ * (interleaved float pairs): real part log|v|, imaginary part an integer multiple of pi, odd for
+ * a negative v (principal branch: log(-r) = log r + i*pi); log 0 = (-inf, anything).
+ *   log_a, log_b : device, [rows,n] complex64;  log_x0: device, [rows] complex64.
+ *   log_x        : device, [rows,n] complex64 = (log|x_t|, 0 or pi); an exact zero is (-inf, 0).
+ *   workspace    : device, at least heinsen_scan_complex_workspace_bytes(rows, n) bytes,
+ *                  256-byte aligned (15 bytes per element: the values are split into the
+ *                  magnitude and sign planes of the sign+magnitude kernels, scanned there, and
+ *                  joined again; the scan itself is the same single-pass kernel).
+ * Device-side errors: heinsen_scan_check(workspace, stream).
+ */
+hs_status heinsen_scan_log_complex(const void* log_a, const void* log_b, const void* log_x0, void* log_x,
+                                   int64_t rows, int64_t n, void* workspace, size_t workspace_bytes, void* stream);
+size_t heinsen_scan_complex_workspace_bytes(int64_t rows, int64_t n);
+
+/*
  * The two calls in their shortest form: fp32 storage, legacy default stream, automatic kernel
  * selection, scratch from the library's fixed 1 MiB array (the rules of heinsen_scan_log_static
  * apply: problems whose look-back descriptors do not fit return HS_ERR_WORKSPACE_TOO_SMALL; calls

@@ -397,6 +397,50 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
     return HS_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Complex-logarithm interface (Summary, last paragraph: the logarithm of a negative value is
+// complex, log r + i*pi on the principal branch).  Values arrive and leave as complex64; the
+// imaginary part divided by pi, modulo 2, is the sign bit of the sign+magnitude kernels.
+constexpr float kPi = 3.14159265358979323846f;
+
+__global__ void __launch_bounds__(256) split_complex_kernel(const float2* __restrict__ z, float* __restrict__ mag,
+                                                            uint8_t* __restrict__ sign, long long count) {
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += stride) {
+        const float2 v = z[i];
+        mag[i] = v.x;
+        sign[i] = (uint8_t)(__float2int_rn(v.y * (1.0f / kPi)) & 1);
+    }
+}
+__global__ void __launch_bounds__(256) join_complex_kernel(const float* __restrict__ mag, const uint8_t* __restrict__ sign,
+                                                           float2* __restrict__ z, long long count) {
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += stride) {
+        z[i] = make_float2(mag[i], (sign[i] & 1) ? kPi : 0.0f);
+    }
+}
+
+struct ComplexLayout {
+    size_t ws, mag_a, mag_b, mag_x, sign_a, sign_b, sign_x, mag_x0, sign_x0, total;
+};
+ComplexLayout complex_layout(long long rows, long long n) {
+    auto up = [](size_t v) { return (v + 255) & ~size_t(255); };
+    const size_t cnt = (size_t)rows * (size_t)n;
+    ComplexLayout L;
+    size_t o = 0;
+    L.ws = o;      o += up(workspace_bytes_for(rows, n));
+    L.mag_a = o;   o += up(cnt * 4);
+    L.mag_b = o;   o += up(cnt * 4);
+    L.mag_x = o;   o += up(cnt * 4);
+    L.sign_a = o;  o += up(cnt);
+    L.sign_b = o;  o += up(cnt);
+    L.sign_x = o;  o += up(cnt);
+    L.mag_x0 = o;  o += up((size_t)rows * 4);
+    L.sign_x0 = o; o += up((size_t)rows);
+    L.total = o;
+    return L;
+}
+
 // Scratch of heinsen_scan_log_static(): lives in the library image, so every GPU that loads the
 // library holds these bytes until the process exits.  In host code `g_static_scratch` is only a
 // handle for the runtime; the device address comes from cudaGetSymbolAddress().
@@ -480,6 +524,46 @@ hs_status heinsen_scan_log_static(const void* log_a, const void* log_b, const vo
     // run() clears the descriptors it is about to use (cudaMemsetAsync on `stream`), so what the
     // previous call left in the array does not matter
     return run(pr, scratch, kStaticScratchBytes, static_cast<cudaStream_t>(stream), HS_PATH_LOOKBACK);
+}
+
+size_t heinsen_scan_complex_workspace_bytes(int64_t rows, int64_t n) {
+    if (rows <= 0 || n <= 0 || rows > 0x7fffffffll || n > kMaxN || rows > (1ll << 62) / n) return 0;
+    return complex_layout(rows, n).total;
+}
+
+hs_status heinsen_scan_log_complex(const void* log_a, const void* log_b, const void* log_x0, void* log_x, int64_t rows,
+                                   int64_t n, void* workspace, size_t workspace_bytes, void* stream) {
+    hs_status st = validate_common(log_a, log_b, log_x0, log_x, rows, n);
+    if (st != HS_OK || rows == 0 || n == 0) return st;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HS_ERR_INVALID_ARG;
+    const ComplexLayout L = complex_layout(rows, n);
+    if (workspace_bytes < L.total) return HS_ERR_WORKSPACE_TOO_SMALL;
+    DeviceInfo dev;
+    st = device_info(dev);
+    if (st != HS_OK) return st;
+    if (dev.cc_major != 10) return HS_ERR_UNSUPPORTED_DEVICE;
+    uint8_t* w = static_cast<uint8_t*>(workspace);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const long long cnt = (long long)rows * n;
+    auto blocks = [&](long long c) { long long b = (c + 255) / 256; return (int)(b < 8LL * dev.sm_count ? b : 8LL * dev.sm_count); };
+    split_complex_kernel<<<blocks(cnt), 256, 0, s>>>(static_cast<const float2*>(log_a), reinterpret_cast<float*>(w + L.mag_a),
+                                                     w + L.sign_a, cnt);
+    split_complex_kernel<<<blocks(cnt), 256, 0, s>>>(static_cast<const float2*>(log_b), reinterpret_cast<float*>(w + L.mag_b),
+                                                     w + L.sign_b, cnt);
+    split_complex_kernel<<<blocks(rows), 256, 0, s>>>(static_cast<const float2*>(log_x0), reinterpret_cast<float*>(w + L.mag_x0),
+                                                      w + L.sign_x0, rows);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail("split_complex_kernel", e);
+    g_launches.fetch_add(3);
+    st = heinsen_scan_log(w + L.mag_a, w + L.mag_b, w + L.mag_x0, w + L.mag_x, w + L.sign_a, w + L.sign_b, w + L.sign_x0,
+                          w + L.sign_x, rows, n, HS_F32, HS_F32, w + L.ws, workspace_bytes_for(rows, n), stream);
+    if (st != HS_OK) return st;
+    join_complex_kernel<<<blocks(cnt), 256, 0, s>>>(reinterpret_cast<const float*>(w + L.mag_x), w + L.sign_x,
+                                                    static_cast<float2*>(log_x), cnt);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail("join_complex_kernel", e);
+    g_launches.fetch_add(1);
+    return HS_OK;
 }
 
 hs_status scan_linear(const void* a, const void* b, const void* x0, void* x, int64_t rows, int64_t n) {

@@ -27,6 +27,7 @@ EXPORTS = [
     "heinsen_scan_set_path", "heinsen_scan_debug_config", "heinsen_scan_last_path",
     "heinsen_scan_launch_count", "heinsen_scan_strerror",
     "heinsen_scan_log_static", "heinsen_scan_check_static", "heinsen_scan_static_max_elements",
+    "heinsen_scan_log_complex", "heinsen_scan_complex_workspace_bytes",
 ]
 SHORT_EXPORTS = ["scan_linear", "scan_log"]  # the six/ten-argument forms of the two calls
 
@@ -75,6 +76,10 @@ def lib() -> ctypes.CDLL:
         L.heinsen_scan_check_static.argtypes = [vp]
         L.heinsen_scan_check_static.restype = ci
         L.heinsen_scan_static_max_elements.restype = sz
+        L.heinsen_scan_log_complex.argtypes = [vp, vp, vp, vp, i64, i64, vp, sz, vp]
+        L.heinsen_scan_log_complex.restype = ci
+        L.heinsen_scan_complex_workspace_bytes.argtypes = [i64, i64]
+        L.heinsen_scan_complex_workspace_bytes.restype = sz
         L.scan_linear.argtypes = [vp, vp, vp, vp, i64, i64]
         L.scan_linear.restype = ci
         L.scan_log.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i64, i64]
@@ -254,6 +259,27 @@ def check_static(device):
 
 def static_max_elements() -> int:
     return int(lib().heinsen_scan_static_max_elements())
+
+
+def scan_log_complex(log_a: torch.Tensor, log_b: torch.Tensor, log_x0: torch.Tensor,
+                     log_x: torch.Tensor | None = None, workspace: torch.Tensor | None = None) -> torch.Tensor:
+    """heinsen_scan_log_complex: complex64 tensors (log|v| + i*k*pi, k odd for negative v) in and out.  Asynchronous."""
+    rows, n = log_a.shape
+    _require(log_a, (rows, n), "log_a"); _require(log_b, (rows, n), "log_b"); _require(log_x0, (rows,), "log_x0")
+    if not (log_a.dtype == log_b.dtype == log_x0.dtype == torch.complex64):
+        raise TypeError("scan_log_complex takes complex64 tensors")
+    if log_x is None:
+        log_x = torch.empty_like(log_a)
+    _require(log_x, (rows, n), "log_x")
+    if rows == 0 or n == 0:
+        return log_x
+    if workspace is None:
+        workspace = torch.empty(int(lib().heinsen_scan_complex_workspace_bytes(rows, n)), dtype=torch.uint8,
+                                device=log_a.device)
+    with _on_device(log_a.device):
+        _check(lib().heinsen_scan_log_complex(_ptr(log_a), _ptr(log_b), _ptr(log_x0), _ptr(log_x), rows, n,
+                                              _ptr(workspace), workspace.numel(), _stream_ptr(log_a.device)))
+    return log_x
 
 
 def host_scratch_bytes(rows: int, n: int, dtype_in: torch.dtype, dtype_out: torch.dtype, with_signs: bool) -> int:

@@ -54,6 +54,9 @@ def test_host_side_validation_needs_no_gpu(lib):
     aligned = (p + 255) & ~255
     assert lib.heinsen_scan_log(p, p, p, p, None, None, None, None, 2, 8, 0, 0, aligned, 16, None) == TOO_SMALL
     assert lib.heinsen_scan_log_static(p, p, p, p, 1 << 20, 4096, None) == TOO_SMALL
+    assert lib.heinsen_scan_log_complex(None, p, p, p, 2, 8, aligned, 1 << 20, None) == INVALID
+    assert lib.heinsen_scan_log_complex(p, p, p, p, 2, 8, aligned, 64, None) == TOO_SMALL
+    assert lib.heinsen_scan_complex_workspace_bytes(2, 8) >= 256 + 15 * 16
     assert lib.scan_linear(None, p, p, p, 2, 8) == INVALID and lib.scan_linear(p, p, p, p, 0, 8) == OK
     assert lib.scan_log(p, p, p, p, p, None, None, None, 2, 8) == INVALID and lib.scan_log(p, p, p, p, None, None, None, None, 2, 0) == OK
     assert lib.heinsen_scan_set_path(7) == INVALID and lib.heinsen_scan_set_path(0) == OK

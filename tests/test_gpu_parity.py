@@ -339,6 +339,25 @@ def test_lookback_several_rows_several_groups(hs, oracle):
     assert_log_close(to_f64(out), ref, tol_positive(t["log_a"].astype(np.float64), ref), "3 rows x 2.65M")
 
 
+@pytest.mark.parametrize("path", ["batched", "lookback"])
+def test_complex_logarithm_interface(hs, oracle, path):
+    """Negative a, b, x0 as complex logarithms (log r + i*pi): the result is real, i.e. its imaginary part is
+    0 or pi, and exp of it equals the recurrence in the linear domain."""
+    w = workloads.make(4, rows=40, n=3000)
+    a, b, x0 = (w.tensors[k].astype(np.float64) for k in ("a", "b", "x0"))
+    with np.errstate(divide="ignore"):
+        la, lb, lx0 = (np.log(v.astype(np.complex128)).astype(np.complex64) for v in (a, b, x0))
+    la.imag[::3] += np.float32(2 * np.pi)         # any odd/even multiple of pi is the same sign
+    lb.imag[1::5] -= np.float32(2 * np.pi)
+    hs.set_path(getattr(hs, "PATH_" + path.upper()))
+    out = hs.scan_log_complex(*(torch.from_numpy(v).cuda() for v in (la, lb, lx0)))
+    z = out.cpu().numpy()
+    assert np.isin(np.round(z.imag / np.pi), (0, 1)).all() and np.allclose(z.imag, np.round(z.imag / np.pi) * np.pi, atol=1e-6)
+    got = np.exp(z.real.astype(np.float64)) * np.where(np.round(z.imag / np.pi) == 1, -1.0, 1.0)
+    ref = oracle.scan_linear(w.tensors["a"], w.tensors["b"], w.tensors["x0"])
+    assert_signed_close(got, ref, f"complex interface/{path}")
+
+
 def test_short_forms_of_the_two_calls(hs, oracle):
     """scan_linear(a, b, x0, x, rows, n) and scan_log(..., rows, n): fp32, default stream, library scratch."""
     L = hs.lib()
