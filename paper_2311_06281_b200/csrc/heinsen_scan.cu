@@ -283,7 +283,6 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
     p.call_id = next_call_id();
     p.spin_limit = g_spin_limit.load();
     p.mute_tile = g_mute_tile.load();
-    p.debug_flags = env_int("HEINSEN_SCAN_DEBUG_FLAGS", 0, 0, 255);
     p.ws = reinterpret_cast<Header*>(workspace);
 
     int warps, stages, grid, lb_smem = 0;

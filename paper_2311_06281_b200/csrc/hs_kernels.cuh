@@ -66,7 +66,6 @@ struct Params {
     unsigned int lb_sleep_ready;  // ns between polls afterwards
     unsigned int spin_limit;    // bound on polls of predecessor flags
     long long mute_tile;        // test hook: this tile never publishes (-1: none)
-    int debug_flags;            // timing experiments only (results are wrong when non-zero)
 };
 
 // The first thread to report an error in this call records it; heinsen_scan_check() reports it
@@ -668,7 +667,7 @@ struct Lookback {
     __device__ static __forceinline__ E run(const Params& p, long long T, int j, long long row, int lane,
                                             uint32_t agg_bar, uint32_t agg_parity, const float4* total_src,
                                             const volatile int* abort_flag, bool& failed,
-                                            unsigned int& total_polls, unsigned long long* stamps = nullptr) {
+                                            unsigned int& total_polls) {
         failed = false;
         const int gsz = p.lb_group;
         const int g = j / gsz, k = j - g * gsz;                    // group, position in group
@@ -686,11 +685,10 @@ struct Lookback {
         for (int q = 0; q < kLbPerLane; ++q) { td[q].lo = 0ull; td[q].hi = 0ull; }
         Desc gd;
         gd.lo = 0ull; gd.hi = 0ull;
-        bool own_ready = false, tiles_done = (k == 0), groups_done = (p.debug_flags & 1) != 0, group_agg_sent = false;
+        bool own_ready = false, tiles_done = (k == 0), groups_done = false, group_agg_sent = false;
         E tile_total = identity_elem<SIGNED>();
         E before_in_group = identity_elem<SIGNED>();
-        E acc = (p.debug_flags & 1) ? x0e : identity_elem<SIGNED>();
-        if (p.debug_flags & 1) tiles_done = true;
+        E acc = identity_elem<SIGNED>();
         int gwin = 1;  // distance of the nearest group of the current group window
         while (true) {
             if (!tiles_done) {
@@ -706,7 +704,6 @@ struct Lookback {
 
             if (!own_ready && mbar_test(agg_bar, agg_parity)) {
                 own_ready = true;
-                if (stamps) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(stamps[2]));
                 tile_total = unpack_elem<SIGNED>(*total_src);  // scanned and published by the compute warps
             }
             if (!tiles_done) {
@@ -725,7 +722,6 @@ struct Lookback {
                     }
                     before_in_group = reduce_newest_first(part, lane);
                     tiles_done = true;
-                    if (stamps) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(stamps[0]));
                 }
             }
             if (own_ready && tiles_done && full_group && publish && !group_agg_sent) {
@@ -745,7 +741,6 @@ struct Lookback {
                     acc = compose(reduce_newest_first(gp, lane), acc);
                     if (inc_mask) {
                         groups_done = true;
-                        if (stamps) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(stamps[1]));
                     } else gwin += 32;  // every group of this window is an aggregate: look further back
                 }
             }
@@ -910,25 +905,15 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
             const int j = cur.j;
             const int b = (int)(i % kLbRing);
             bool failed = false;
-            unsigned long long stamps[3] = {0, 0, 0}, t_start = 0;
             unsigned int npolls = 0;
-            if (p.debug_flags & 2) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_start));
             const E carry = LB::run(p, T, j, row, lane, total_bar + 8 * b, (uint32_t)((i / kLbRing) & 1), &xc->total[b],
-                                    &xc->abort, failed, npolls, (p.debug_flags & 2) ? stamps : nullptr);
+                                    &xc->abort, failed, npolls);
             if (lane == 0) {
                 if (failed) {
                     record_error(p, kErrLookbackTimeout, T);
                     xc->abort = 1;
                 }
                 xc->carry[b] = make_float4(carry.m, carry.s, 0.0f, 0.0f);
-            }
-            if ((p.debug_flags & 2) && lane == 0) {
-                unsigned long long t_done;
-                asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_done));
-                const unsigned long long t_agg = stamps[2];
-                auto d16 = [&](unsigned long long t) { return (unsigned long long)(t > t_agg ? ((t - t_agg) >> 5) & 0xffff : 0); };
-                reinterpret_cast<ulonglong2*>(p.gdesc + p.rows * p.groups_per_row)[T] =
-                    make_ulonglong2(t_agg, d16(t_start) | (d16(stamps[0]) << 16) | (d16(stamps[1]) << 32) | (d16(t_done) << 48));
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(carry_bar + 8 * b);  // releases wexcl, carry and abort to the CTA
@@ -1048,14 +1033,7 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
             const long long row = c2.row;
             const int colbase = colbase_of(c2);
             const int st = st2, b = b2;
-            unsigned long long tw0 = 0;
-            if ((p.debug_flags & 2) && warp == 0 && lane == 0) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tw0));
             const bool carry_ok = mbar_wait_bounded(carry_bar + 8 * b, parb2, kCopySpinLimit);
-            if ((p.debug_flags & 2) && warp == 0 && lane == 0) {
-                unsigned long long tw1;
-                asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tw1));
-                reinterpret_cast<ulonglong2*>(p.gdesc + p.rows * p.groups_per_row)[p.num_tiles + c2.T] = make_ulonglong2(tw0, tw1 - tw0);
-            }
             if (!carry_ok) {
                 if (lane == 0) { record_error(p, kErrLookbackTimeout, c2.T); xc->abort = 1; }
                 aborted = true;
