@@ -47,9 +47,11 @@ def parse_args():
     ap.add_argument("--fig1", action="store_true",
                     help="the paper's only experiment: sequential (CPU oracle, one core) over parallel (this library) "
                          "time for one sequence of n = 2^10..2^28 elements, means of 30 runs; prints one JSON object")
-    ap.add_argument("--ablation", default=None, choices=["unfused"],
+    ap.add_argument("--ablation", default=None, choices=["unfused", "pairs"],
                     help="'unfused': the paper's own recipe (Eq. 7) as separate framework kernels -- torch.cumsum, "
-                         "torch.logcumsumexp and elementwise ops, one pass over memory each -- on the same workload")
+                         "torch.logcumsumexp and elementwise ops, one pass over memory each -- on the same workload; "
+                         "'pairs': the linear-domain (alpha, beta) pair scan (no logarithms) beside the log-space "
+                         "scan_linear on the signed linear workload (cfg4)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -427,10 +429,63 @@ def run_unfused(args):
     }), flush=True)
 
 
+def run_pairs(args):
+    """Comparison: the linear-domain pair scan (no logarithms) beside the log-space heinsen_scan_linear on the
+    same signed linear workload (cfg4 unless --rows/--n say otherwise), three rotating buffer sets."""
+    import numpy as np
+    import torch
+
+    from oracle import heinsen_oracle
+    from paper_2311_06281_b200 import heinsen_scan as hs
+    from paper_2311_06281_b200 import workloads
+
+    cid = 4
+    w = workloads.make(cid, rows=args.rows, n=args.n)
+    dev = torch.device("cuda", 0)
+    t = w.tensors
+    sets = [[torch.from_numpy(t[k]).to(dev) for k in ("a", "b", "x0")] for _ in range(3)]
+    outs = [torch.empty_like(s[0]) for s in sets]
+    wss = [hs.new_workspace(w.rows, w.n, dev) for _ in sets]
+    elements = w.rows * w.n
+    rows = list(range(min(w.rows, 64)))
+    ref = heinsen_oracle.scan_linear(t["a"][rows], t["b"][rows], t["x0"][rows])
+    result = {}
+    for name, fn in (("pairs", hs.scan_linear_pairs), ("log_space", hs.scan_linear)):
+        def step(i):
+            k = i % 3
+            fn(*sets[k], x=outs[k], workspace=wss[k])
+        for i in range(max(args.warmup, 3)):
+            step(i)
+        torch.cuda.synchronize()
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        start.record()
+        for i in range(args.steps):
+            step(i)
+        stop.record()
+        torch.cuda.synchronize()
+        for ws in wss:
+            hs.check(ws)
+        ms = start.elapsed_time(stop) / args.steps
+        got = outs[0][rows].double().cpu().numpy()
+        err = np.abs(got - ref) / (1e-3 * np.abs(ref).max(axis=1, keepdims=True))
+        result[name] = {"ms_per_step": ms, "value": elements / (ms * 1e-3), "algorithmic_GBs": elements * 12 / (ms * 1e-3) / 1e9,
+                        "max_err_over_tolerance": float(err.max())}
+    peak, _ = measured_peak()
+    print(json.dumps({
+        "ablation": "pairs", "metric": METRIC, "unit": UNIT, "value": result["pairs"]["value"],
+        "ms_per_step": result["pairs"]["ms_per_step"], "steps": args.steps,
+        "config": {"workload": workload_name(cid, w)}, "pairs": result["pairs"], "log_space": result["log_space"],
+        "frac_of_measured_hbm": {k: v["algorithmic_GBs"] / peak for k, v in result.items()},
+    }), flush=True)
+
+
 def main():
     args = parse_args()
     if args.ablation == "unfused":
         run_unfused(args)
+        return
+    if args.ablation == "pairs":
+        run_pairs(args)
         return
     if args.fig1:
         run_fig1(args)

@@ -92,6 +92,22 @@ hs_status heinsen_scan_linear(const void* a, const void* b, const void* x0, void
                               void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Comparison path, NOT the paper's method: the same recurrence scanned in the linear
+ * domain as pairs (alpha, beta) = "x -> alpha x + beta" combined by
+ * (alpha2 alpha1, alpha2 beta1 + beta2), i.e. the general two-operator formulation that
+ * the section "Compared to Blelloch's Formulation" sets the log-space expression
+ * against.  No logarithm or exponential is taken, so every prefix product and partial
+ * sum must fit fp32's own range: a product of |a| over one part that overflows gives
+ * inf/NaN, one that underflows drops what the log-space entry points still carry.
+ * Arguments, layout, workspace and errors as for heinsen_scan_linear (HS_F32 only).
+ * Always runs the row-batched kernel (one warp per row or per few rows); it is meant
+ * for batches of rows and is slow for a single long row.
+ */
+hs_status heinsen_scan_linear_pairs(const void* a, const void* b, const void* x0, void* x,
+                                    int64_t rows, int64_t n, hs_dtype dtype,
+                                    void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Log-domain entry point: Eq. 7 as printed, on log inputs, returning log x.
  *   log_x[r,t] = a*_t + logaddexp(log_x0[r], logcumsumexp(log_b - a*)_t),  a* = cumsum(log_a)
  * with an optional sign bit per value (sign + magnitude of a negative real).

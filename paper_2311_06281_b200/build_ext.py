@@ -9,7 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libheinsen_scan.so")
 SOURCES = ["heinsen_scan.cu"]
-HEADERS = ["hs_device.cuh", "hs_kernels.cuh", os.path.join("..", "..", "include", "heinsen_scan.h")]
+HEADERS = ["hs_device.cuh", "hs_kernels.cuh", "hs_pairs.cuh", os.path.join("..", "..", "include", "heinsen_scan.h")]
 NVCC_FLAGS = ["-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-shared", "-Xcompiler", "-fPIC"]
 

@@ -158,6 +158,20 @@ KernelEntry entry() {
     return e;
 }
 
+// Modes that exist for the row-batched kernel only.
+template <int MODE, typename TIn, typename TOut, int K, bool TMA>
+KernelEntry entry_batched_only() {
+    KernelEntry e;
+    e.batched = reinterpret_cast<const void*>(&batched_scan_kernel<MODE, TIn, TOut, K, TMA>);
+    e.lookback = nullptr;
+    e.lb_K = K;
+    e.K = K;
+    e.warp_smem_per_stage = 2 * 32 * K * (int)sizeof(TIn);
+    e.warp_smem_out = 2 * 32 * K * (int)sizeof(TOut);
+    e.lb_smem = nullptr;
+    return e;
+}
+
 bool find_kernel(int mode, hs_dtype din, hs_dtype dout, bool tma, KernelEntry& e) {
 #define HS_PICK(M, TI, TO, KK)                                               \
     do {                                                                     \
@@ -167,6 +181,14 @@ bool find_kernel(int mode, hs_dtype din, hs_dtype dout, bool tma, KernelEntry& e
     using bf16 = __nv_bfloat16;
     if (mode == kLinear) {
         if (din == HS_F32 && dout == HS_F32) HS_PICK(kLinear, float, float, 16);
+        return false;
+    }
+    if (mode == kPairs) {
+        if (din == HS_F32 && dout == HS_F32) {
+            e = tma ? entry_batched_only<kPairs, float, float, 16, true>()
+                    : entry_batched_only<kPairs, float, float, 16, false>();
+            return true;
+        }
         return false;
     }
     if (mode == kLogUnsigned) {
@@ -482,6 +504,20 @@ hs_status heinsen_scan_linear(const void* a, const void* b, const void* x0, void
     pr.p.in_a = a; pr.p.in_b = b; pr.p.x0 = x0; pr.p.out = x;
     pr.p.rows = rows; pr.p.n = n;
     return run(pr, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
+}
+
+hs_status heinsen_scan_linear_pairs(const void* a, const void* b, const void* x0, void* x, int64_t rows, int64_t n,
+                                    hs_dtype dtype, void* workspace, size_t workspace_bytes, void* stream) {
+    hs_status st = validate_common(a, b, x0, x, rows, n);
+    if (st != HS_OK || rows == 0 || n == 0) return st;
+    if (dtype != HS_F32) return HS_ERR_INVALID_ARG;
+    Problem pr;
+    std::memset(&pr, 0, sizeof pr);
+    pr.mode = kPairs;
+    pr.din = pr.dout = dtype;
+    pr.p.in_a = a; pr.p.in_b = b; pr.p.x0 = x0; pr.p.out = x;
+    pr.p.rows = rows; pr.p.n = n;
+    return run(pr, workspace, workspace_bytes, static_cast<cudaStream_t>(stream), HS_PATH_BATCHED);
 }
 
 hs_status heinsen_scan_log(const void* log_a, const void* log_b, const void* log_x0, void* log_x,

@@ -24,7 +24,7 @@ constexpr uint32_t kSignBit = 0x80000000u;
 // differences of references free of inf - inf without a guard in the inner combine.
 constexpr float kEmpty = -1e20f;
 
-enum Mode : int { kLogUnsigned = 0, kLogSigned = 1, kLinear = 2 };
+enum Mode : int { kLogUnsigned = 0, kLogSigned = 1, kLinear = 2, kPairs = 3 /* linear-domain comparison path */ };
 
 __device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000); }
 

@@ -313,6 +313,10 @@ struct ChunkEngine {
     }
 };
 
+}  // namespace hs
+#include "hs_pairs.cuh"
+namespace hs {
+
 __device__ __forceinline__ uint8_t* align_1024(uint8_t* p) {
     return reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(p) + 1023) & ~uintptr_t(1023));
 }
@@ -454,7 +458,9 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
 
     // All hot-loop indices are 32-bit and advance incrementally (rows < 2^31; with TMA also n < 2^31);
     // 64-bit products appear once per row only.
-    const int gw = blockIdx.x * nwarps + warp;
+    // Warp slots are numbered CTA-fastest, so that a last, partly filled round of row groups spreads
+    // over all SMs instead of loading the first CTAs only.
+    const int gw = warp * (int)gridDim.x + (int)blockIdx.x;
     const int GW = gridDim.x * nwarps;
     const int groups = (int)((p.rows + R - 1) / R);
     if (gw >= groups) return;

@@ -28,6 +28,7 @@ EXPORTS = [
     "heinsen_scan_launch_count", "heinsen_scan_strerror",
     "heinsen_scan_log_static", "heinsen_scan_check_static", "heinsen_scan_static_max_elements",
     "heinsen_scan_log_complex", "heinsen_scan_complex_workspace_bytes",
+    "heinsen_scan_linear_pairs",
 ]
 SHORT_EXPORTS = ["scan_linear", "scan_log"]  # the six/ten-argument forms of the two calls
 
@@ -53,6 +54,8 @@ def lib() -> ctypes.CDLL:
         vp, i64, ci, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_size_t
         L.heinsen_scan_linear.argtypes = [vp, vp, vp, vp, i64, i64, ci, vp, sz, vp]
         L.heinsen_scan_linear.restype = ci
+        L.heinsen_scan_linear_pairs.argtypes = [vp, vp, vp, vp, i64, i64, ci, vp, sz, vp]
+        L.heinsen_scan_linear_pairs.restype = ci
         L.heinsen_scan_log.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i64, i64, ci, ci, vp, sz, vp]
         L.heinsen_scan_log.restype = ci
         L.heinsen_scan_workspace_bytes.argtypes = [i64, i64]
@@ -192,6 +195,27 @@ def scan_linear(a: torch.Tensor, b: torch.Tensor, x0: torch.Tensor, x: torch.Ten
     with _on_device(a.device):
         _check(lib().heinsen_scan_linear(_ptr(a), _ptr(b), _ptr(x0), _ptr(x), rows, n, _dtype_code(a),
                                          _ptr(workspace), workspace.numel(), _stream_ptr(a.device)))
+    return x
+
+
+def scan_linear_pairs(a: torch.Tensor, b: torch.Tensor, x0: torch.Tensor, x: torch.Tensor | None = None,
+                      workspace: torch.Tensor | None = None) -> torch.Tensor:
+    """Comparison path: the same recurrence scanned in the linear domain as (alpha, beta) pairs, no logarithms.
+    Arguments as for scan_linear.  Asynchronous."""
+    rows, n = a.shape
+    _require(a, (rows, n), "a"); _require(b, (rows, n), "b"); _require(x0, (rows,), "x0")
+    if x is None:
+        x = torch.empty_like(a)
+    _require(x, (rows, n), "x")
+    if not (a.dtype == b.dtype == x0.dtype == x.dtype):
+        raise TypeError("a, b, x0, x must share one dtype")
+    if rows == 0 or n == 0:
+        return x
+    if workspace is None:
+        workspace = new_workspace(rows, n, a.device)
+    with _on_device(a.device):
+        _check(lib().heinsen_scan_linear_pairs(_ptr(a), _ptr(b), _ptr(x0), _ptr(x), rows, n, _dtype_code(a),
+                                               _ptr(workspace), workspace.numel(), _stream_ptr(a.device)))
     return x
 
 
