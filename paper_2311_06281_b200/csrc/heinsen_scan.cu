@@ -347,8 +347,14 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         warps = W + nlb + 1;  // + the publisher warp
         p.tiles_per_row = (int)lookback_tiles_per_row(p.n, chunk, W);
         p.num_tiles = p.rows * p.tiles_per_row;
-        // group = the tiles one wave of CTAs processes (the grid is sm_count CTAs: one per SM)
-        p.lb_group = dev.sm_count < kLbMaxGroup ? dev.sm_count : kLbMaxGroup;
+        // group = a little less than the tiles one wave of CTAs processes (the grid is sm_count CTAs, one
+        // per SM).  With exactly one wave per group the group's last tile always sits on the last CTA and
+        // the group closes only after the slowest CTA of the wave; 11/12 of a wave lets the closing position
+        // move through the CTAs and the bulk of a wave close before its stragglers (measured on cfg3:
+        // 148 tiles per group 157 us, 136: 149 us, 128: 150 us, 112: 154 us, 74: 154 us).
+        p.lb_group = dev.sm_count - dev.sm_count / 12;
+        if (p.lb_group > kLbMaxGroup) p.lb_group = kLbMaxGroup;
+        if (p.lb_group < 2) p.lb_group = 2;
         p.lb_group = env_int("HEINSEN_SCAN_LB_GROUP", p.lb_group, 2, kLbMaxGroup);
         p.groups_per_row = (p.tiles_per_row + p.lb_group - 1) / p.lb_group;
         const size_t need = sizeof(Header) + ((size_t)p.num_tiles + (size_t)p.rows * p.groups_per_row) * 16;
