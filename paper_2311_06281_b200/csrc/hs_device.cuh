@@ -453,6 +453,24 @@ struct Run {
         bad = false;
     }
 
+    // The K parity masks of the run as 16 bits (K == 16), P[t] at bit 16 + t, and back; with adopt() the
+    // look-back kernel carries A_t and the parities of a kLinear run from its first phase to its second
+    // instead of taking the logarithms of a_t twice.
+    __device__ __forceinline__ uint32_t parity_bits() const {
+        uint32_t bits = 0u;
+#pragma unroll
+        for (int t = 0; t < K; ++t) bits = (bits >> 1) | (SIGNED ? P[t] : 0u);
+        return bits;
+    }
+    __device__ __forceinline__ void adopt(const float* a_parked, uint32_t bits) {
+#pragma unroll
+        for (int t = 0; t < K; ++t) {
+            A[t] = a_parked[t];
+            if (SIGNED) P[t] = (bits << (K - 1 - t)) & kSignBit;
+        }
+        bad = false;
+    }
+
     // Apply the value entering the run and produce the K outputs.
     // out_mag: log|x_t| (log modes) or x_t (kLinear);  out_sign: sign masks (kLogSigned).
     // Returns false when an early prefix is too small relative to the run's reference for the

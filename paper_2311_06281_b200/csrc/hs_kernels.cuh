@@ -788,6 +788,7 @@ struct LanePark {
     float r;              // reference of the lane's run
     Elem<SIGNED> excl;    // parts of the chunk before the lane's run
     bool slow;            // the chunk took the tracked form in phase 1 (warp-uniform)
+    uint32_t par;         // kLinear: parity masks of the lane's run (Run::parity_bits)
 };
 
 // One input stage of a compute warp: [a-tensor chunk][b-tensor chunk][park].  The partial sums
@@ -942,7 +943,7 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
     auto st_park = [&](int st) { return wb + st * ST::BYTES + ST::PARK_OFF; };
     LanePark<SIGNED> lp[4];  // lp[d]: the tile that went through phase 1 d iterations ago
 #pragma unroll
-    for (int d = 0; d < 4; ++d) { lp[d].r = neg_inf(); lp[d].excl = identity_elem<SIGNED>(); lp[d].slow = false; }
+    for (int d = 0; d < 4; ++d) { lp[d].r = neg_inf(); lp[d].excl = identity_elem<SIGNED>(); lp[d].slow = false; lp[d].par = 0u; }
     const uint32_t bars = warp_bars + warp * (8 * kLbMaxStages);
 
     // TMA helpers (same box geometry as WarpPipe, buffers laid out per stage here)
@@ -1022,6 +1023,14 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                     const uint32_t pb = st_park(st);
 #pragma unroll
                     for (int jx = 0; jx < K / 4; ++jx) sts128(pb + park_off[jx], Storage<float>::pack(pd.run.s + 4 * jx));
+                    if (MODE == kLinear) {
+                        // ... and A_t over the a-tensor chunk, the parities in a register: phase 2 would
+                        // otherwise take the logarithm of every a_t a second time
+                        const uint32_t ab = st_a(st);
+#pragma unroll
+                        for (int jx = 0; jx < K / 4; ++jx) sts128(ab + park_off[jx], Storage<float>::pack(pd.run.A + 4 * jx));
+                        lp[0].par = pd.run.parity_bits();
+                    }
                 }
                 lp[0].r = pd.run.r;
                 lp[0].excl = pd.excl;
@@ -1062,18 +1071,25 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                 bool ok = false;
                 const bool was_slow = mine.slow;
                 if (!was_slow) {
-                    // rebuild A_t (and the parity of a) from the inputs, fetch the parked s_t, apply
+                    // rebuild A_t (and the parity of a) from the inputs -- kLinear: fetch the parked A_t --,
+                    // fetch the parked s_t, apply
                     float va[K];
                     uint32_t sa[MODE == kLogSigned ? K : 1];
-                    R_::load_a(sm_a, off.in, va);
-                    if (colbase + CHUNK > p.n) {
-#pragma unroll
-                        for (int t = 0; t < K; ++t)
-                            if (t >= left) va[t] = neutral_a<MODE>();
-                    }
-                    if (MODE == kLogSigned) CE::load_signs(p.sign_a, row * p.n + col0, left, p.sign_vec_ok != 0, sa);
                     R_ run;
-                    run.rebuild(va, sa);
+                    if (MODE == kLinear) {
+#pragma unroll
+                        for (int jx = 0; jx < K / 4; ++jx) Storage<float>::unpack(lds128(sm_a + park_off[jx]), va + 4 * jx);
+                        run.adopt(va, mine.par);
+                    } else {
+                        R_::load_a(sm_a, off.in, va);
+                        if (colbase + CHUNK > p.n) {
+#pragma unroll
+                            for (int t = 0; t < K; ++t)
+                                if (t >= left) va[t] = neutral_a<MODE>();
+                        }
+                        if (MODE == kLogSigned) CE::load_signs(p.sign_a, row * p.n + col0, left, p.sign_vec_ok != 0, sa);
+                        run.rebuild(va, sa);
+                    }
                     run.r = mine.r;
 #pragma unroll
                     for (int jx = 0; jx < K / 4; ++jx) Storage<float>::unpack(lds128(pb + park_off[jx]), run.s + 4 * jx);
@@ -1092,6 +1108,10 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                         for (int t = 0; t < K; ++t) {
                             const float v = (t < left) ? Storage<TIn>::load(p.in_b, row * p.n + col0 + t) : neutral_b<MODE>();
                             Storage<TIn>::to_smem(sm_b + chunk_off(1, 0, (uint32_t)((lane * K + t) * sizeof(TIn))), v);
+                            if (MODE == kLinear) {  // A_t replaced the a-tensor chunk as well
+                                const float u = (t < left) ? Storage<TIn>::load(p.in_a, row * p.n + col0 + t) : neutral_a<MODE>();
+                                Storage<TIn>::to_smem(sm_a + chunk_off(1, 0, (uint32_t)((lane * K + t) * sizeof(TIn))), u);
+                            }
                         }
                         __syncwarp();
                     }
