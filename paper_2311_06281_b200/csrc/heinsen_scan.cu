@@ -323,13 +323,17 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         p.rows_per_warp = R;
         p.nchunks = (int)((p.n + (32 / R) * ke.K - 1) / ((32 / R) * ke.K));
         const long long groups = (p.rows + R - 1) / R;
-        stages = tma ? env_int("HEINSEN_SCAN_STAGES", 2, 2, kMaxStages) : 1;
+        stages = tma ? 2 : 1;  // loads run one chunk ahead of the arithmetic (the kernel keeps one row group ahead)
         const int max_warps = 16;
         long long per_sm = (groups + dev.sm_count - 1) / dev.sm_count;
         warps = (int)(per_sm < 1 ? 1 : (per_sm > max_warps ? max_warps : per_sm));
         warps = env_int("HEINSEN_SCAN_WARPS", warps, 1, 16);
         const long long ctas_needed = (groups + warps - 1) / warps;
         grid = (int)(ctas_needed < dev.sm_count ? ctas_needed : dev.sm_count);
+        // tickets balance SMs of unequal speed when every warp slot sees several groups; with fewer, a
+        // greedy hand-out of the last round loses more than it gains (cfg4, 1.7 groups per slot: 81 vs 74 us)
+        p.row_tickets = groups >= 4ll * grid * warps ? 1 : 0;
+        p.row_tickets = env_int("HEINSEN_SCAN_ROW_TICKETS", p.row_tickets, 0, 1);
         fn = ke.batched;
     } else {
         p.rows_per_warp = 1;

@@ -30,7 +30,8 @@ struct Header {
     unsigned long long error_id;    // id of the call that recorded `error_code`
     int error_code;
     int error_where;                // tile or row index, for diagnosis
-    unsigned long long reserved[29];
+    unsigned long long ticket;      // batched kernel: {call id (low 32 bits), next row group} of the running call
+    unsigned long long reserved[28];
 };
 static_assert(sizeof(Header) == 256, "workspace header is 256 bytes");
 
@@ -49,6 +50,7 @@ struct Params {
     int stages;         // input stages per warp (2..kMaxStages)
     int sign_vec_ok;    // sign tensors may be accessed with 16-byte vectors
     int rows_per_warp;  // R: rows held by one warp of the batched kernel (1, 2, 4, 8); look-back: 1
+    int row_tickets;    // batched kernel: row groups after a warp's first one are drawn from Header::ticket
     int flat_boxes;     // R == 1 and rows start on 128-byte lines: a chunk moves as ONE box of consecutive
                         // 128-byte lines of the flat [rows*n/line, line] view instead of one box per line
                         // (the partial last chunk of a row is stored line by line so as not to touch the next row)
@@ -422,9 +424,10 @@ struct WarpPipe {
 };
 
 // ------------------------------------------------------------------------------------------
-// (a) Row-batched kernel.  Persistent: warp w of G handles the row groups w, w+G, w+2G, ...; a
-// group is R consecutive rows (p.rows_per_warp), each walked chunk by chunk by 32/R lanes with
-// the value of x carried in registers.
+// (a) Row-batched kernel.  Persistent: every warp walks row groups one after the other -- the first
+// by its slot, the following ones drawn from a ticket counter --; a group is R consecutive rows
+// (p.rows_per_warp), each walked chunk by chunk by 32/R lanes with the value of x carried in
+// registers.
 template <int MODE, typename TIn, typename TOut, int K, bool TMA>
 __global__ void __launch_bounds__(512, 1)
 batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
@@ -454,39 +457,90 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
     pipe.setup(R, p.flat_boxes != 0);
     if (TMA) pipe.init();
 
-    if (blockIdx.x == 0 && threadIdx.x == 0) p.ws->started_id = p.call_id;
+    // With many row groups per warp slot (p.row_tickets) the groups are handed out by tickets: every warp
+    // starts with the group of its slot and draws the next one from a counter in the workspace, so that
+    // an SM that streams faster than another (their shares of the memory system differ by several
+    // percent) simply takes more rows.  With few groups per slot greedy hand-out would pile the last
+    // round on the SMs that are ahead, and the groups stay with their slots: slot, slot + GW, ...
+    // The counter word carries the low 32
+    // bits of the call id in its upper half: the first CTA to find another call's word there replaces it
+    // by {this call, first ticket = number of warp slots}; the workspace needs no initialisation and no
+    // host-side reset.
+    unsigned long long* const ticket_word = &p.ws->ticket;
+    const unsigned long long ticket_tag = (p.call_id & 0xffffffffull) << 32;
+    const int GW = gridDim.x * nwarps;
+    if (threadIdx.x == 0) {
+        if (blockIdx.x == 0) p.ws->started_id = p.call_id;
+        const unsigned long long seen = *(volatile unsigned long long*)ticket_word;
+        if ((seen & 0xffffffff00000000ull) != ticket_tag) atomicCAS(ticket_word, seen, ticket_tag | (unsigned long long)GW);
+    }
+    __syncthreads();  // from here on the word belongs to this call
 
     // All hot-loop indices are 32-bit and advance incrementally (rows < 2^31; with TMA also n < 2^31);
     // 64-bit products appear once per row only.
-    // Warp slots are numbered CTA-fastest, so that a last, partly filled round of row groups spreads
-    // over all SMs instead of loading the first CTAs only.
+    // Warp slots are numbered CTA-fastest, so that few row groups spread over all SMs.
     const int gw = warp * (int)gridDim.x + (int)blockIdx.x;
-    const int GW = gridDim.x * nwarps;
     const int groups = (int)((p.rows + R - 1) / R);
     if (gw >= groups) return;
-    const int my_groups = (groups - gw + GW - 1) / GW;
-    const long long items = (long long)my_groups * p.nchunks;
     const int nchunks = p.nchunks;
     const bool tail_ragged = (p.n % lm.W) != 0;  // the last chunk of a row is partial
     auto first_line = [&](int grp, int per_box) { return (int)(((long long)grp * R * p.n) / per_box); };
+    // A ticket is drawn a few chunks before the end of the current group -- late, so that the groups go
+    // to the warps that get there first, but early enough for the atomic's latency to stay off the path --
+    // and stays in lane 0 until the warp needs it.
+    const bool by_ticket = p.row_tickets != 0;
+    int static_next = gw;  // without tickets: slot, slot + GW, slot + 2 GW, ...
+    auto draw = [&]() -> unsigned int {
+        unsigned int t = 0u;
+        if (by_ticket) {
+            if (lane == 0) t = (unsigned int)atomicAdd(ticket_word, 1ull);
+        } else {
+            static_next = (static_next < groups) ? static_next + GW : groups;
+            t = (unsigned int)static_next;
+        }
+        return t;
+    };
+    auto take = [&](unsigned int t) -> int {
+        const unsigned int v = __shfl_sync(0xffffffffu, t, 0);
+        return v >= (unsigned int)groups ? groups : (int)v;
+    };
+    unsigned int drawn = 0u;
+    const int draw_at = nchunks > 3 ? nchunks - 3 : 0;  // index of the chunk with which the next ticket is drawn
+
+    // The row group the loads have entered and the arithmetic has not (the loads run one chunk ahead:
+    // p.stages == 2), with the x_0 of the lane's row, fetched when the group is entered.
+    int qn = 0, qa_group = 0;
+    typename CE::RawX0 qa_x0 = CE::load_x0(p, p.rows);
+    auto enter_group = [&](int g) {
+        qa_x0 = CE::load_x0(p, (long long)g * R + lm.g);
+        qa_group = g;
+        qn = 1;
+    };
 
     // producer cursor (TMA loads run S-1 chunks ahead)
     int pgroup = gw, pchunk = 0, pstage = 0;
+    bool loading = true;  // the producer still has a row group
     int pline = pipe.flat ? first_line(pgroup, Pipe::IN_PER_BOX) : 0;
-    long long issued = 0;
+    unsigned int issued = 0, consumed = 0;
     auto issue_next = [&]() {
+        if (pchunk == 0 && issued != 0) {  // the previous group is complete: enter the next one
+            pgroup = take(drawn);
+            if (pgroup >= groups) {
+                loading = false;
+                return;
+            }
+            enter_group(pgroup);
+            if (pipe.flat) pline = first_line(pgroup, Pipe::IN_PER_BOX);
+        }
         pipe.issue(&tm_a, &tm_b, pgroup * R, pchunk * lm.W, pline, pstage);
+        if (pchunk == draw_at) drawn = draw();
         ++issued;
         pline += Pipe::IN_LINES;
         if (++pstage == S) pstage = 0;
-        if (++pchunk == nchunks) {
-            pchunk = 0;
-            pgroup += GW;
-            if (pipe.flat && pgroup < groups) pline = first_line(pgroup, Pipe::IN_PER_BOX);
-        }
+        if (++pchunk == nchunks) pchunk = 0;
     };
     if (TMA) {
-        for (int s = 0; s < S - 1 && issued < items; ++s) issue_next();
+        for (int s = 0; s < S - 1 && loading; ++s) issue_next();
     }
 
     int group = gw, chunk = 0, colbase = 0;
@@ -494,15 +548,14 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
     long long row = (long long)group * R + lm.g;
     bool group_ragged = (group + 1) * (long long)R > p.rows;
     E state = CE::row_start(p, row);
-    typename CE::RawX0 x0_next = CE::load_x0(p, row + (long long)GW * R);  // in flight during this row
     int stage = 0;
     uint32_t parity = 0;
-    for (long long q = 0; q < items; ++q) {
+    while (group < groups) {
         if (TMA) {
-            if (issued < items) issue_next();
+            if (loading) issue_next();
             if (!pipe.wait(stage, parity)) {
                 if (lane == 0) record_error(p, kErrCopyTimeout, row);
-                pipe.drain_loads(q + 1, issued);
+                pipe.drain_loads(consumed + 1, issued);
                 break;
             }
         } else {
@@ -511,7 +564,7 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
         }
         const uint32_t sm_a = pipe.in_a(stage);
         const uint32_t sm_b = pipe.in_b(stage);
-        const uint32_t sm_out = pipe.out((int)(q & 1));
+        const uint32_t sm_out = pipe.out((int)(consumed & 1));
         const int col0 = colbase + lm.i * K;
         const bool ragged = group_ragged || (tail_ragged && chunk == nchunks - 1);
 
@@ -531,18 +584,25 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
             CE::generic_store(p, sm_out, lm, lane, (long long)group * R, colbase);
         }
         __syncwarp();  // every lane is done with this input stage
+        ++consumed;
+        if (!TMA && chunk == draw_at) drawn = draw();
 
         colbase += lm.W;
         oline += Pipe::OUT_LINES;
         if (++chunk == nchunks) {
             chunk = 0;
             colbase = 0;
-            group += GW;
+            if (!TMA) {  // no loads ahead: the arithmetic enters the next group itself
+                const int g = take(drawn);
+                if (g < groups) enter_group(g);
+            }
+            if (qn == 0) break;  // no group left for this warp
+            group = qa_group;
+            state = CE::x0_elem(qa_x0);
+            qn = 0;
             row = (long long)group * R + lm.g;
             group_ragged = (group + 1) * (long long)R > p.rows;
-            state = CE::x0_elem(x0_next);
-            x0_next = CE::load_x0(p, row + (long long)GW * R);
-            if (pipe.flat && group < groups) oline = first_line(group, Pipe::OUT_PER_BOX);
+            if (pipe.flat) oline = first_line(group, Pipe::OUT_PER_BOX);
         }
         if (++stage == S) { stage = 0; parity ^= 1u; }
     }
