@@ -420,7 +420,20 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
             e = cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(warps * 32), args, smem, stream);
         }
     } else {
-        e = cudaLaunchKernel(fn, dim3(grid), dim3(warps * 32), args, smem, stream);
+        // programmatic stream serialisation: the kernel's set-up may overlap the end of the previous kernel
+        // of the stream; it waits (griddepcontrol.wait) before its first access to global memory
+        cudaLaunchConfig_t cfg;
+        std::memset(&cfg, 0, sizeof cfg);
+        cfg.gridDim = dim3(grid);
+        cfg.blockDim = dim3(warps * 32);
+        cfg.dynamicSmemBytes = (size_t)smem;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = env_int("HEINSEN_SCAN_NO_PDL", 0, 0, 1) ? 0 : 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        e = cudaLaunchKernelExC(&cfg, fn, args);
     }
     if (e != cudaSuccess) return cuda_fail("kernel launch", e);
     g_last_path.store(path);

@@ -456,6 +456,11 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
     pipe.lane = lane;
     pipe.setup(R, p.flat_boxes != 0);
     if (TMA) pipe.init();
+    // Programmatic dependent launch: the next kernel of the stream may be set up while this one runs
+    // (it waits below before it touches memory), and this kernel touches global memory only after
+    // everything before it in the stream has completed.  Both are no-ops for an ordinary launch.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // With many row groups per warp slot (p.row_tickets) the groups are handed out by tickets: every warp
     // starts with the group of its slot and draws the next one from a counter in the workspace, so that
