@@ -514,12 +514,11 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
 
     // The row group the loads have entered and the arithmetic has not (the loads run one chunk ahead:
     // p.stages == 2), with the x_0 of the lane's row, fetched when the group is entered.
-    int qn = 0, qa_group = 0;
+    int qa_group = -1;  // -1: none
     typename CE::RawX0 qa_x0 = CE::load_x0(p, p.rows);
     auto enter_group = [&](int g) {
         qa_x0 = CE::load_x0(p, (long long)g * R + lm.g);
         qa_group = g;
-        qn = 1;
     };
 
     // producer cursor (TMA loads run S-1 chunks ahead)
@@ -601,10 +600,10 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
                 const int g = take(drawn);
                 if (g < groups) enter_group(g);
             }
-            if (qn == 0) break;  // no group left for this warp
+            if (qa_group < 0) break;  // no group left for this warp
             group = qa_group;
             state = CE::x0_elem(qa_x0);
-            qn = 0;
+            qa_group = -1;
             row = (long long)group * R + lm.g;
             group_ragged = (group + 1) * (long long)R > p.rows;
             if (pipe.flat) oline = first_line(group, Pipe::OUT_PER_BOX);
