@@ -134,6 +134,28 @@ def test_odd_shapes_both_paths(hs, oracle, rows, n):
         run_log(hs, oracle, w.tensors, path=path, what=f"{rows}x{n}/{path}")
 
 
+@pytest.mark.parametrize("rows,n", [(40000, 77), (30001, 160), (12000, 1536), (70000, 33)])
+def test_many_rows_handed_out_by_tickets(hs, oracle, rows, n):
+    """Enough row groups per warp slot for the batched kernel to draw them from its ticket counter: several rows
+    per warp without TMA (n*4 % 16 != 0), several rows per warp with TMA boxes, one row per warp with flat boxes."""
+    w = workloads.make(2, rows=rows, n=n, seed=rows + n)
+    run_log(hs, oracle, w.tensors, path=hs.PATH_BATCHED, what=f"tickets {rows}x{n}")
+    # twice on the same workspace: the second call must take over the first call's ticket word
+    la, lb, lx0 = to_dev(w.tensors["log_a"]), to_dev(w.tensors["log_b"]), to_dev(w.tensors["log_x0"])
+    ws = hs.new_workspace(rows, n, "cuda")
+    first = hs.scan_log(la, lb, lx0, workspace=ws)
+    second = hs.scan_log(la, lb, lx0, workspace=ws)
+    hs.check(ws)
+    assert torch.equal(first, second)
+
+
+def test_tickets_forced_on_few_rows(hs, oracle, monkeypatch):
+    monkeypatch.setenv("HEINSEN_SCAN_ROW_TICKETS", "1")
+    for rows, n in ((5, 4100), (300, 515), (2400, 2048)):
+        w = workloads.make(2, rows=rows, n=n, seed=rows)
+        run_log(hs, oracle, w.tensors, path=hs.PATH_BATCHED, what=f"forced tickets {rows}x{n}")
+
+
 @pytest.mark.parametrize("n", [7, 520, 4099])
 def test_odd_shapes_signed_linear(hs, oracle, n):
     w = workloads.make(4, rows=5, n=n, seed=n)
