@@ -135,7 +135,8 @@ struct Problem {
 using BatchedFn = void (*)(const Params, const CUtensorMap, const CUtensorMap, const CUtensorMap);
 
 struct KernelEntry {
-    const void* batched;
+    const void* batched;      // row groups stay with their warp slots
+    const void* batched_tk;   // row groups handed out by tickets
     const void* lookback;
     int K;
     int warp_smem_per_stage;  // bytes of one input stage (both tensors) of one warp
@@ -148,7 +149,8 @@ template <int MODE, typename TIn, typename TOut, int K, bool TMA>
 KernelEntry entry() {
     KernelEntry e;
     constexpr int LBK = 16;  // the look-back kernel parks fp32 partial sums: 16 per lane for every type
-    e.batched = reinterpret_cast<const void*>(&batched_scan_kernel<MODE, TIn, TOut, K, TMA>);
+    e.batched = reinterpret_cast<const void*>(&batched_scan_kernel<MODE, TIn, TOut, K, TMA, false>);
+    e.batched_tk = reinterpret_cast<const void*>(&batched_scan_kernel<MODE, TIn, TOut, K, TMA, true>);
     e.lookback = reinterpret_cast<const void*>(&lookback_scan_kernel<MODE, TIn, TOut, LBK, TMA>);
     e.lb_K = LBK;
     e.K = K;
@@ -162,7 +164,8 @@ KernelEntry entry() {
 template <int MODE, typename TIn, typename TOut, int K, bool TMA>
 KernelEntry entry_batched_only() {
     KernelEntry e;
-    e.batched = reinterpret_cast<const void*>(&batched_scan_kernel<MODE, TIn, TOut, K, TMA>);
+    e.batched = reinterpret_cast<const void*>(&batched_scan_kernel<MODE, TIn, TOut, K, TMA, false>);
+    e.batched_tk = reinterpret_cast<const void*>(&batched_scan_kernel<MODE, TIn, TOut, K, TMA, true>);
     e.lookback = nullptr;
     e.lb_K = K;
     e.K = K;
@@ -332,9 +335,10 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         grid = (int)(ctas_needed < dev.sm_count ? ctas_needed : dev.sm_count);
         // tickets balance SMs of unequal speed when every warp slot sees several groups; with fewer, a
         // greedy hand-out of the last round loses more than it gains (cfg4, 1.7 groups per slot: 81 vs 74 us)
-        p.row_tickets = groups >= 4ll * grid * warps ? 1 : 0;
-        p.row_tickets = env_int("HEINSEN_SCAN_ROW_TICKETS", p.row_tickets, 0, 1);
-        fn = ke.batched;
+        // ... and only for rows of at least four chunks, where a ticket can be drawn early enough to arrive in time
+        int tickets = (groups >= 4ll * grid * warps && p.nchunks >= 4) ? 1 : 0;
+        tickets = env_int("HEINSEN_SCAN_ROW_TICKETS", tickets, 0, 1);
+        fn = tickets ? ke.batched_tk : ke.batched;
     } else {
         p.rows_per_warp = 1;
         // S input stages per compute warp (phase 2 of a tile runs S-2 iterations after its phase 1),

@@ -50,7 +50,6 @@ struct Params {
     int stages;         // input stages per warp (2..kMaxStages)
     int sign_vec_ok;    // sign tensors may be accessed with 16-byte vectors
     int rows_per_warp;  // R: rows held by one warp of the batched kernel (1, 2, 4, 8); look-back: 1
-    int row_tickets;    // batched kernel: row groups after a warp's first one are drawn from Header::ticket
     int flat_boxes;     // R == 1 and rows start on 128-byte lines: a chunk moves as ONE box of consecutive
                         // 128-byte lines of the flat [rows*n/line, line] view instead of one box per line
                         // (the partial last chunk of a row is stored line by line so as not to touch the next row)
@@ -428,7 +427,7 @@ struct WarpPipe {
 // by its slot, the following ones drawn from a ticket counter --; a group is R consecutive rows
 // (p.rows_per_warp), each walked chunk by chunk by 32/R lanes with the value of x carried in
 // registers.
-template <int MODE, typename TIn, typename TOut, int K, bool TMA>
+template <int MODE, typename TIn, typename TOut, int K, bool TMA, bool TICKETS>
 __global__ void __launch_bounds__(512, 1)
 batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                     const __grid_constant__ CUtensorMap tm_o, const __grid_constant__ CUtensorMap tm_o1) {
@@ -462,7 +461,7 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
-    // With many row groups per warp slot (p.row_tickets) the groups are handed out by tickets: every warp
+    // With many row groups per warp slot (TICKETS; the host decides) the groups are handed out by tickets: every warp
     // starts with the group of its slot and draws the next one from a counter in the workspace, so that
     // an SM that streams faster than another (their shares of the memory system differ by several
     // percent) simply takes more rows.  With few groups per slot greedy hand-out would pile the last
@@ -476,10 +475,13 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
     const int GW = gridDim.x * nwarps;
     if (threadIdx.x == 0) {
         if (blockIdx.x == 0) p.ws->started_id = p.call_id;
-        const unsigned long long seen = *(volatile unsigned long long*)ticket_word;
-        if ((seen & 0xffffffff00000000ull) != ticket_tag) atomicCAS(ticket_word, seen, ticket_tag | (unsigned long long)GW);
+        if (TICKETS) {
+            const unsigned long long seen = *(volatile unsigned long long*)ticket_word;
+            if ((seen & 0xffffffff00000000ull) != ticket_tag)
+                atomicCAS(ticket_word, seen, ticket_tag | (unsigned long long)GW);
+        }
     }
-    __syncthreads();  // from here on the word belongs to this call
+    if (TICKETS) __syncthreads();  // from here on the word belongs to this call
 
     // All hot-loop indices are 32-bit and advance incrementally (rows < 2^31; with TMA also n < 2^31);
     // 64-bit products appear once per row only.
@@ -492,17 +494,11 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
     auto first_line = [&](int grp, int per_box) { return (int)(((long long)grp * R * p.n) / per_box); };
     // A ticket is drawn a few chunks before the end of the current group -- late, so that the groups go
     // to the warps that get there first, but early enough for the atomic's latency to stay off the path --
-    // and stays in lane 0 until the warp needs it.
-    const bool by_ticket = p.row_tickets != 0;
-    int static_next = gw;  // without tickets: slot, slot + GW, slot + 2 GW, ...
+    // and stays in lane 0 until the warp needs it.  Without tickets a warp walks slot, slot + GW, ...
+    constexpr bool by_ticket = TICKETS;  // two instantiations: the hand-over code of one does not burden the other
     auto draw = [&]() -> unsigned int {
         unsigned int t = 0u;
-        if (by_ticket) {
-            if (lane == 0) t = (unsigned int)atomicAdd(ticket_word, 1ull);
-        } else {
-            static_next = (static_next < groups) ? static_next + GW : groups;
-            t = (unsigned int)static_next;
-        }
+        if (lane == 0) t = (unsigned int)atomicAdd(ticket_word, 1ull);
         return t;
     };
     auto take = [&](unsigned int t) -> int {
@@ -511,11 +507,14 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
     };
     unsigned int drawn = 0u;
     const int draw_at = nchunks > 3 ? nchunks - 3 : 0;  // index of the chunk with which the next ticket is drawn
+    // without tickets the warp's share is known: groups gw, gw + GW, ... and so many chunks
+    const long long items = TICKETS ? 0 : (long long)((groups - gw + GW - 1) / GW) * nchunks;
 
-    // The row group the loads have entered and the arithmetic has not (the loads run one chunk ahead:
-    // p.stages == 2), with the x_0 of the lane's row, fetched when the group is entered.
-    int qa_group = -1;  // -1: none
-    typename CE::RawX0 qa_x0 = CE::load_x0(p, p.rows);
+    // x_0 of the lane's row in the next group, in flight while the current group is worked on.  With
+    // tickets: the group the loads have entered and the arithmetic has not (the loads run one chunk ahead:
+    // p.stages == 2; -1: none), x_0 fetched when the group is entered.  Without: the group after this one.
+    int qa_group = -1;
+    typename CE::RawX0 qa_x0 = CE::load_x0(p, TICKETS ? p.rows : ((long long)gw + GW) * R + lm.g);
     auto enter_group = [&](int g) {
         qa_x0 = CE::load_x0(p, (long long)g * R + lm.g);
         qa_group = g;
@@ -525,23 +524,36 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
     int pgroup = gw, pchunk = 0, pstage = 0;
     bool loading = true;  // the producer still has a row group
     int pline = pipe.flat ? first_line(pgroup, Pipe::IN_PER_BOX) : 0;
-    unsigned int issued = 0, consumed = 0;
+    long long issued = 0, consumed = 0;
     auto issue_next = [&]() {
-        if (pchunk == 0 && issued != 0) {  // the previous group is complete: enter the next one
-            pgroup = take(drawn);
-            if (pgroup >= groups) {
-                loading = false;
-                return;
+        if (TICKETS) {
+            if (pchunk == 0 && issued != 0) {  // the previous group is complete: enter the next one
+                pgroup = take(drawn);
+                if (pgroup >= groups) {
+                    loading = false;
+                    return;
+                }
+                enter_group(pgroup);
+                if (pipe.flat) pline = first_line(pgroup, Pipe::IN_PER_BOX);
             }
-            enter_group(pgroup);
-            if (pipe.flat) pline = first_line(pgroup, Pipe::IN_PER_BOX);
+            pipe.issue(&tm_a, &tm_b, pgroup * R, pchunk * lm.W, pline, pstage);
+            if (pchunk == draw_at) drawn = draw();
+            ++issued;
+            pline += Pipe::IN_LINES;
+            if (++pstage == S) pstage = 0;
+            if (++pchunk == nchunks) pchunk = 0;
+        } else {
+            pipe.issue(&tm_a, &tm_b, pgroup * R, pchunk * lm.W, pline, pstage);
+            ++issued;
+            pline += Pipe::IN_LINES;
+            if (++pstage == S) pstage = 0;
+            if (++pchunk == nchunks) {
+                pchunk = 0;
+                pgroup += GW;
+                if (pipe.flat && pgroup < groups) pline = first_line(pgroup, Pipe::IN_PER_BOX);
+            }
+            loading = issued < items;
         }
-        pipe.issue(&tm_a, &tm_b, pgroup * R, pchunk * lm.W, pline, pstage);
-        if (pchunk == draw_at) drawn = draw();
-        ++issued;
-        pline += Pipe::IN_LINES;
-        if (++pstage == S) pstage = 0;
-        if (++pchunk == nchunks) pchunk = 0;
     };
     if (TMA) {
         for (int s = 0; s < S - 1 && loading; ++s) issue_next();
@@ -554,7 +566,7 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
     E state = CE::row_start(p, row);
     int stage = 0;
     uint32_t parity = 0;
-    while (group < groups) {
+    while (TICKETS ? group < groups : consumed < items) {
         if (TMA) {
             if (loading) issue_next();
             if (!pipe.wait(stage, parity)) {
@@ -589,21 +601,27 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
         }
         __syncwarp();  // every lane is done with this input stage
         ++consumed;
-        if (!TMA && chunk == draw_at) drawn = draw();
+        if (!TMA && by_ticket && chunk == draw_at) drawn = draw();
 
         colbase += lm.W;
         oline += Pipe::OUT_LINES;
         if (++chunk == nchunks) {
             chunk = 0;
             colbase = 0;
-            if (!TMA) {  // no loads ahead: the arithmetic enters the next group itself
-                const int g = take(drawn);
-                if (g < groups) enter_group(g);
+            if (by_ticket) {
+                if (!TMA) {  // no loads ahead: the arithmetic enters the next group itself
+                    const int g = take(drawn);
+                    if (g < groups) enter_group(g);
+                }
+                if (qa_group < 0) break;  // no group left for this warp
+                group = qa_group;
+                state = CE::x0_elem(qa_x0);
+                qa_group = -1;
+            } else {
+                group += GW;  // beyond the last group only when the loop is about to end
+                state = CE::x0_elem(qa_x0);
+                qa_x0 = CE::load_x0(p, ((long long)group + GW) * R + lm.g);
             }
-            if (qa_group < 0) break;  // no group left for this warp
-            group = qa_group;
-            state = CE::x0_elem(qa_x0);
-            qa_group = -1;
             row = (long long)group * R + lm.g;
             group_ragged = (group + 1) * (long long)R > p.rows;
             if (pipe.flat) oline = first_line(group, Pipe::OUT_PER_BOX);
