@@ -315,13 +315,28 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
     if (path == HS_PATH_BATCHED) {
         // R rows per warp (32/R lanes per row): the largest R that still leaves about a dozen warps
         // per SM, so that rows with many steps use few scan steps and few rows still fill the GPU.
-        int R = 8;
+        // (16 only where a row's piece of the output chunk, 2 lanes x K elements, still fills a 128-byte line)
+        int R = (2 * ke.K * es_out >= 128) ? 16 : 8;
         while (R > 1 && (p.rows + R - 1) / R < (long long)kBatchedMinWarpsPerSm * dev.sm_count) R >>= 1;
-        // rows that start on 128-byte lines, and enough of them: one row per warp, each chunk one contiguous box
-        if (tma && (p.n * es_in) % 128 == 0 && (p.n * es_out) % 128 == 0 &&
-            p.rows >= (long long)kBatchedMinWarpsPerSm * dev.sm_count)
+        const int full_chunk = 32 * ke.K;  // columns of a chunk when the warp holds one row
+        if (R == 16 && p.n >= full_chunk / 8) R = 8;  // 16 rows per warp only for rows shorter than an eighth of a chunk
+        if (p.n < full_chunk) {
+            // short rows: among the R allowed, the one whose chunks (full_chunk / R columns wide) pad the row
+            // least, the larger R on a tie (fewer scan steps); 262144 x 128: R = 1 1.7 TB/s, R = 4 5.8 TB/s
+            int best = R;
+            long long best_cols = -1;
+            for (int r = R; r >= 1; r >>= 1) {
+                const int w = full_chunk / r;
+                const long long cols = (p.n + w - 1) / w * w;  // columns processed per row
+                if (best_cols < 0 || cols < best_cols) { best_cols = cols; best = r; }
+            }
+            R = best;
+        } else if (tma && (p.n * es_in) % 128 == 0 && (p.n * es_out) % 128 == 0 &&
+                   p.rows >= (long long)kBatchedMinWarpsPerSm * dev.sm_count) {
+            // rows that start on 128-byte lines, and enough of them: one row per warp, each chunk one contiguous box
             R = 1;
-        R = env_int("HEINSEN_SCAN_ROWS_PER_WARP", R, 1, 8);
+        }
+        R = env_int("HEINSEN_SCAN_ROWS_PER_WARP", R, 1, 16);
         while (R & (R - 1)) R &= R - 1;  // power of two
         p.rows_per_warp = R;
         p.nchunks = (int)((p.n + (32 / R) * ke.K - 1) / ((32 / R) * ke.K));

@@ -49,7 +49,7 @@ struct Params {
     int nchunks;        // chunks per row
     int stages;         // input stages per warp (2..kMaxStages)
     int sign_vec_ok;    // sign tensors may be accessed with 16-byte vectors
-    int rows_per_warp;  // R: rows held by one warp of the batched kernel (1, 2, 4, 8); look-back: 1
+    int rows_per_warp;  // R: rows held by one warp of the batched kernel (1, 2, 4, 8, 16); look-back: 1
     int flat_boxes;     // R == 1 and rows start on 128-byte lines: a chunk moves as ONE box of consecutive
                         // 128-byte lines of the flat [rows*n/line, line] view instead of one box per line
                         // (the partial last chunk of a row is stored line by line so as not to touch the next row)
@@ -88,7 +88,7 @@ __device__ __forceinline__ float neutral_b() { return MODE == kLinear ? 0.0f : n
 // Where a lane sits in its warp's chunk: the warp holds R rows, lane = i*R + g is segment i
 // (K consecutive elements) of row g; a row's piece of the chunk is W = (32/R)*K elements wide.
 struct LaneMap {
-    int R;     // rows per warp: 1, 2, 4 or 8
+    int R;     // rows per warp: 1, 2, 4, 8 or 16
     int g;     // row within the warp's group
     int i;     // segment within the row's piece
     int W;     // elements per row per chunk

@@ -149,6 +149,17 @@ def test_many_rows_handed_out_by_tickets(hs, oracle, rows, n):
     assert torch.equal(first, second)
 
 
+@pytest.mark.parametrize("rows,n,cid", [(50000, 16, 2), (40000, 24, 2), (30011, 32, 2), (30000, 40, 2), (25000, 64, 2),
+                                         (20000, 100, 2), (20000, 128, 2), (30000, 48, 5), (30000, 40, 4)])
+def test_many_short_rows(hs, oracle, rows, n, cid):
+    """Rows shorter than a chunk: the warp holds 2 to 16 rows, chosen so that the chunks pad the rows least."""
+    w = workloads.make(cid, rows=rows, n=n, seed=rows + n)
+    if cid == 4:
+        run_linear(hs, oracle, w.tensors, path=hs.PATH_BATCHED, signed=True, what=f"short rows {rows}x{n}")
+    else:
+        run_log(hs, oracle, w.tensors, path=hs.PATH_BATCHED, what=f"short rows {rows}x{n}")
+
+
 def test_tickets_forced_on_few_rows(hs, oracle, monkeypatch):
     monkeypatch.setenv("HEINSEN_SCAN_ROW_TICKETS", "1")
     for rows, n in ((5, 4100), (300, 515), (2400, 2048)):
