@@ -95,23 +95,30 @@ EncodeFn encode_fn() {
 }
 
 // [rows, n] row-major as a 2-D tensor map whose box is {128 bytes of a row, box_rows rows}, 128-byte swizzle.
-// flat: the same memory as [rows*n*es/128, 128 bytes] (lines), box = box_rows consecutive lines.
+// flat: the same memory as (element in 128-byte line, whole line of the row, row), box = box_rows consecutive
+// lines of one row; the hardware clips a box at the row's last whole line, the n % line elements after it
+// are not part of this view.
 bool make_tmap(CUtensorMap* tm, const void* ptr, hs_dtype dt, long long rows, long long n, int box_rows, bool flat) {
     EncodeFn fn = encode_fn();
     if (!fn) return false;
     const int es = (dt == HS_F32) ? 4 : 2;
-    cuuint64_t dims[2] = {(cuuint64_t)n, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)n * es};
+    const CUtensorMapDataType type = dt == HS_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r;
     if (flat) {
-        dims[0] = (cuuint64_t)(128 / es);
-        dims[1] = (cuuint64_t)(rows * n * es / 128);
-        strides[0] = 128;
+        const cuuint64_t line = (cuuint64_t)(128 / es);
+        cuuint64_t dims[3] = {line, (cuuint64_t)n / line, (cuuint64_t)rows};
+        cuuint64_t strides[2] = {128, (cuuint64_t)n * es};
+        cuuint32_t box[3] = {(cuuint32_t)line, (cuuint32_t)box_rows, 1};
+        r = fn(tm, type, 3, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    } else {
+        cuuint64_t dims[2] = {(cuuint64_t)n, (cuuint64_t)rows};
+        cuuint64_t strides[1] = {(cuuint64_t)n * es};
+        cuuint32_t box[2] = {(cuuint32_t)(128 / es), (cuuint32_t)box_rows};
+        r = fn(tm, type, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     }
-    cuuint32_t box[2] = {(cuuint32_t)(128 / es), (cuuint32_t)box_rows};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(tm, dt == HS_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
-                    const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
 
@@ -331,9 +338,8 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
                 if (best_cols < 0 || cols < best_cols) { best_cols = cols; best = r; }
             }
             R = best;
-        } else if (tma && (p.n * es_in) % 128 == 0 && (p.n * es_out) % 128 == 0 &&
-                   p.rows >= (long long)kBatchedMinWarpsPerSm * dev.sm_count) {
-            // rows that start on 128-byte lines, and enough of them: one row per warp, each chunk one contiguous box
+        } else if (tma && p.rows >= (long long)kBatchedMinWarpsPerSm * dev.sm_count) {
+            // enough rows that TMA can address: one row per warp, each chunk one box of 128-byte lines
             R = 1;
         }
         R = env_int("HEINSEN_SCAN_ROWS_PER_WARP", R, 1, 16);
@@ -388,22 +394,20 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         grid = 0;  // set below from occupancy
     }
 
-    CUtensorMap tm_a, tm_b, tm_o, tm_o1;
-    std::memset(&tm_o1, 0, sizeof tm_o1);
+    CUtensorMap tm_a, tm_b, tm_o;
     std::memset(&tm_a, 0, sizeof tm_a);
     std::memset(&tm_b, 0, sizeof tm_b);
     std::memset(&tm_o, 0, sizeof tm_o);
     if (tma) {
-        // one row per warp and whole chunks only: move a chunk as a single box of consecutive lines
-        const bool flat = p.rows_per_warp == 1 && (p.n * es_in) % 128 == 0 && (p.n * es_out) % 128 == 0 &&
-                          p.rows * p.n * es_in / 128 < (1ll << 31) && !env_int("HEINSEN_SCAN_NO_FLAT", 0, 0, 1);
+        // one row per warp, rows of at least one whole 128-byte line: move a chunk as a single box of lines
+        const bool flat = p.rows_per_warp == 1 && p.n * es_in >= 128 && p.n * es_out >= 128 &&
+                          !env_int("HEINSEN_SCAN_NO_FLAT", 0, 0, 1);
         p.flat_boxes = flat ? 1 : 0;
         const int br_in = flat ? chunk * es_in / 128 : p.rows_per_warp;
         const int br_out = flat ? chunk * es_out / 128 : p.rows_per_warp;
         if (!make_tmap(&tm_a, p.in_a, pr.din, p.rows, p.n, br_in, flat) ||
             !make_tmap(&tm_b, p.in_b, pr.din, p.rows, p.n, br_in, flat) ||
-            !make_tmap(&tm_o, p.out, pr.dout, p.rows, p.n, br_out, flat) ||
-            (flat && !make_tmap(&tm_o1, p.out, pr.dout, p.rows, p.n, 1, true))) {
+            !make_tmap(&tm_o, p.out, pr.dout, p.rows, p.n, br_out, flat)) {
             snprintf(g_cuda_msg, sizeof g_cuda_msg, "cuTensorMapEncodeTiled failed");
             return HS_ERR_CUDA;
         }
@@ -416,7 +420,7 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
     cudaError_t e = ensure_smem_attr(fn, smem);
     if (e != cudaSuccess) return cuda_fail("cudaFuncSetAttribute", e);
 
-    void* args[] = {&p, &tm_a, &tm_b, &tm_o, &tm_o1};
+    void* args[] = {&p, &tm_a, &tm_b, &tm_o};
     if (path == HS_PATH_LOOKBACK) {
         // Tiles wait for their predecessors, so every CTA must be resident: size the grid from the
         // occupancy of this kernel and launch cooperatively (the launch fails rather than deadlocks).

@@ -50,9 +50,9 @@ struct Params {
     int stages;         // input stages per warp (2..kMaxStages)
     int sign_vec_ok;    // sign tensors may be accessed with 16-byte vectors
     int rows_per_warp;  // R: rows held by one warp of the batched kernel (1, 2, 4, 8, 16); look-back: 1
-    int flat_boxes;     // R == 1 and rows start on 128-byte lines: a chunk moves as ONE box of consecutive
-                        // 128-byte lines of the flat [rows*n/line, line] view instead of one box per line
-                        // (the partial last chunk of a row is stored line by line so as not to touch the next row)
+    int flat_boxes;     // R == 1: the tensor maps show a matrix as (element in 128-byte line, whole line of the row,
+                        // row), and a chunk moves as ONE box of consecutive lines instead of one box per line;
+                        // the last n % line elements of a row, if any, move by plain loads and stores
     unsigned long long call_id;
     Header* ws;
     // look-back kernel only
@@ -312,6 +312,34 @@ struct ChunkEngine {
             }
         }
     }
+
+    // Flat boxes move whole 128-byte lines of a row; the last n % line elements of the row travel by
+    // plain loads and stores, into and out of the places they have in the chunk that holds them
+    // (one row per warp; colbase: first column of that chunk).
+    static constexpr int IN_LINE = 128 / (int)sizeof(TIn), OUT_LINE = 128 / (int)sizeof(TOut);
+    // (out of line: rare, and the chunk loop should stay small)
+    __device__ static __noinline__ void tail_load_impl(const void* in_a, const void* in_b, long long n, uint32_t sm_a,
+                                                       uint32_t sm_b, int lane, long long row, int colbase) {
+        for (int col = (int)(n / IN_LINE) * IN_LINE + lane; col < n; col += 32) {
+            const uint32_t off = chunk_off(1, 0, (uint32_t)((col - colbase) * sizeof(TIn)));
+            Storage<TIn>::to_smem(sm_a + off, Storage<TIn>::load(in_a, row * n + col));
+            Storage<TIn>::to_smem(sm_b + off, Storage<TIn>::load(in_b, row * n + col));
+        }
+    }
+    __device__ static __noinline__ void tail_store_impl(void* out, long long n, uint32_t sm_out, int lane, long long row,
+                                                        int colbase) {
+        for (int col = (int)(n / OUT_LINE) * OUT_LINE + lane; col < n; col += 32) {
+            const uint32_t off = chunk_off(1, 0, (uint32_t)((col - colbase) * sizeof(TOut)));
+            Storage<TOut>::store(out, row * n + col, Storage<TOut>::from_smem(sm_out + off));
+        }
+    }
+    __device__ static __forceinline__ void tail_load(const Params& p, uint32_t sm_a, uint32_t sm_b, int lane, long long row,
+                                                     int colbase) {
+        tail_load_impl(p.in_a, p.in_b, p.n, sm_a, sm_b, lane, row, colbase);
+    }
+    __device__ static __forceinline__ void tail_store(const Params& p, uint32_t sm_out, int lane, long long row, int colbase) {
+        tail_store_impl(p.out, p.n, sm_out, lane, row, colbase);
+    }
 };
 
 }  // namespace hs
@@ -343,13 +371,13 @@ struct WarpPipe {
     int R;           // rows per box
     int in_boxes;    // boxes per tensor per chunk, input / output
     int out_boxes;
-    bool flat;       // one box per chunk, addressed by line number (see Params::flat_boxes)
+    bool flat;       // one box per chunk (see Params::flat_boxes)
 
     __device__ __forceinline__ void setup(int rows_per_warp, bool flat_boxes = false) {
         R = rows_per_warp;
         flat = flat_boxes;
         in_boxes = flat ? 1 : IN_BYTES / (128 * R);
-        out_boxes = flat ? OUT_BYTES / 128 : OUT_BYTES / (128 * R);  // lanes that issue (or may issue) stores
+        out_boxes = flat ? 1 : OUT_BYTES / (128 * R);  // lanes that issue stores
     }
     __device__ __forceinline__ uint32_t in_a(int s) const { return base + s * 2 * IN_BYTES; }
     __device__ __forceinline__ uint32_t in_b(int s) const { return base + s * 2 * IN_BYTES + IN_BYTES; }
@@ -362,17 +390,17 @@ struct WarpPipe {
         }
         __syncwarp();
     }
-    // colbase: first column of the chunk, row0: first row of the group; `line` (flat boxes only):
-    // index of the chunk's first 128-byte line in the flat view
-    __device__ __forceinline__ void issue(const CUtensorMap* tm_a, const CUtensorMap* tm_b, int row0, int colbase, int line,
-                                          int s) {
+    // colbase: first column of the chunk, row0: first row of the group.  Flat boxes: the tensor maps
+    // show a matrix as (element in line, whole line of the row, row); a chunk is the box of IN_LINES
+    // lines from line colbase / IN_PER_BOX of row row0, clipped by the hardware at the row's last whole line.
+    __device__ __forceinline__ void issue(const CUtensorMap* tm_a, const CUtensorMap* tm_b, int row0, int colbase, int s) {
         const uint32_t bar = bars + 8 * s;
         if (lane == 0) mbar_expect_tx(bar, 2 * IN_BYTES);
         __syncwarp();
         if (flat) {
             if (lane == 0) {
-                tma_load_2d(in_a(s), tm_a, 0, line, bar);
-                tma_load_2d(in_b(s), tm_b, 0, line, bar);
+                tma_load_3d(in_a(s), tm_a, 0, colbase / IN_PER_BOX, row0, bar);
+                tma_load_3d(in_b(s), tm_b, 0, colbase / IN_PER_BOX, row0, bar);
             }
         } else if (lane < in_boxes) {
             const int x = colbase + lane * IN_PER_BOX;
@@ -389,20 +417,15 @@ struct WarpPipe {
         if (lane < out_boxes) bulk_wait_read<1>();
         __syncwarp();
     }
-    // store the chunk held in shared memory at `src`; `line`: as for issue(), in output lines;
-    // flat boxes: `valid_lines` < OUT_LINES for the partial last chunk of a row, which goes out as
-    // single lines through `tm_o1` (same view, one-line box)
-    __device__ __forceinline__ void store_from(const CUtensorMap* tm_o, const CUtensorMap* tm_o1, int row0, int colbase,
-                                               int line, uint32_t src, int valid_lines) const {
+    // store the chunk held in shared memory at `src` (flat boxes: its whole lines; see issue())
+    __device__ __forceinline__ void store_from(const CUtensorMap* tm_o, int row0, int colbase, uint32_t src) const {
         fence_async_smem();
         __syncwarp();
         if (flat) {
-            if (valid_lines >= OUT_BYTES / 128) {
-                if (lane == 0) tma_store_2d(tm_o, 0, line, src);
-            } else if (lane < valid_lines) {
-                tma_store_2d(tm_o1, 0, line + lane, src + (uint32_t)(lane * 128));
+            if (lane == 0) {
+                tma_store_3d(tm_o, 0, colbase / OUT_PER_BOX, row0, src);
+                bulk_commit();
             }
-            if (lane < out_boxes) bulk_commit();  // every lane that may ever store keeps its group count in step
         } else if (lane < out_boxes) {
             const int x = colbase + lane * OUT_PER_BOX;
             tma_store_2d(tm_o, x, row0, src + (uint32_t)(lane * R * 128));
@@ -430,7 +453,7 @@ struct WarpPipe {
 template <int MODE, typename TIn, typename TOut, int K, bool TMA, bool TICKETS>
 __global__ void __launch_bounds__(512, 1)
 batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-                    const __grid_constant__ CUtensorMap tm_o, const __grid_constant__ CUtensorMap tm_o1) {
+                    const __grid_constant__ CUtensorMap tm_o) {
     using CE = ChunkEngine<MODE, TIn, TOut, K>;
     using E = typename CE::E;
     extern __shared__ uint8_t smem_raw[];
@@ -491,7 +514,10 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
     if (gw >= groups) return;
     const int nchunks = p.nchunks;
     const bool tail_ragged = (p.n % lm.W) != 0;  // the last chunk of a row is partial
-    auto first_line = [&](int grp, int per_box) { return (int)(((long long)grp * R * p.n) / per_box); };
+    // flat boxes: the chunk of a row that holds its last n % line elements, if there are any (-1: none)
+    const int tail_chunk_in = (pipe.flat && p.n % CE::IN_LINE) ? (int)(p.n / CE::IN_LINE) * CE::IN_LINE / lm.W : -1;
+    const int tail_chunk_out = sizeof(TIn) == sizeof(TOut) ? tail_chunk_in  // same lines: one variable
+                               : (pipe.flat && p.n % CE::OUT_LINE) ? (int)(p.n / CE::OUT_LINE) * CE::OUT_LINE / lm.W : -1;
     // A ticket is drawn a few chunks before the end of the current group -- late, so that the groups go
     // to the warps that get there first, but early enough for the atomic's latency to stay off the path --
     // and stays in lane 0 until the warp needs it.  Without tickets a warp walks slot, slot + GW, ...
@@ -523,7 +549,6 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
     // producer cursor (TMA loads run S-1 chunks ahead)
     int pgroup = gw, pchunk = 0, pstage = 0;
     bool loading = true;  // the producer still has a row group
-    int pline = pipe.flat ? first_line(pgroup, Pipe::IN_PER_BOX) : 0;
     long long issued = 0, consumed = 0;
     auto issue_next = [&]() {
         if (TICKETS) {
@@ -534,23 +559,19 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
                     return;
                 }
                 enter_group(pgroup);
-                if (pipe.flat) pline = first_line(pgroup, Pipe::IN_PER_BOX);
             }
-            pipe.issue(&tm_a, &tm_b, pgroup * R, pchunk * lm.W, pline, pstage);
+            pipe.issue(&tm_a, &tm_b, pgroup * R, pchunk * lm.W, pstage);
             if (pchunk == draw_at) drawn = draw();
             ++issued;
-            pline += Pipe::IN_LINES;
             if (++pstage == S) pstage = 0;
             if (++pchunk == nchunks) pchunk = 0;
         } else {
-            pipe.issue(&tm_a, &tm_b, pgroup * R, pchunk * lm.W, pline, pstage);
+            pipe.issue(&tm_a, &tm_b, pgroup * R, pchunk * lm.W, pstage);
             ++issued;
-            pline += Pipe::IN_LINES;
             if (++pstage == S) pstage = 0;
             if (++pchunk == nchunks) {
                 pchunk = 0;
                 pgroup += GW;
-                if (pipe.flat && pgroup < groups) pline = first_line(pgroup, Pipe::IN_PER_BOX);
             }
             loading = issued < items;
         }
@@ -560,7 +581,6 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
     }
 
     int group = gw, chunk = 0, colbase = 0;
-    int oline = pipe.flat ? first_line(group, Pipe::OUT_PER_BOX) : 0;
     long long row = (long long)group * R + lm.g;
     bool group_ragged = (group + 1) * (long long)R > p.rows;
     E state = CE::row_start(p, row);
@@ -581,6 +601,10 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
         const uint32_t sm_a = pipe.in_a(stage);
         const uint32_t sm_b = pipe.in_b(stage);
         const uint32_t sm_out = pipe.out((int)(consumed & 1));
+        if (TMA && chunk == tail_chunk_in) {  // the box brought the row's whole lines; fetch the rest
+            CE::tail_load(p, sm_a, sm_b, lane, row, colbase);
+            __syncwarp();
+        }
         const int col0 = colbase + lm.i * K;
         const bool ragged = group_ragged || (tail_ragged && chunk == nchunks - 1);
 
@@ -593,8 +617,8 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
         renormalise(state);
 
         if (TMA) {
-            pipe.store_from(&tm_o, &tm_o1, group * R, colbase, oline, sm_out,
-                            ragged ? (int)((p.n - colbase) / Pipe::OUT_PER_BOX) : Pipe::OUT_LINES);
+            pipe.store_from(&tm_o, group * R, colbase, sm_out);
+            if (chunk == tail_chunk_out) CE::tail_store(p, sm_out, lane, row, colbase);
         } else {
             __syncwarp();
             CE::generic_store(p, sm_out, lm, lane, (long long)group * R, colbase);
@@ -604,7 +628,6 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
         if (!TMA && by_ticket && chunk == draw_at) drawn = draw();
 
         colbase += lm.W;
-        oline += Pipe::OUT_LINES;
         if (++chunk == nchunks) {
             chunk = 0;
             colbase = 0;
@@ -624,7 +647,6 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
             }
             row = (long long)group * R + lm.g;
             group_ragged = (group + 1) * (long long)R > p.rows;
-            if (pipe.flat) oline = first_line(group, Pipe::OUT_PER_BOX);
         }
         if (++stage == S) { stage = 0; parity ^= 1u; }
     }
@@ -912,7 +934,7 @@ struct TileCursor {
 template <int MODE, typename TIn, typename TOut, int K, bool TMA>
 __global__ void __launch_bounds__(512, 1)
 lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-                     const __grid_constant__ CUtensorMap tm_o, const __grid_constant__ CUtensorMap tm_o1) {
+                     const __grid_constant__ CUtensorMap tm_o) {
     using CE = ChunkEngine<MODE, TIn, TOut, K>;
     using LB = Lookback<MODE, TIn, TOut, K>;
     using R_ = Run<MODE, TIn, TOut, K>;
@@ -1033,7 +1055,10 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
     constexpr int IN_PER_BOX = 128 / (int)sizeof(TIn), OUT_PER_BOX = 128 / (int)sizeof(TOut);
     const int in_boxes = flat ? 1 : ST::IN_BYTES / 128;
     constexpr int OUT_LINES = (CHUNK * (int)sizeof(TOut)) / 128;
-    const int out_boxes = OUT_LINES;  // lanes that issue (or may issue) stores
+    const int out_boxes = flat ? 1 : OUT_LINES;  // lanes that issue stores
+    // flat boxes: first column of the chunk that holds the row's last n % line elements, if there are any
+    const int tail_colbase_in = (flat && p.n % CE::IN_LINE) ? (int)(p.n / CE::IN_LINE) * CE::IN_LINE / CHUNK * CHUNK : -1;
+    const int tail_colbase_out = (flat && p.n % CE::OUT_LINE) ? (int)(p.n / CE::OUT_LINE) * CE::OUT_LINE / CHUNK * CHUNK : -1;
 
     const int g_rows = (int)G / tpr, g_rem = (int)G % tpr;
     TileCursor ci, c1, c2;  // tiles being loaded, in phase 1, in phase 2
@@ -1051,9 +1076,8 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
             __syncwarp();
             if (flat) {
                 if (lane == 0) {
-                    const int line = (int)(((long long)ci.row * p.n + cb) / IN_PER_BOX);
-                    tma_load_2d(st_a(istage), &tm_a, 0, line, bar);
-                    tma_load_2d(st_b(istage), &tm_b, 0, line, bar);
+                    tma_load_3d(st_a(istage), &tm_a, 0, cb / IN_PER_BOX, ci.row, bar);
+                    tma_load_3d(st_b(istage), &tm_b, 0, cb / IN_PER_BOX, ci.row, bar);
                 }
             } else if (lane < in_boxes) {
                 const int x = cb + lane * IN_PER_BOX;
@@ -1091,6 +1115,10 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                     aborted = true;
                 } else {
                     ++consumed;
+                    if (colbase == tail_colbase_in) {  // the box brought the row's whole lines; fetch the rest
+                        CE::tail_load(p, st_a(st), st_b(st), lane, row, colbase);
+                        __syncwarp();
+                    }
                 }
             } else {
                 CE::generic_load(p, st_a(st), st_b(st), lm, lane, row, colbase);
@@ -1209,18 +1237,14 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                 if (TMA) {
                     fence_async_smem();
                     __syncwarp();
-                    // a flat box is not clipped per row: a chunk wholly beyond the row end stores nothing, the
-                    // partial last chunk of a row goes out line by line
+                    // a flat box holds the whole lines of the row that fall into the chunk (the hardware clips it
+                    // at the row's last whole line); what is left of the row goes out by plain stores
                     if (flat) {
-                        const long long rem = p.n - colbase;
-                        const int valid = rem >= CHUNK ? OUT_LINES : (rem > 0 ? (int)(rem / OUT_PER_BOX) : 0);
-                        const int line = (int)((row * p.n + colbase) / OUT_PER_BOX);
-                        if (valid >= OUT_LINES) {
-                            if (lane == 0) tma_store_2d(&tm_o, 0, line, pb);
-                        } else if (lane < valid) {
-                            tma_store_2d(&tm_o1, 0, line + lane, pb + (uint32_t)(lane * 128));
+                        if (lane == 0 && colbase < p.n) {
+                            tma_store_3d(&tm_o, 0, colbase / OUT_PER_BOX, (int)row, pb);
+                            bulk_commit();
                         }
-                        if (lane < OUT_LINES) bulk_commit();
+                        if (colbase == tail_colbase_out) CE::tail_store(p, pb, lane, row, colbase);
                     } else if (lane < out_boxes) {
                         tma_store_2d(&tm_o, colbase + lane * OUT_PER_BOX, (int)row, pb + (uint32_t)(lane * 128));
                         bulk_commit();

@@ -125,6 +125,14 @@ struct ChunkEngine<kPairs, TIn, TOut, K> {
                                                          long long row0, long long colbase) {
         Base::generic_store(p, sm_out, lm, lane, row0, colbase);
     }
+    static constexpr int IN_LINE = Base::IN_LINE, OUT_LINE = Base::OUT_LINE;
+    __device__ static __forceinline__ void tail_load(const Params& p, uint32_t sm_a, uint32_t sm_b, int lane, long long row,
+                                                     int colbase) {
+        Base::tail_load(p, sm_a, sm_b, lane, row, colbase);
+    }
+    __device__ static __forceinline__ void tail_store(const Params& p, uint32_t sm_out, int lane, long long row, int colbase) {
+        Base::tail_store(p, sm_out, lane, row, colbase);
+    }
 };
 
 }  // namespace hs

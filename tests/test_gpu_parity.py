@@ -160,6 +160,19 @@ def test_many_short_rows(hs, oracle, rows, n, cid):
         run_log(hs, oracle, w.tensors, path=hs.PATH_BATCHED, what=f"short rows {rows}x{n}")
 
 
+@pytest.mark.parametrize("rows,n,cid", [(1300, 2796, 2), (1500, 1060, 2), (40, 20004, 2), (3, 70004, 2), (1300, 1096, 5),
+                                         (2, 33000 + 8, 5), (1400, 2052, 4), (5, 9000 + 4, 4)])
+def test_rows_of_whole_lines_plus_a_remainder(hs, oracle, rows, n, cid):
+    """Row pitch a multiple of 16 bytes but not of 128: a chunk travels as one box of the row's whole 128-byte lines,
+    the remainder of the row by plain loads and stores; both kernels; neighbouring rows must stay untouched."""
+    w = workloads.make(cid, rows=rows, n=n, seed=rows * 7 + n)
+    for path in (hs.PATH_BATCHED, hs.PATH_LOOKBACK):
+        if cid == 4:
+            run_linear(hs, oracle, w.tensors, path=path, signed=True, what=f"lines+rest {rows}x{n}/{path}")
+        else:
+            run_log(hs, oracle, w.tensors, path=path, what=f"lines+rest {rows}x{n}/{path}")
+
+
 def test_tickets_forced_on_few_rows(hs, oracle, monkeypatch):
     monkeypatch.setenv("HEINSEN_SCAN_ROW_TICKETS", "1")
     for rows, n in ((5, 4100), (300, 515), (2400, 2048)):
