@@ -338,8 +338,9 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
                 if (best_cols < 0 || cols < best_cols) { best_cols = cols; best = r; }
             }
             R = best;
-        } else if (tma && p.rows >= (long long)kBatchedMinWarpsPerSm * dev.sm_count) {
-            // enough rows that TMA can address: one row per warp, each chunk one box of 128-byte lines
+        } else if (p.rows >= (long long)kBatchedMinWarpsPerSm * dev.sm_count) {
+            // enough rows: one row per warp, each chunk one TMA box of 128-byte lines (or, where TMA cannot
+            // address the rows, sixteen coalesced steps along one row instead of two along each of eight)
             R = 1;
         }
         R = env_int("HEINSEN_SCAN_ROWS_PER_WARP", R, 1, 16);
@@ -347,7 +348,9 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         p.rows_per_warp = R;
         p.nchunks = (int)((p.n + (32 / R) * ke.K - 1) / ((32 / R) * ke.K));
         const long long groups = (p.rows + R - 1) / R;
-        stages = tma ? 2 : 1;  // loads run one chunk ahead of the arithmetic (the kernel keeps one row group ahead)
+        // loads run one chunk ahead of the arithmetic (the kernel keeps one row group ahead): TMA boxes, or
+        // asynchronous 4-byte copies where TMA cannot address the rows; 2-byte elements are staged in step
+        stages = (tma || es_in == 4) ? 2 : 1;
         const int max_warps = 16;
         long long per_sm = (groups + dev.sm_count - 1) / dev.sm_count;
         warps = (int)(per_sm < 1 ? 1 : (per_sm > max_warps ? max_warps : per_sm));

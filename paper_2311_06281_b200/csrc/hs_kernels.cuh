@@ -289,26 +289,63 @@ struct ChunkEngine {
     __device__ static __forceinline__ E row_start(const Params& p, long long row) { return x0_elem(load_x0(p, row)); }
 
     // Plain-load staging for rows that TMA cannot address (unaligned base or row pitch).
-    // row0: first row of the warp's group, colbase: first column of the chunk.
+    // row0: first row of the warp's group, colbase: first column of the chunk.  Row by row of the group,
+    // 32 consecutive columns per step (one coalesced access), so that the row's base address and bounds
+    // are formed once per row and no division is left in the loop.
     __device__ static __forceinline__ void generic_load(const Params& p, uint32_t sm_a, uint32_t sm_b, const LaneMap& lm,
                                                         int lane, long long row0, long long colbase) {
-        for (int e = lane; e < 32 * K; e += 32) {
-            const int rg = e / lm.W, c = e - rg * lm.W;
-            const long long row = row0 + rg, col = colbase + c;
-            const bool in = row < p.rows && col < p.n;
-            const uint32_t off = chunk_off(lm.R, rg, (uint32_t)(c * sizeof(TIn)));
-            Storage<TIn>::to_smem(sm_a + off, in ? Storage<TIn>::load(p.in_a, row * p.n + col) : neutral_a<MODE>());
-            Storage<TIn>::to_smem(sm_b + off, in ? Storage<TIn>::load(p.in_b, row * p.n + col) : neutral_b<MODE>());
+#pragma unroll 1
+        for (int rg = 0; rg < lm.R; ++rg) {
+            const long long row = row0 + rg;
+            const long long base = row * p.n + colbase;
+            const long long left = row < p.rows ? p.n - colbase : 0;  // columns of the row from colbase on
+#pragma unroll 4
+            for (int c = lane; c < lm.W; c += 32) {
+                const bool in = c < left;
+                const uint32_t off = chunk_off(lm.R, rg, (uint32_t)(c * sizeof(TIn)));
+                Storage<TIn>::to_smem(sm_a + off, in ? Storage<TIn>::load(p.in_a, base + c) : neutral_a<MODE>());
+                Storage<TIn>::to_smem(sm_b + off, in ? Storage<TIn>::load(p.in_b, base + c) : neutral_b<MODE>());
+            }
         }
+    }
+    // The same as one group of asynchronous 4-byte copies, so that it can run a chunk ahead of the arithmetic
+    // like the TMA loads do (4-byte element types only).
+    static constexpr bool ASYNC_PLAIN = sizeof(TIn) == 4;
+    __device__ static __forceinline__ void generic_load_async(const Params& p, uint32_t sm_a, uint32_t sm_b,
+                                                              const LaneMap& lm, int lane, long long row0, long long colbase) {
+#pragma unroll 1
+        for (int rg = 0; rg < lm.R; ++rg) {
+            const long long row = row0 + rg;
+            const TIn* const pa = static_cast<const TIn*>(p.in_a) + (row * p.n + colbase);
+            const TIn* const pb = static_cast<const TIn*>(p.in_b) + (row * p.n + colbase);
+            const long long left = row < p.rows ? p.n - colbase : 0;
+#pragma unroll 4
+            for (int c = lane; c < lm.W; c += 32) {
+                const uint32_t off = chunk_off(lm.R, rg, (uint32_t)(c * sizeof(TIn)));
+                if (c < left) {
+                    cp_async4(sm_a + off, pa + c);
+                    cp_async4(sm_b + off, pb + c);
+                } else {
+                    Storage<TIn>::to_smem(sm_a + off, neutral_a<MODE>());
+                    Storage<TIn>::to_smem(sm_b + off, neutral_b<MODE>());
+                }
+            }
+        }
+        cp_async_commit();
     }
     __device__ static __forceinline__ void generic_store(const Params& p, uint32_t sm_out, const LaneMap& lm, int lane,
                                                          long long row0, long long colbase) {
-        for (int e = lane; e < 32 * K; e += 32) {
-            const int rg = e / lm.W, c = e - rg * lm.W;
-            const long long row = row0 + rg, col = colbase + c;
-            if (row < p.rows && col < p.n) {
-                const uint32_t off = chunk_off(lm.R, rg, (uint32_t)(c * sizeof(TOut)));
-                Storage<TOut>::store(p.out, row * p.n + col, Storage<TOut>::from_smem(sm_out + off));
+#pragma unroll 1
+        for (int rg = 0; rg < lm.R; ++rg) {
+            const long long row = row0 + rg;
+            const long long base = row * p.n + colbase;
+            const long long left = row < p.rows ? p.n - colbase : 0;
+#pragma unroll 4
+            for (int c = lane; c < lm.W; c += 32) {
+                if (c < left) {
+                    const uint32_t off = chunk_off(lm.R, rg, (uint32_t)(c * sizeof(TOut)));
+                    Storage<TOut>::store(p.out, base + c, Storage<TOut>::from_smem(sm_out + off));
+                }
             }
         }
     }
@@ -459,7 +496,9 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align_1024(smem_raw);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    const int S = TMA ? p.stages : 1;
+    // loads run ahead of the arithmetic: TMA boxes, or groups of asynchronous 4-byte copies
+    constexpr bool AHEAD = TMA || CE::ASYNC_PLAIN;
+    const int S = AHEAD ? p.stages : 1;
     const int per_warp = warp_smem_bytes<MODE, TIn, TOut, K>(S);
     const int R = p.rows_per_warp;
 
@@ -546,10 +585,14 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
         qa_group = g;
     };
 
-    // producer cursor (TMA loads run S-1 chunks ahead)
+    // producer cursor (the loads run S-1 chunks ahead)
     int pgroup = gw, pchunk = 0, pstage = 0;
     bool loading = true;  // the producer still has a row group
     long long issued = 0, consumed = 0;
+    auto issue_chunk = [&]() {
+        if (TMA) pipe.issue(&tm_a, &tm_b, pgroup * R, pchunk * lm.W, pstage);
+        else CE::generic_load_async(p, pipe.in_a(pstage), pipe.in_b(pstage), lm, lane, (long long)pgroup * R, pchunk * lm.W);
+    };
     auto issue_next = [&]() {
         if (TICKETS) {
             if (pchunk == 0 && issued != 0) {  // the previous group is complete: enter the next one
@@ -560,13 +603,13 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
                 }
                 enter_group(pgroup);
             }
-            pipe.issue(&tm_a, &tm_b, pgroup * R, pchunk * lm.W, pstage);
+            issue_chunk();
             if (pchunk == draw_at) drawn = draw();
             ++issued;
             if (++pstage == S) pstage = 0;
             if (++pchunk == nchunks) pchunk = 0;
         } else {
-            pipe.issue(&tm_a, &tm_b, pgroup * R, pchunk * lm.W, pstage);
+            issue_chunk();
             ++issued;
             if (++pstage == S) pstage = 0;
             if (++pchunk == nchunks) {
@@ -576,7 +619,7 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
             loading = issued < items;
         }
     };
-    if (TMA) {
+    if (AHEAD) {
         for (int s = 0; s < S - 1 && loading; ++s) issue_next();
     }
 
@@ -594,6 +637,12 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
                 pipe.drain_loads(consumed + 1, issued);
                 break;
             }
+        } else if (AHEAD) {
+            if (loading) issue_next();
+            // this chunk's group of copies is the oldest one pending; at most one newer group is in flight
+            if (issued - consumed > 1) cp_async_wait<1>();
+            else cp_async_wait<0>();
+            __syncwarp();
         } else {
             CE::generic_load(p, pipe.in_a(0), pipe.in_b(0), lm, lane, (long long)group * R, colbase);
             __syncwarp();
@@ -625,14 +674,14 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
         }
         __syncwarp();  // every lane is done with this input stage
         ++consumed;
-        if (!TMA && by_ticket && chunk == draw_at) drawn = draw();
+        if (!AHEAD && by_ticket && chunk == draw_at) drawn = draw();
 
         colbase += lm.W;
         if (++chunk == nchunks) {
             chunk = 0;
             colbase = 0;
             if (by_ticket) {
-                if (!TMA) {  // no loads ahead: the arithmetic enters the next group itself
+                if (!AHEAD) {  // no loads ahead: the arithmetic enters the next group itself
                     const int g = take(drawn);
                     if (g < groups) enter_group(g);
                 }
@@ -1068,28 +1117,36 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
     auto colbase_of = [&](const TileCursor& c) { return (c.j * W + warp) * CHUNK; };
     long long issued = 0;
     int istage = 0;
+    // loads run a tile ahead of phase 1: TMA boxes, or groups of asynchronous 4-byte copies
+    constexpr bool AHEAD = TMA || CE::ASYNC_PLAIN;
     auto issue_next = [&]() {
         if (issued < my_tiles) {
             const int cb = colbase_of(ci);
             const uint32_t bar = bars + 8 * istage;
-            if (lane == 0) mbar_expect_tx(bar, 2 * ST::IN_BYTES);
-            __syncwarp();
-            if (flat) {
+            if (!TMA) {
+                CE::generic_load_async(p, st_a(istage), st_b(istage), lm, lane, ci.row, cb);
+            } else if (flat) {
+                if (lane == 0) mbar_expect_tx(bar, 2 * ST::IN_BYTES);
+                __syncwarp();
                 if (lane == 0) {
                     tma_load_3d(st_a(istage), &tm_a, 0, cb / IN_PER_BOX, ci.row, bar);
                     tma_load_3d(st_b(istage), &tm_b, 0, cb / IN_PER_BOX, ci.row, bar);
                 }
-            } else if (lane < in_boxes) {
-                const int x = cb + lane * IN_PER_BOX;
-                tma_load_2d(st_a(istage) + lane * 128, &tm_a, x, ci.row, bar);
-                tma_load_2d(st_b(istage) + lane * 128, &tm_b, x, ci.row, bar);
+            } else {
+                if (lane == 0) mbar_expect_tx(bar, 2 * ST::IN_BYTES);
+                __syncwarp();
+                if (lane < in_boxes) {
+                    const int x = cb + lane * IN_PER_BOX;
+                    tma_load_2d(st_a(istage) + lane * 128, &tm_a, x, ci.row, bar);
+                    tma_load_2d(st_b(istage) + lane * 128, &tm_b, x, ci.row, bar);
+                }
             }
             ++issued;
             if (++istage == S) istage = 0;
             ci.advance((int)G, g_rows, g_rem, tpr);
         }
     };
-    if (TMA) issue_next();
+    if (AHEAD) issue_next();
 
     bool aborted = false;
     long long consumed = 0;
@@ -1120,6 +1177,14 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                         __syncwarp();
                     }
                 }
+            } else if (AHEAD) {
+                // (the tile that left this stage was stored by plain stores, which are done)
+                issue_next();
+                // this tile's group of copies is the oldest one pending; at most one newer group is in flight
+                if (issued - consumed > 1) cp_async_wait<1>();
+                else cp_async_wait<0>();
+                __syncwarp();
+                ++consumed;
             } else {
                 CE::generic_load(p, st_a(st), st_b(st), lm, lane, row, colbase);
                 __syncwarp();

@@ -125,6 +125,11 @@ struct ChunkEngine<kPairs, TIn, TOut, K> {
                                                          long long row0, long long colbase) {
         Base::generic_store(p, sm_out, lm, lane, row0, colbase);
     }
+    static constexpr bool ASYNC_PLAIN = Base::ASYNC_PLAIN;
+    __device__ static __forceinline__ void generic_load_async(const Params& p, uint32_t sm_a, uint32_t sm_b,
+                                                              const LaneMap& lm, int lane, long long row0, long long colbase) {
+        Base::generic_load_async(p, sm_a, sm_b, lm, lane, row0, colbase);
+    }
     static constexpr int IN_LINE = Base::IN_LINE, OUT_LINE = Base::OUT_LINE;
     __device__ static __forceinline__ void tail_load(const Params& p, uint32_t sm_a, uint32_t sm_b, int lane, long long row,
                                                      int colbase) {
