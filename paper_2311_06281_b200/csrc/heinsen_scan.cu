@@ -139,7 +139,6 @@ struct Problem {
     bool tma;
 };
 
-using BatchedFn = void (*)(const Params, const CUtensorMap, const CUtensorMap, const CUtensorMap);
 
 struct KernelEntry {
     const void* batched;      // row groups stay with their warp slots

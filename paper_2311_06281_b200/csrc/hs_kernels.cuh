@@ -1,14 +1,16 @@
 // Kernels of libheinsen_scan (sm_100a only).
 //
-//   batched_scan_kernel  : one warp walks one row chunk by chunk, the value of x carried in
-//                          registers from chunk to chunk (rows >= a few per SM).
+//   batched_scan_kernel  : a warp walks one row (or 2-16 rows shorter than a chunk) chunk by chunk,
+//                          the value of x carried in registers from chunk to chunk (rows >= a few
+//                          per SM); rows are handed out to the warps by slot or by ticket.
 //   lookback_scan_kernel : rows are cut into tiles of WARPS chunks; one CTA per tile, single
 //                          pass, the carry between tiles found by decoupled look-back over
 //                          per-tile descriptors in the caller's workspace (few, long rows).
 //
 // Both read every input element once and write every output element once.  Chunks travel
 // HBM -> shared memory by TMA (per-warp mbarrier pipelines, 128-byte swizzle) and back by TMA
-// stores; the scans themselves run in registers (hs_device.cuh).
+// stores -- or, for rows that TMA cannot address, by asynchronous 4-byte copies and plain stores --;
+// the scans themselves run in registers (hs_device.cuh).
 #pragma once
 #include <cuda.h>
 
