@@ -424,6 +424,33 @@ def test_short_forms_of_the_two_calls(hs, oracle):
     assert_log_close(to_f64(out), ref, tol_positive(w.tensors["log_a"].astype(np.float64), ref), "scan_log short form")
 
 
+def test_two_streams_with_their_own_workspaces(hs):
+    """Calls on two streams may overlap on the GPU; each has its own workspace (ticket word, descriptors)."""
+    shapes = [(20000, 2048, 2), (3, 300000, 2), (9000, 4096, 2), (1, 1 << 20, 2)]
+    data = []
+    for rows, n, cid in shapes:
+        t = workloads.make(cid, rows=rows, n=n, seed=rows).tensors
+        la, lb, lx0 = to_dev(t["log_a"]), to_dev(t["log_b"]), to_dev(t["log_x0"])
+        ws = hs.new_workspace(rows, n, "cuda")
+        ref = hs.scan_log(la, lb, lx0, workspace=ws)
+        hs.check(ws)
+        data.append((la, lb, lx0, ref.clone()))
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    outs, wss = [], []
+    for rep in range(3):
+        for k, (la, lb, lx0, ref) in enumerate(data):
+            with torch.cuda.stream(streams[k % 2]):
+                ws = hs.new_workspace(la.shape[0], la.shape[1], "cuda")
+                outs.append((hs.scan_log(la, lb, lx0, workspace=ws), ref))
+                wss.append(ws)
+    torch.cuda.synchronize()
+    for ws in wss:
+        hs.check(ws)
+    for out, ref in outs:
+        assert torch.equal(out, ref)
+
+
 def test_repeatability(hs):
     w = workloads.make(3, rows=1, n=1 << 21)
     la, lb, lx0 = (to_dev(w.tensors[k]) for k in ("log_a", "log_b", "log_x0"))
