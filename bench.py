@@ -30,7 +30,7 @@ UNIT = "elements/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (None until a capture of that workload exists).
-NCU_TRAFFIC_BYTES = {2: 362.2e6, 3: 664.7e6, 4: 371.8e6, 5: 3024.0e6}  # cfg3, cfg5: small-case captures scaled (see profiles/)
+NCU_TRAFFIC_BYTES = {2: 364.2e6, 3: 659.6e6, 4: 371.8e6, 5: 3007.0e6}  # cfg3, cfg5: small-case captures scaled (see profiles/)
 
 HBM_FALLBACK_GBS = 6650.0  # used only when MEASURED_PEAKS.json is absent
 
