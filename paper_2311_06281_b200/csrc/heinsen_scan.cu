@@ -822,12 +822,14 @@ static hs_status host_run(int linear, const void* a, const void* b, const void* 
         e = (call);                                           \
         if (e != cudaSuccess) return cuda_fail(#call, e);     \
     } while (0)
+    // x_0 of all rows goes first, in one copy, on the caller's stream
+    HS_TRY(cudaMemcpyAsync(d_x0, x0, (size_t)rows * es_in, cudaMemcpyHostToDevice, stream));
+    if (sx0) HS_TRY(cudaMemcpyAsync(d_sx0, sx0, (size_t)rows, cudaMemcpyHostToDevice, stream));
     // the side streams start after everything already queued on the caller's stream
     HS_TRY(cudaEventRecord(hl->start, stream));
     HS_TRY(cudaStreamWaitEvent(hl->side[0], hl->start, 0));
     HS_TRY(cudaStreamWaitEvent(hl->side[1], hl->start, 0));
-    const uint8_t *ha = static_cast<const uint8_t*>(a), *hb = static_cast<const uint8_t*>(b),
-                  *hx0 = static_cast<const uint8_t*>(x0);
+    const uint8_t *ha = static_cast<const uint8_t*>(a), *hb = static_cast<const uint8_t*>(b);
     uint8_t* hx = static_cast<uint8_t*>(x);
     for (int k = 0; k < nblk; ++k) {
         const int64_t r0 = (int64_t)k * rows_blk;
@@ -837,11 +839,8 @@ static hs_status host_run(int linear, const void* a, const void* b, const void* 
         const size_t e0 = (size_t)r0 * (size_t)n, ec = (size_t)rb * (size_t)n;
         HS_TRY(cudaMemcpyAsync(d_a + e0 * es_in, ha + e0 * es_in, ec * es_in, cudaMemcpyHostToDevice, s));
         HS_TRY(cudaMemcpyAsync(d_b + e0 * es_in, hb + e0 * es_in, ec * es_in, cudaMemcpyHostToDevice, s));
-        HS_TRY(cudaMemcpyAsync(d_x0 + (size_t)r0 * es_in, hx0 + (size_t)r0 * es_in, (size_t)rb * es_in,
-                               cudaMemcpyHostToDevice, s));
         if (sa) HS_TRY(cudaMemcpyAsync(d_sa + e0, sa + e0, ec, cudaMemcpyHostToDevice, s));
         if (sb) HS_TRY(cudaMemcpyAsync(d_sb + e0, sb + e0, ec, cudaMemcpyHostToDevice, s));
-        if (sx0) HS_TRY(cudaMemcpyAsync(d_sx0 + r0, sx0 + r0, (size_t)rb, cudaMemcpyHostToDevice, s));
         void* ws = ws0 + (size_t)k * up256(ws_bytes);
         if (linear)
             st = heinsen_scan_linear(d_a + e0 * es_in, d_b + e0 * es_in, d_x0 + (size_t)r0 * es_in, d_x + e0 * es_out, rb, n,
@@ -859,9 +858,17 @@ static hs_status host_run(int linear, const void* a, const void* b, const void* 
         HS_TRY(cudaStreamWaitEvent(stream, hl->done[i], 0));
     }
 #undef HS_TRY
+    // one synchronisation and one strided read-back of the row blocks' status words
+    e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) return cuda_fail("cudaStreamSynchronize", e);
+    Header heads[kHostBlocks];
+    e = cudaMemcpy2D(heads, sizeof(Header), ws0, up256(ws_bytes), sizeof(Header), (size_t)nblk, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail("cudaMemcpy2D", e);
     for (int k = 0; k < nblk; ++k) {
-        st = heinsen_scan_check(ws0 + (size_t)k * up256(ws_bytes), stream);
-        if (st != HS_OK) return st;
+        const Header& h = heads[k];
+        if (h.error_id == h.started_id && h.started_id != 0 &&
+            (h.error_code == HS_ERR_LOOKBACK_TIMEOUT || h.error_code == HS_ERR_COPY_TIMEOUT))
+            return static_cast<hs_status>(h.error_code);
     }
     return HS_OK;
 }

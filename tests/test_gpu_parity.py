@@ -371,6 +371,28 @@ def test_host_buffer_entry_point(hs, oracle):
     assert_log_close(out.double().numpy(), ref, tol_positive(t["log_a"].astype(np.float64), ref), "host entry")
 
 
+def test_host_buffer_entry_points_signed_and_linear(hs, oracle):
+    """Host buffers with sign tensors (log domain) and the linear entry point, more rows than row blocks."""
+    rows, n = 37, 1500
+    t = workloads.make(4, rows=rows, n=n, seed=9).tensors
+    a, b, x0 = (torch.from_numpy(t[k]).pin_memory() for k in ("a", "b", "x0"))
+    x = torch.empty_like(a).pin_memory()
+    scratch = torch.empty(hs.host_scratch_bytes(rows, n, torch.float32, torch.float32, True), dtype=torch.uint8, device="cuda")
+    hs.scan_linear_host(a, b, x0, x, scratch)
+    ref = oracle.scan_linear(t["a"], t["b"], t["x0"])
+    assert_signed_close(x.double().numpy(), ref, "host linear")
+    # the same recurrence handed over as logarithms of magnitudes and sign bytes
+    with np.errstate(divide="ignore"):
+        la, lb, lx0 = (torch.from_numpy(np.log(np.abs(t[k])).astype(np.float32)).pin_memory() for k in ("a", "b", "x0"))
+    sa, sb, sx0 = (torch.from_numpy(np.signbit(t[k]).astype(np.uint8)).pin_memory() for k in ("a", "b", "x0"))
+    lx = torch.empty_like(la).pin_memory()
+    sx = torch.empty((rows, n), dtype=torch.uint8).pin_memory()
+    hs.scan_log_host(la, lb, lx0, lx, scratch, sign_a=sa, sign_b=sb, sign_x0=sx0, sign_x=sx)
+    got = np.exp(lx.double().numpy()) * np.where(sx.numpy() == 1, -1.0, 1.0)
+    ref_log, ref_sign = oracle.scan_log(la.numpy(), lb.numpy(), lx0.numpy(), sa.numpy(), sb.numpy(), sx0.numpy())
+    assert_signed_close(got, np.exp(ref_log) * np.where(ref_sign == 1, -1.0, 1.0), "host log with signs")
+
+
 def test_lookback_several_rows_several_groups(hs, oracle):
     """Look-back path with a few rows, each several descriptor groups long (a group is one wave of tiles),
     plus a ragged last tile: exercises group aggregates, group values and the row start inside a launch."""
