@@ -446,6 +446,26 @@ def test_short_forms_of_the_two_calls(hs, oracle):
     assert_log_close(to_f64(out), ref, tol_positive(w.tensors["log_a"].astype(np.float64), ref), "scan_log short form")
 
 
+@pytest.mark.parametrize("seed", range(10))
+def test_random_shapes_all_modes(hs, oracle, seed):
+    """Seeded random shapes (short and long rows, few and many, aligned and not) through every mode and both kernels."""
+    rng = np.random.default_rng(1000 + seed)
+    for _ in range(5):
+        n = int(rng.choice([rng.integers(1, 40), rng.integers(40, 700), rng.integers(700, 6000), rng.integers(6000, 40000)]))
+        if rng.random() < 0.5:
+            n = max(4, n // 4 * 4)  # a pitch that TMA can address
+        rows = int(rng.choice([rng.integers(1, 8), rng.integers(8, 400), rng.integers(400, 6000)]))
+        rows = max(1, min(rows, 3_000_000 // n))
+        cid = int(rng.choice([2, 4, 5]))
+        w = workloads.make(cid, rows=rows, n=n, seed=seed)
+        for path in (hs.PATH_BATCHED, hs.PATH_LOOKBACK):
+            what = f"random cfg{cid} {rows}x{n}/{path}"
+            if cid == 4:
+                run_linear(hs, oracle, w.tensors, path=path, signed=True, what=what)
+            else:
+                run_log(hs, oracle, w.tensors, path=path, what=what)
+
+
 def test_two_streams_with_their_own_workspaces(hs):
     """Calls on two streams may overlap on the GPU; each has its own workspace (ticket word, descriptors)."""
     shapes = [(20000, 2048, 2), (3, 300000, 2), (9000, 4096, 2), (1, 1 << 20, 2)]
