@@ -2,21 +2,33 @@
 """Benchmark of the fused recurrence scan (one JSON line on stdout).
 
 A "step" is one pass of the whole hot path -- one call of the C ABI on one batch of seeded
-synthetic input.  Default workload: configuration 2 of the benchmark contract (16384 rows x 2048
-steps, fp32, log-space inputs of a linear-RNN layer), the configuration the headline metric is
-quoted on.  `value` is elements/s with the inputs resident in HBM; `e2e` is the same metric through
-the host-buffer entry point with pinned host buffers and both copies inside the timed region.
+synthetic input.  Headline workload: configuration 2 of the benchmark contract (16384 rows x 2048
+steps, fp32, log-space inputs of a linear-RNN layer), the configuration the metric is quoted on.
+`value` is elements/s with the inputs resident in HBM; `e2e` is the same metric through the
+host-buffer entry point with pinned host buffers and both copies inside the timed region.
+
+The same line carries, under `workloads`, one record per benchmark configuration measured in the same
+process (both kernels: the row-batched one on configurations 2, 4, 5, the look-back one on
+configuration 3 and its linear / bf16 variants, the call latency of configuration 1), each with
+median / min / mean time per step over repeated batches, the clocks sampled meanwhile, and a
+two-legged roofline: algorithmic bytes at the measured HBM copy bandwidth against algorithmic
+transcendentals at the MUFU rate that a register-only probe kernel measures in the same run.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 2|3|4|5] [--impl reference]
+                  [--only-headline] [--fig1] [--ablation unfused|pairs]
 
-N > 1 is launched by torchrun (one rank per GPU); rows are independent, so every rank runs its own
-batch (weak scaling) and the only communication is the barrier and the max-over-ranks of the time.
+N > 1: one rank per GPU (launched by torchrun, or spawned from here when the torchrun environment is
+absent); rows are independent, so every rank runs its own batch (weak scaling) and the only
+communication is the barrier and the max-over-ranks of the time.
 """
 from __future__ import annotations
 
 import argparse
+import ctypes
 import json
 import os
+import socket
+import subprocess
 import sys
 import threading
 import time
@@ -27,12 +39,11 @@ if ROOT not in sys.path:
 
 METRIC = "recurrence_elements_per_s"
 UNIT = "elements/s"
-
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# captures summarised under profiles/ (None until a capture of that workload exists).
-NCU_TRAFFIC_BYTES = {2: 364.2e6, 3: 659.6e6, 4: 371.8e6, 5: 3007.0e6}  # cfg3, cfg5: small-case captures scaled (see profiles/)
-
-HBM_FALLBACK_GBS = 6650.0  # used only when MEASURED_PEAKS.json is absent
+ARITHMETIC = "f32"            # every kernel computes in fp32 whatever the storage type
+HBM_FALLBACK_GBS = 6650.0     # used only when MEASURED_PEAKS.json is absent
+NOMINAL_HBM_GBS = 8000.0      # the figure the benchmark contract quotes for B200
+MIN_TIMED_SECONDS = 0.15      # per record: long enough for a few dozen clock samples
+MIN_REPEATS = 10
 
 
 def parse_args():
@@ -40,10 +51,15 @@ def parse_args():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--workload", type=int, default=2, choices=[2, 3, 4, 5])
+    ap.add_argument("--workload", type=int, default=2, choices=[2, 3, 4, 5], help="headline workload")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--rows", type=int, default=None, help="override the workload's rows (profiling of small cases)")
     ap.add_argument("--n", type=int, default=None, help="override the workload's n (profiling of small cases)")
+    ap.add_argument("--variant", default=None, choices=["linear", "bf16"],
+                    help="with --workload 3: time the linear entry point / bf16 storage on the same sequence")
+    ap.add_argument("--only-headline", action="store_true",
+                    help="skip the per-configuration records, the MUFU probe, the end-to-end leg and the CPU baselines "
+                         "(profiling runs)")
     ap.add_argument("--fig1", action="store_true",
                     help="the paper's only experiment: sequential (CPU oracle, one core) over parallel (this library) "
                          "time for one sequence of n = 2^10..2^28 elements, means of 30 runs; prints one JSON object")
@@ -54,36 +70,39 @@ def parse_args():
                          "scan_linear on the signed linear workload (cfg4)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-workloads", action="store_true", help="headline record only (keeps e2e and CPU baseline)")
     return ap.parse_args()
 
 
 def measured_peak():
     try:
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
-            return float(json.load(f)["hbm_gbs"]), "measured"
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
     except Exception:
-        return HBM_FALLBACK_GBS, "fallback"
+        return HBM_FALLBACK_GBS, "fallback (no MEASURED_PEAKS.json)"
 
 
-def bytes_per_element(w) -> int:
-    es = 4 if w.storage == "f32" else 2
-    return 3 * es  # two inputs read once, one output written once
-
-
-def workload_name(cid, w):
-    return f"cfg{cid}: {w.name} ({w.rows} rows x n={w.n}, {'scan_linear' if w.kind == 'linear' else 'scan_log'}, {w.storage} storage)"
+def ncu_traffic():
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of each workload's kernel, as summarised from the
+    ncu captures under profiles/ (absent workload: None)."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.json")) as f:
+            return json.load(f)
+    except Exception:
+        return {}
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons of one GPU through NVML while a timed region runs."""
+    """Samples SM clock, power and throttle reasons of one GPU through NVML while a timed region runs."""
     REASONS = {
         0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
         0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
         0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting",
     }
 
-    def __init__(self, index: int):
-        self.samples, self.reasons, self.max_mhz = [], set(), None
+    def __init__(self, index: int, period_s: float = 0.003):
+        self.samples, self.reasons, self.max_mhz, self.power = [], set(), None, []
+        self.period = period_s
         self._stop = threading.Event()
         self._thread = None
         try:
@@ -111,17 +130,240 @@ class ClockSampler:
         def loop():
             while not self._stop.is_set():
                 self.sample()
-                time.sleep(0.005)
+                time.sleep(self.period)
         self._thread = threading.Thread(target=loop, daemon=True)
         self._thread.start()
+        return self
 
     def stop(self):
         self._stop.set()
         if self._thread:
             self._thread.join()
         s = sorted(self.samples)
-        return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-                "samples": len(s)}
+        return {"sm_mhz": s[len(s) // 2] if s else None, "sm_mhz_min": s[0] if s else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(s)}
+
+
+# ---------------------------------------------------------------------------------------------- workloads
+def describe(cid, w, variant=None):
+    call = "scan_linear" if w.kind == "linear" else "scan_log"
+    extra = f", variant {variant}" if variant else ""
+    return f"cfg{cid}: {w.name} ({w.rows} rows x n={w.n}, {call}, {w.storage} storage{extra})"
+
+
+def make_workload(cid, variant=None, rows=None, n=None, seed=0):
+    """Configuration `cid`, or one of configuration 3's variants: 'linear' = the linear entry point on
+    a = fp32(exp(log_a)), b, x0 = 0.5; 'bf16' = the same log-space sequence stored in bf16."""
+    from paper_2311_06281_b200 import workloads
+    w = workloads.make(cid, rows=rows, n=n, seed=seed)
+    if variant == "linear":
+        assert cid == 3
+        w.kind = "linear"
+    elif variant == "bf16":
+        assert cid == 3
+        for k in ("log_a", "log_b", "log_x0"):
+            w.tensors[k] = workloads.to_bf16_bits(w.tensors[k].astype("float64")).reshape(w.tensors[k].shape)
+        w.storage = "bf16"
+    return w
+
+
+def input_keys(w):
+    return ("a", "b", "x0") if w.kind == "linear" else ("log_a", "log_b", "log_x0")
+
+
+def mufu_per_element(w):
+    """Algorithmic transcendentals per element: scan_log one ex2 for the scan and one lg2 for the output;
+    scan_linear two logarithms on the way in, one ex2 for the scan and one for the output."""
+    return 4 if w.kind == "linear" else 2
+
+
+def algorithmic_bytes(w):
+    es = 4 if w.storage == "f32" else 2
+    return w.rows * w.n * 3 * es + w.rows * es   # two inputs read once, one output written once, x0
+
+
+class DeviceWorkload:
+    """A workload resident on the device in `nsets` rotating buffer sets, each larger than L2."""
+
+    def __init__(self, w, dev, hs, nsets=3):
+        import numpy as np
+        import torch
+        self.w, self.hs, self.nsets = w, hs, nsets
+
+        def dev_tensor(arr):
+            x = torch.from_numpy(np.ascontiguousarray(arr))
+            if arr.dtype == np.uint16:
+                x = x.view(torch.bfloat16)
+            return x.to(dev)
+
+        base = [dev_tensor(w.tensors[k]) for k in input_keys(w)]
+        self.sets = [base] + [[x.clone() for x in base] for _ in range(nsets - 1)]
+        self.outs = [torch.empty((w.rows, w.n), dtype=base[0].dtype, device=dev) for _ in range(nsets)]
+        self.wss = [hs.new_workspace(w.rows, w.n, dev) for _ in range(nsets)]
+
+    def step(self, i):
+        s, hs = i % self.nsets, self.hs
+        if self.w.kind == "linear":
+            hs.scan_linear(*self.sets[s], x=self.outs[s], workspace=self.wss[s])
+        else:
+            hs.scan_log(*self.sets[s], log_x=self.outs[s], workspace=self.wss[s])
+
+    def check(self):
+        for ws in self.wss:
+            self.hs.check(ws)
+
+
+def timed_batches(dw, steps, repeats, local, torch):
+    """`repeats` batches of `steps` steps back to back, an event between batches; returns the per-step time of
+    every batch (ms) and the clocks sampled meanwhile."""
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(repeats + 1)]
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local).start()
+    k = 0
+    ev[0].record()
+    for r in range(repeats):
+        for _ in range(steps):
+            dw.step(k)
+            k += 1
+        ev[r + 1].record()
+    sampler.sample()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    per_step = [ev[r].elapsed_time(ev[r + 1]) / steps for r in range(repeats)]
+    return per_step, clocks
+
+
+def roofline_record(w, us_per_step, clocks, peak, peak_source, mufu_rate, kernel, traffic):
+    """Two legs: bytes at the measured HBM bandwidth, transcendentals at the measured MUFU rate at the clock
+    sampled during the run; the slower one is the roofline."""
+    elements = w.rows * w.n
+    alg_bytes = algorithmic_bytes(w)
+    t_hbm = alg_bytes / (peak * 1e9) * 1e6
+    achieved = alg_bytes / (us_per_step * 1e-6) / 1e9
+    rec = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": t_hbm / us_per_step,
+           "traffic": traffic, "peak_source": peak_source, "kernel": kernel,
+           "algorithmic_bytes_per_launch": alg_bytes, "bytes_per_element": 3 * (4 if w.storage == "f32" else 2),
+           "hbm": {"time_us": t_hbm, "frac": t_hbm / us_per_step},
+           "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS}
+    if mufu_rate and clocks.get("sm_mhz"):
+        ops = mufu_per_element(w)
+        peak_ops = mufu_rate["results_per_clk_per_sm"] * mufu_rate["sm_count"] * clocks["sm_mhz"] * 1e6
+        t_mufu = elements * ops / peak_ops * 1e6
+        rec["mufu"] = {"ops_per_element": ops, "peak_ops_per_s": peak_ops, "at_sm_mhz": clocks["sm_mhz"],
+                       "time_us": t_mufu, "frac": t_mufu / us_per_step}
+        if t_mufu > t_hbm:   # the transcendental leg is the slower one: report against it
+            rec.update(bound="mufu", achieved=elements * ops / (us_per_step * 1e-6) / 1e12, peak=peak_ops / 1e12,
+                       unit="Tops/s", frac=t_mufu / us_per_step)
+    return rec
+
+
+def stats(values):
+    s = sorted(values)
+    return {"median": s[len(s) // 2], "min": s[0], "mean": sum(s) / len(s), "max": s[-1]}
+
+
+def measure_record(cid, variant, dev, local, hs, args, peak, peak_source, mufu_rate, torch):
+    """One record of `workloads`: build the configuration, warm up, time repeated batches."""
+    w = make_workload(cid, variant)
+    dw = DeviceWorkload(w, dev, hs)
+    for i in range(max(args.warmup, 3)):
+        dw.step(i)
+    torch.cuda.synchronize()
+    dw.check()
+    kernel = "batched_scan_kernel" if hs.last_path() == hs.PATH_BATCHED else "lookback_scan_kernel"
+    # a first short batch sizes the run: at least MIN_REPEATS batches and MIN_TIMED_SECONDS of device time
+    probe, _ = timed_batches(dw, max(3, min(args.steps, 10)), 1, local, torch)
+    steps = max(3, args.steps if cid == 2 else min(args.steps, 100))
+    repeats = max(MIN_REPEATS, int(MIN_TIMED_SECONDS / (probe[0] * 1e-3 * steps)) + 1)
+    per_step_ms, clocks = timed_batches(dw, steps, repeats, local, torch)
+    dw.check()
+    st = stats([1e3 * v for v in per_step_ms])
+    key = f"cfg{cid}" + (f"_{variant}" if variant else "")
+    traffic = ncu_traffic().get(key)
+    rec = {"workload": describe(cid, w, variant), "kernel": kernel, "elements_per_s": w.rows * w.n / (st["median"] * 1e-6),
+           "us_per_step": st, "repeats": repeats, "steps_per_repeat": steps, "timed_launches": repeats * steps,
+           "clocks": clocks, "us_times_sm_ghz": st["median"] * (clocks["sm_mhz"] or 0) * 1e-3,
+           "roofline": roofline_record(w, st["median"], clocks, peak, peak_source, mufu_rate, kernel,
+                                       traffic["bytes"] if traffic else None)}
+    if traffic:
+        rec["roofline"]["traffic_source"] = traffic.get("source")
+    del dw
+    torch.cuda.empty_cache()
+    return rec, w
+
+
+def measure_small_call(dev, hs, torch):
+    """Configuration 1 (one sequence of 4096 elements) is bound by the cost of a call, not by bytes: time the
+    C ABI itself -- pre-marshalled arguments, no tensor wrapping -- back to back, and one call plus its
+    synchronisation."""
+    w = make_workload(1)
+    t = w.tensors
+    a, b, x0 = (torch.from_numpy(t[k]).to(dev) for k in ("a", "b", "x0"))
+    x = torch.empty_like(a)
+    ws = hs.new_workspace(w.rows, w.n, dev)
+    L = hs.lib()
+    vp = ctypes.c_void_p
+    argv = (vp(a.data_ptr()), vp(b.data_ptr()), vp(x0.data_ptr()), vp(x.data_ptr()), w.rows, w.n, hs.HS_F32,
+            vp(ws.data_ptr()), ws.numel(), vp(torch.cuda.current_stream(dev).cuda_stream))
+    fn = L.heinsen_scan_linear
+    for _ in range(20):
+        assert fn(*argv) == 0
+    torch.cuda.synchronize()
+    runs = []
+    for _ in range(10):
+        calls = 300
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.perf_counter()
+        e0.record()
+        for _ in range(calls):
+            fn(*argv)
+        e1.record()
+        host_us = (time.perf_counter() - t0) / calls * 1e6
+        torch.cuda.synchronize()
+        runs.append((e0.elapsed_time(e1) * 1e3 / calls, host_us))
+    lat = []
+    for _ in range(30):
+        t0 = time.perf_counter()
+        fn(*argv)
+        torch.cuda.synchronize()
+        lat.append((time.perf_counter() - t0) * 1e6)
+    hs.check(ws)
+    dev_us = stats([r[0] for r in runs])
+    return {"workload": describe(1, w), "kernel": "lookback_scan_kernel (one tile)" if hs.last_path() == hs.PATH_LOOKBACK
+            else "batched_scan_kernel",
+            "us_per_call_back_to_back": dev_us, "host_us_per_call": stats([r[1] for r in runs])["median"],
+            "us_call_plus_sync": stats(lat), "calls_per_batch": 300, "batches": 10,
+            "elements_per_s": w.rows * w.n / (dev_us["median"] * 1e-6),
+            "note": "latency-bound: 48 KB of traffic per call; timed through the C ABI with pre-marshalled arguments"}, w
+
+
+def cpu_oracle_rate(w, cores, budget_s=2.5, max_elements=1 << 25):
+    """The float64 oracle, as it stands, on a bounded sample of workload `w` with `cores` threads."""
+    import numpy as np
+    from oracle import heinsen_oracle
+    heinsen_oracle.build()
+    t, keys = w.tensors, input_keys(w)
+    if w.rows == 1:
+        srows, sn = 1, min(w.n, max_elements if cores > 1 else max_elements // 4)
+    else:
+        limit = max_elements if cores > 1 else max_elements // 4
+        srows, sn = max(1, min(w.rows, limit // w.n)), w.n
+    sub = {k: np.ascontiguousarray(t[k][:srows, :sn] if t[k].ndim == 2 else t[k][:srows]) for k in keys}
+    threads = cores if srows > 1 else 1
+    passes, t0 = 0, time.perf_counter()
+    while True:
+        if w.kind == "linear":
+            heinsen_oracle.scan_linear(sub["a"], sub["b"], sub["x0"], nthreads=threads)
+        else:
+            heinsen_oracle.scan_log(sub["log_a"], sub["log_b"], sub["log_x0"], nthreads=threads)
+        passes += 1
+        dt = time.perf_counter() - t0
+        if dt > budget_s or passes >= 8:
+            break
+    return {"value": srows * sn * passes / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"{passes} passes over {srows} rows x n={sn} of the workload "
+                      f"({'whole batch' if srows * sn == w.rows * w.n else 'first rows / first elements'}), float64 sequential "
+                      f"loop" + (", OpenMP over rows" if threads > 1 else ", one core (the paper's sequential computation)")}
 
 
 # ---------------------------------------------------------------------------------------------- reference arm
@@ -130,7 +372,6 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    import numpy as np
     from oracle import heinsen_oracle
     from paper_2311_06281_b200 import workloads
 
@@ -159,12 +400,13 @@ def run_reference(args):
         step()
     dt = time.perf_counter() - t0
     value = rows * n * args.steps / dt
-    sample = f"{rows} rows x n={n} of {workload_name(cid, workloads.Workload(**{**full, 'tensors': {}}))} per step"
+    name = describe(cid, workloads.Workload(**{**full, "tensors": {}}))
+    sample = f"{rows} rows x n={n} of {name} per step"
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": workload_name(cid, workloads.Workload(**{**full, "tensors": {}})), "sample": sample},
+        "config": {"workload": name, "sample": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -173,12 +415,24 @@ def run_reference(args):
 
 
 # ---------------------------------------------------------------------------------------------- our arm
+def spawn_ranks(args):
+    """`--gpus N` without a torchrun environment: start the N ranks from here, the way the contract launches them."""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    raise SystemExit(subprocess.call(cmd))
+
+
 def run_ours(args):
     import numpy as np
     import torch
 
-    from paper_2311_06281_b200 import build_ext, heinsen_scan as hs, sharding, workloads
+    from paper_2311_06281_b200 import build_ext, heinsen_scan as hs, sharding
 
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        spawn_ranks(args)
     rank, world, local = sharding.init_from_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
@@ -186,40 +440,33 @@ def run_ours(args):
     dev = torch.device("cuda", local)
     build_ext.build()
     hs.lib()
+    peak, peak_source = measured_peak()
+    full = not args.only_headline
+    reduced = args.rows is not None or args.n is not None
 
+    # MUFU leg of the roofline: a register-only ex2/lg2 kernel, its rate per clock and SM at the clock sampled meanwhile
+    mufu_rate = None
+    if full:
+        hs.probe_mufu(1024)
+        sampler = ClockSampler(local, 0.002).start()
+        results, seconds = hs.probe_mufu(1 << 15)
+        pc = sampler.stop()
+        sms = torch.cuda.get_device_properties(dev).multi_processor_count
+        if pc["sm_mhz"]:
+            mufu_rate = {"results_per_clk_per_sm": results / seconds / (sms * pc["sm_mhz"] * 1e6), "sm_count": sms,
+                         "results_per_s": results / seconds, "probe_seconds": seconds, "probe_clocks": pc,
+                         "kernel": "heinsen_scan_probe_mufu: 8 independent ex2/lg2 chains per thread, 64 warps per SM"}
+
+    # ------------------------------------------------------------------ headline: EXACTLY K timed steps
     cid = args.workload
-    # weak scaling: every rank runs its own full batch, seeded by its rank
-    w = workloads.make(cid, rows=args.rows, n=args.n, seed=rank)
-    t = w.tensors
+    w = make_workload(cid, args.variant, rows=args.rows, n=args.n, seed=rank)  # weak scaling: every rank its own batch
     rows, n = w.rows, w.n
-    keys = ("a", "b", "x0") if w.kind == "linear" else ("log_a", "log_b", "log_x0")
-
-    def dev_tensor(arr):
-        x = torch.from_numpy(np.ascontiguousarray(arr))
-        if arr.dtype == np.uint16:
-            x = x.view(torch.bfloat16)
-        return x.to(dev)
-
-    # rotate independent buffer sets so that no step finds its inputs in L2 (each set alone exceeds L2)
-    nsets = 3
-    base = [dev_tensor(t[k]) for k in keys]
-    sets = [base] + [[x.clone() for x in base] for _ in range(nsets - 1)]
-    outs = [torch.empty((rows, n), dtype=base[0].dtype, device=dev) for _ in range(nsets)]
-    wss = [hs.new_workspace(rows, n, dev) for _ in range(nsets)]
-    call = hs.scan_linear if w.kind == "linear" else hs.scan_log
-
-    def step(i):
-        s = i % nsets
-        if w.kind == "linear":
-            hs.scan_linear(sets[s][0], sets[s][1], sets[s][2], x=outs[s], workspace=wss[s])
-        else:
-            hs.scan_log(sets[s][0], sets[s][1], sets[s][2], log_x=outs[s], workspace=wss[s])
-
+    dw = DeviceWorkload(w, dev, hs)
     for i in range(max(args.warmup, 3)):
-        step(i)
+        dw.step(i)
     torch.cuda.synchronize()
-    for ws in wss:
-        hs.check(ws)
+    dw.check()
+    kernel = "batched_scan_kernel" if hs.last_path() == hs.PATH_BATCHED else "lookback_scan_kernel"
 
     sampler = ClockSampler(local)
     launches0 = hs.launch_count()
@@ -229,7 +476,7 @@ def run_ours(args):
     sampler.start()
     start.record()
     for i in range(args.steps):
-        step(i)
+        dw.step(i)
     stop.record()
     sampler.sample()
     torch.cuda.synchronize()
@@ -238,28 +485,44 @@ def run_ours(args):
     ms_local = start.elapsed_time(stop)
     ms_total = sharding.max_over_ranks(ms_local, dev)
     launches = hs.launch_count() - launches0
-    for ws in wss:
-        hs.check(ws)
+    dw.check()
 
     elements = rows * n
     ms_per_step = ms_total / args.steps
     value = world * elements / (ms_per_step * 1e-3)
+    key = f"cfg{cid}" + (f"_{args.variant}" if args.variant else "")
+    traffic = None if reduced else ncu_traffic().get(key)
+    roofline = roofline_record(w, 1e3 * ms_local / args.steps, clocks, peak, peak_source, mufu_rate, kernel,
+                               traffic["bytes"] if traffic else None)
+    if traffic:
+        roofline["traffic_source"] = traffic.get("source")
+    alg_bytes = algorithmic_bytes(w)
 
-    # roofline of the (single) kernel of a step: algorithmic bytes per launch / mean launch duration
-    peak, peak_kind = measured_peak()
-    bpe = bytes_per_element(w)
-    alg_bytes = elements * bpe + rows * (4 if w.storage == "f32" else 2)
-    achieved = alg_bytes / (ms_local / args.steps * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": NCU_TRAFFIC_BYTES.get(cid) if args.rows is None and args.n is None else None, "peak_source": f"{peak_kind} (MEASURED_PEAKS.json hbm_gbs)"
-                if peak_kind == "measured" else "fallback (no MEASURED_PEAKS.json)",
-                "algorithmic_bytes_per_launch": alg_bytes, "bytes_per_element": bpe,
-                "kernel": "batched_scan_kernel" if hs.last_path() == hs.PATH_BATCHED else "lookback_scan_kernel",
-                "frac_of_nominal_8TBs": achieved / 8000.0}
+    # ------------------------------------------------------------------ per-configuration records (rank 0 of 1 only)
+    records = {}
+    cpu_1core = {}
+    if full and not args.no_workloads and world == 1 and not reduced:
+        # the headline workload again as repeated batches, then the other configurations
+        del dw
+        torch.cuda.empty_cache()
+        for c, variant in ((2, None), (4, None), (5, None), (3, None), (3, "linear"), (3, "bf16")):
+            rec, wl = measure_record(c, variant, dev, local, hs, args, peak, peak_source, mufu_rate, torch)
+            k = f"cfg{c}" + (f"_{variant}" if variant else "")
+            if not args.no_cpu_baseline and variant != "bf16":
+                rec["cpu_baseline_1core"] = cpu_oracle_rate(wl, 1, budget_s=1.5)
+            records[k] = rec
+            del wl
+        rec1, w1 = measure_small_call(dev, hs, torch)
+        if not args.no_cpu_baseline:
+            rec1["cpu_baseline_1core"] = cpu_oracle_rate(w1, 1, budget_s=0.5)
+        records["cfg1"] = rec1
+        dw = None
 
-    # end to end through the host-buffer entry point: pinned host buffers, H2D + kernel + D2H per step
+    # ------------------------------------------------------------------ end to end: pinned host buffers, H2D + kernel + D2H per step
     e2e = None
-    if not args.no_e2e:
+    if full and not args.no_e2e:
+        t = w.tensors
+        keys = input_keys(w)
         host_in = [torch.from_numpy(np.ascontiguousarray(t[k])) for k in keys]
         host_in = [(x.view(torch.bfloat16) if x.dtype == torch.uint16 else x).pin_memory() for x in host_in]
         host_out = torch.empty((rows, n), dtype=host_in[0].dtype).pin_memory()
@@ -284,42 +547,25 @@ def run_ours(args):
         del scratch
 
     cpu_baseline = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    cpu_baseline_1core = None
+    if full and rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import heinsen_oracle
         heinsen_oracle.build()
-        # bounded sample of the same workload: at most 2^25 elements per pass, repeated for a few seconds
-        if rows == 1:
-            srows, sn = 1, min(n, 1 << 25)
-        else:
-            srows, sn = max(1, min(rows, (1 << 25) // n)), n
-        sub = {k: (t[k][:srows, :sn] if t[k].ndim == 2 else t[k][:srows]) for k in keys}
-        sub = {k: np.ascontiguousarray(v) for k, v in sub.items()}
-        cores = heinsen_oracle.max_threads() if srows > 1 else 1
-        passes, t0 = 0, time.perf_counter()
-        while True:
-            if w.kind == "linear":
-                heinsen_oracle.scan_linear(sub["a"], sub["b"], sub["x0"], nthreads=cores)
-            else:
-                heinsen_oracle.scan_log(sub["log_a"], sub["log_b"], sub["log_x0"], nthreads=cores)
-            passes += 1
-            dt = time.perf_counter() - t0
-            if dt > 4.0 or passes >= 8:
-                break
-        cpu_baseline = {"value": srows * sn * passes / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-                        "sample": f"{passes} passes over {srows} rows x n={sn} of the bench workload "
-                                  f"({'whole batch' if srows * sn == elements else 'first rows'}), float64 sequential loop, "
-                                  f"OpenMP over rows"}
+        cpu_baseline = cpu_oracle_rate(w, heinsen_oracle.max_threads(), budget_s=4.0)
+        cpu_baseline_1core = cpu_oracle_rate(w, 1, budget_s=2.0)
 
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32", "data": "synthetic",
-            "config": {"workload": workload_name(cid, w) + ("" if args.rows is None and args.n is None else " [reduced size]"), "rows_per_gpu": rows, "n": n, "storage": w.storage,
+            "dtype": ARITHMETIC, "data": "synthetic",
+            "config": {"workload": describe(cid, w, args.variant) + (" [reduced size]" if reduced else ""), "rows_per_gpu": rows,
+                       "n": n, "storage": w.storage,
                        "entry_point": "heinsen_scan_linear" if w.kind == "linear" else "heinsen_scan_log",
-                       "l2": f"{nsets} rotating buffer sets of {alg_bytes / 1e6:.0f} MB each (every set exceeds the 126 MB L2)",
+                       "l2": f"3 rotating buffer sets of {alg_bytes / 1e6:.0f} MB each (every set exceeds the 126 MB L2)",
                        "parallelism": f"rows sharded, {world} rank(s), no data-path collective"},
             "clocks": clocks, "gpu_launches": launches, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu_baseline,
+            "cpu_baseline_1core": cpu_baseline_1core, "mufu_probe": mufu_rate, "workloads": records or None,
         }
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -383,7 +629,7 @@ def run_unfused(args):
     import torch
 
     from oracle import heinsen_oracle
-    from paper_2311_06281_b200 import workloads
+    from paper_2311_06281_b200 import unfused_eq7, workloads
 
     cid = args.workload
     w = workloads.make(cid, rows=args.rows, n=args.n)
@@ -393,20 +639,15 @@ def run_unfused(args):
     t = w.tensors
     la, lb, lx0 = (torch.from_numpy(t[k]).to(dev) for k in ("log_a", "log_b", "log_x0"))
 
-    def eq7():
-        a_star = torch.cumsum(la, dim=1)                                  # Eq. 2, first prefix sum
-        z = torch.cat([lx0[:, None], lb - a_star], dim=1)                 # cat(log x0, log b - a*)
-        return a_star + torch.logcumsumexp(z, dim=1)[:, 1:]               # a* + tail(LCSE(.))  (= log x; Eq. 3 adds exp)
-
     for _ in range(max(args.warmup, 3)):
-        out = eq7()
+        out = unfused_eq7.scan_log_unfused(la, lb, lx0)
     torch.cuda.synchronize()
     torch.cuda.reset_peak_memory_stats()
     base = torch.cuda.memory_allocated()
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     start.record()
     for _ in range(args.steps):
-        out = eq7()
+        out = unfused_eq7.scan_log_unfused(la, lb, lx0)
     stop.record()
     torch.cuda.synchronize()
     ms = start.elapsed_time(stop) / args.steps
@@ -417,12 +658,11 @@ def run_unfused(args):
     got = out[rows].double().cpu().numpy()
     astar = np.cumsum(t["log_a"][rows].astype(np.float64), axis=1)
     tol = 2e-6 * (1 + np.abs(astar) + np.abs(ref - astar)) + 1e-5
-    # minimum traffic of the un-fused recipe: cumsum r+w, subtract r+r+w, cat r+w, LCSE r+w, slice+add r+r+w (4-byte elements)
-    passes_bytes = (2 + 3 + 2 + 2 + 3) * 4
+    passes_bytes = unfused_eq7.MIN_BYTES_PER_ELEMENT
     print(json.dumps({
         "ablation": "unfused", "metric": METRIC, "value": elements / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms,
-        "steps": args.steps, "config": {"workload": workload_name(cid, w)},
-        "framework_kernels_per_step": 5, "min_bytes_per_element": passes_bytes,
+        "steps": args.steps, "config": {"workload": describe(cid, w)},
+        "framework_kernels_per_step": unfused_eq7.FRAMEWORK_KERNELS_PER_CALL, "min_bytes_per_element": passes_bytes,
         "achieved_GBs_at_min_bytes": elements * passes_bytes / (ms * 1e-3) / 1e9,
         "extra_device_memory_bytes": int(torch.cuda.max_memory_allocated() - base),
         "max_err_over_tolerance": float(np.max(np.abs(got - ref) / tol)),
@@ -474,7 +714,7 @@ def run_pairs(args):
     print(json.dumps({
         "ablation": "pairs", "metric": METRIC, "unit": UNIT, "value": result["pairs"]["value"],
         "ms_per_step": result["pairs"]["ms_per_step"], "steps": args.steps,
-        "config": {"workload": workload_name(cid, w)}, "pairs": result["pairs"], "log_space": result["log_space"],
+        "config": {"workload": describe(cid, w)}, "pairs": result["pairs"], "log_space": result["log_space"],
         "frac_of_measured_hbm": {k: v["algorithmic_GBs"] / peak for k, v in result.items()},
     }), flush=True)
 

@@ -26,9 +26,14 @@
  *     sign_x0: [rows].  The output has n entries per row, x_1..x_n; x_0 is not part
  *     of it (Eq. 7's tail()).
  *   - Device entry points take DEVICE pointers owned by the caller.  The library
- *     never allocates, frees or keeps device memory.  Work is enqueued on `stream`
- *     (a cudaStream_t passed as void*; NULL = legacy default stream) and the call
- *     returns without synchronising.
+ *     never allocates or frees device memory and keeps none of the caller's.  Two
+ *     things of its own live as long as the process: the fixed 1 MiB scratch array
+ *     of heinsen_scan_log_static / scan_linear / scan_log (part of the library
+ *     image on every GPU that loads it), and, per device, the two streams and three
+ *     events that the *_host entry points create at their first call; *_host calls
+ *     on one device run one at a time.  Work is enqueued on `stream` (a cudaStream_t
+ *     passed as void*; NULL = legacy default stream) and the device entry points
+ *     return without synchronising.
  *   - Pointers must be aligned to their element size.  When every base pointer is
  *     16-byte aligned and n * sizeof(element) is a multiple of 16 for every tensor,
  *     chunks move by TMA; otherwise a slower in-kernel path with plain loads is used
@@ -238,6 +243,25 @@ hs_status heinsen_scan_set_path(hs_path path);
  * -1 disables it.  Nothing faults or hangs: the kernel returns and the context stays usable.
  */
 hs_status heinsen_scan_debug_config(uint32_t lookback_spin_limit, int64_t mute_tile);
+/*
+ * Tuning knobs, for sweeps and for tests that force a variant; every knob has a measured default
+ * that is chosen per call.  `name` is one of "NO_TMA", "ROWS_PER_WARP", "WARPS", "STAGES",
+ * "ROW_TICKETS", "NO_FLAT", "NO_PDL" (row-batched kernel), "LB_STAGES", "LB_WARPS", "LB_GROUP",
+ * "LB_SLEEP_IDLE", "LB_SLEEP_READY", "LB_CTAS_PER_SM" (look-back kernel); value >= 0 sets the knob
+ * (clamped to its range), value < 0 returns it to its default.  The environment variables
+ * HEINSEN_SCAN_<name> give the initial values; they are read once per process, not per call.
+ * Unknown name: HS_ERR_INVALID_ARG.
+ */
+hs_status heinsen_scan_tune(const char* name, int value);
+/*
+ * Roofline probe (no passage of the paper: a measurement aid).  Runs a register-only kernel that does
+ * nothing but ex2.approx / lg2.approx (the two transcendentals of Eq. 7-8 as the kernels evaluate them)
+ * on every SM of the current device, on the legacy default stream, and returns after it has completed:
+ * `results` = transcendental results produced, `seconds` = device time between two events around the
+ * launch.  results / seconds / (SM count x SM clock) is the MUFU rate per clock and SM that bounds the
+ * transcendental leg of the roofline.  iterations <= 0 or a null pointer: HS_ERR_INVALID_ARG.
+ */
+hs_status heinsen_scan_probe_mufu(int iterations, double* results, double* seconds);
 /* Path taken by the most recent successful launch of this process (hs_path value), 0 if none. */
 int heinsen_scan_last_path(void);
 /* Number of kernels this library has launched in this process (memsets not counted). */

@@ -6,6 +6,7 @@
 #include <cuda_runtime.h>
 
 #include <atomic>
+#include <climits>
 #include <chrono>
 #include <cstdio>
 #include <cstdlib>
@@ -98,7 +99,7 @@ EncodeFn encode_fn() {
 // flat: the same memory as (element in 128-byte line, whole line of the row, row), box = box_rows consecutive
 // lines of one row; the hardware clips a box at the row's last whole line, the n % line elements after it
 // are not part of this view.
-bool make_tmap(CUtensorMap* tm, const void* ptr, hs_dtype dt, long long rows, long long n, int box_rows, bool flat) {
+bool encode_tmap(CUtensorMap* tm, const void* ptr, hs_dtype dt, long long rows, long long n, int box_rows, bool flat) {
     EncodeFn fn = encode_fn();
     if (!fn) return false;
     const int es = (dt == HS_F32) ? 4 : 2;
@@ -122,12 +123,78 @@ bool make_tmap(CUtensorMap* tm, const void* ptr, hs_dtype dt, long long rows, lo
     return r == CUDA_SUCCESS;
 }
 
+// Encoding a tensor map costs about a microsecond and a call needs three; a map depends only on the
+// arguments below (it holds an address and a geometry, no state), so the most recent ones are kept.
+struct TmapKey {
+    const void* ptr;
+    long long rows, n;
+    int dt, box_rows, flat, dev;
+    bool operator==(const TmapKey& o) const {
+        return ptr == o.ptr && rows == o.rows && n == o.n && dt == o.dt && box_rows == o.box_rows && flat == o.flat &&
+               dev == o.dev;
+    }
+};
+struct TmapSlot {
+    TmapKey key;
+    CUtensorMap map;
+    bool used = false;
+};
+constexpr int kTmapSlots = 24;
+std::mutex g_tmap_mu;
+TmapSlot g_tmap_cache[kTmapSlots];
+int g_tmap_next = 0;
+
+bool make_tmap(CUtensorMap* tm, const void* ptr, hs_dtype dt, long long rows, long long n, int box_rows, bool flat) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const TmapKey key{ptr, rows, n, (int)dt, box_rows, flat ? 1 : 0, dev};
+    {
+        std::lock_guard<std::mutex> lk(g_tmap_mu);
+        for (int i = 0; i < kTmapSlots; ++i)
+            if (g_tmap_cache[i].used && g_tmap_cache[i].key == key) {
+                *tm = g_tmap_cache[i].map;
+                return true;
+            }
+    }
+    if (!encode_tmap(tm, ptr, dt, rows, n, box_rows, flat)) return false;
+    std::lock_guard<std::mutex> lk(g_tmap_mu);
+    TmapSlot& slot = g_tmap_cache[g_tmap_next];
+    g_tmap_next = (g_tmap_next + 1) % kTmapSlots;
+    slot.key = key;
+    slot.map = *tm;
+    slot.used = true;
+    return true;
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-int env_int(const char* name, int dflt, int lo, int hi) {
-    const char* v = std::getenv(name);
-    if (!v || !*v) return dflt;
-    int x = std::atoi(v);
+// Tuning knobs.  Each has a measured default chosen per call; a knob overrides it when it is set.  The
+// environment (HEINSEN_SCAN_<NAME>) is read once, when the first knob is looked up; afterwards only
+// heinsen_scan_tune() changes a knob, so that a launch costs no getenv().
+enum Knob : int {
+    kKnobNoTma = 0, kKnobRowsPerWarp, kKnobWarps, kKnobRowTickets, kKnobNoFlat, kKnobNoPdl, kKnobLbStages,
+    kKnobLbWarps, kKnobLbGroup, kKnobLbSleepIdle, kKnobLbSleepReady, kKnobLbCtasPerSm, kKnobStages, kKnobCount
+};
+const char* const kKnobNames[kKnobCount] = {
+    "NO_TMA", "ROWS_PER_WARP", "WARPS", "ROW_TICKETS", "NO_FLAT", "NO_PDL", "LB_STAGES",
+    "LB_WARPS", "LB_GROUP", "LB_SLEEP_IDLE", "LB_SLEEP_READY", "LB_CTAS_PER_SM", "STAGES"};
+constexpr int kKnobUnset = INT_MIN;
+std::atomic<int> g_knobs[kKnobCount];
+std::once_flag g_knobs_once;
+
+void load_knobs_from_env() {
+    for (int k = 0; k < kKnobCount; ++k) {
+        char name[64];
+        snprintf(name, sizeof name, "HEINSEN_SCAN_%s", kKnobNames[k]);
+        const char* v = std::getenv(name);
+        g_knobs[k].store((v && *v) ? std::atoi(v) : kKnobUnset);
+    }
+}
+// value of a knob clamped to [lo, hi], or `dflt` when it is not set
+int knob(Knob k, int dflt, int lo, int hi) {
+    std::call_once(g_knobs_once, load_knobs_from_env);
+    const int x = g_knobs[k].load(std::memory_order_relaxed);
+    if (x == kKnobUnset) return dflt;
     return x < lo ? lo : (x > hi ? hi : x);
 }
 
@@ -301,7 +368,7 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
     const int es_in = pr.din == HS_F32 ? 4 : 2, es_out = pr.dout == HS_F32 ? 4 : 2;
     bool tma = aligned16(p.in_a) && aligned16(p.in_b) && aligned16(p.out) && (p.n * es_in) % 16 == 0 &&
                (p.n * es_out) % 16 == 0 && p.n <= kMaxTmaDim && encode_fn() != nullptr;
-    if (env_int("HEINSEN_SCAN_NO_TMA", 0, 0, 1)) tma = false;
+    if (knob(kKnobNoTma, 0, 0, 1)) tma = false;
     pr.tma = tma;
 
     KernelEntry ke;
@@ -342,7 +409,7 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
             // address the rows, sixteen coalesced steps along one row instead of two along each of eight)
             R = 1;
         }
-        R = env_int("HEINSEN_SCAN_ROWS_PER_WARP", R, 1, 16);
+        R = knob(kKnobRowsPerWarp, R, 1, 16);
         while (R & (R - 1)) R &= R - 1;  // power of two
         p.rows_per_warp = R;
         p.nchunks = (int)((p.n + (32 / R) * ke.K - 1) / ((32 / R) * ke.K));
@@ -350,31 +417,35 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         // loads run one chunk ahead of the arithmetic (the kernel keeps one row group ahead): TMA boxes, or
         // asynchronous 4-byte copies where TMA cannot address the rows; 2-byte elements are staged in step
         stages = (tma || es_in == 4) ? 2 : 1;
-        const int max_warps = 16;
+        if (tma) stages = knob(kKnobStages, stages, 2, kMaxStages);  // deeper TMA pipelines are a knob
+        int max_warps = 16;
+        while (max_warps > 1 && max_warps * (stages * ke.warp_smem_per_stage + ke.warp_smem_out) + max_warps * 8 * kMaxStages +
+                                        1024 > dev.max_smem_optin)
+            --max_warps;
         long long per_sm = (groups + dev.sm_count - 1) / dev.sm_count;
         warps = (int)(per_sm < 1 ? 1 : (per_sm > max_warps ? max_warps : per_sm));
-        warps = env_int("HEINSEN_SCAN_WARPS", warps, 1, 16);
+        warps = knob(kKnobWarps, warps, 1, 16);
         const long long ctas_needed = (groups + warps - 1) / warps;
         grid = (int)(ctas_needed < dev.sm_count ? ctas_needed : dev.sm_count);
         // tickets balance SMs of unequal speed when every warp slot sees several groups; with fewer, a
         // greedy hand-out of the last round loses more than it gains (cfg4, 1.7 groups per slot: 81 vs 74 us)
         // ... and only for rows of at least four chunks, where a ticket can be drawn early enough to arrive in time
         int tickets = (groups >= 4ll * grid * warps && p.nchunks >= 4) ? 1 : 0;
-        tickets = env_int("HEINSEN_SCAN_ROW_TICKETS", tickets, 0, 1);
+        tickets = knob(kKnobRowTickets, tickets, 0, 1);
         fn = tickets ? ke.batched_tk : ke.batched;
     } else {
         p.rows_per_warp = 1;
         // S input stages per compute warp (phase 2 of a tile runs S-2 iterations after its phase 1),
         // W compute warps (as many as shared memory allows, at most the default), NLB look-back warps
-        stages = env_int("HEINSEN_SCAN_LB_STAGES", 4, 3, kLbMaxStages);
-        const int nlb = env_int("HEINSEN_SCAN_LB_LOOKERS", 1, 1, 4);
-        int W = env_int("HEINSEN_SCAN_LB_WARPS", kLookbackWarps, kLookbackMinWarps, kLbMaxWarps);
+        stages = knob(kKnobLbStages, 4, 3, kLbMaxStages);
+        const int nlb = 1;  // look-back (poller) warps per CTA
+        int W = knob(kKnobLbWarps, kLookbackWarps, kLookbackMinWarps, kLbMaxWarps);
         if (stages > 5) stages = 5;
         while (W > kLookbackMinWarps && (ke.lb_smem(W, stages) + 1024 > dev.max_smem_optin || W + nlb + 1 > 16)) --W;
         lb_smem = ke.lb_smem(W, stages) + 1024;
         p.lb_warps = nlb;
-        p.lb_sleep_idle = (unsigned)env_int("HEINSEN_SCAN_LB_SLEEP_IDLE", 200, 0, 100000);
-        p.lb_sleep_ready = (unsigned)env_int("HEINSEN_SCAN_LB_SLEEP_READY", 0, 0, 100000);
+        p.lb_sleep_idle = (unsigned)knob(kKnobLbSleepIdle, 200, 0, 100000);
+        p.lb_sleep_ready = (unsigned)knob(kKnobLbSleepReady, 0, 0, 100000);
         warps = W + nlb + 1;  // + the publisher warp
         p.tiles_per_row = (int)lookback_tiles_per_row(p.n, chunk, W);
         p.num_tiles = p.rows * p.tiles_per_row;
@@ -386,7 +457,7 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         p.lb_group = dev.sm_count - dev.sm_count / 12;
         if (p.lb_group > kLbMaxGroup) p.lb_group = kLbMaxGroup;
         if (p.lb_group < 2) p.lb_group = 2;
-        p.lb_group = env_int("HEINSEN_SCAN_LB_GROUP", p.lb_group, 2, kLbMaxGroup);
+        p.lb_group = knob(kKnobLbGroup, p.lb_group, 2, kLbMaxGroup);
         p.groups_per_row = (p.tiles_per_row + p.lb_group - 1) / p.lb_group;
         const size_t need = sizeof(Header) + ((size_t)p.num_tiles + (size_t)p.rows * p.groups_per_row) * 16;
         if (workspace_bytes < need) return HS_ERR_WORKSPACE_TOO_SMALL;
@@ -403,7 +474,7 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
     if (tma) {
         // one row per warp, rows of at least one whole 128-byte line: move a chunk as a single box of lines
         const bool flat = p.rows_per_warp == 1 && p.n * es_in >= 128 && p.n * es_out >= 128 &&
-                          !env_int("HEINSEN_SCAN_NO_FLAT", 0, 0, 1);
+                          !knob(kKnobNoFlat, 0, 0, 1);
         p.flat_boxes = flat ? 1 : 0;
         const int br_in = flat ? chunk * es_in / 128 : p.rows_per_warp;
         const int br_out = flat ? chunk * es_out / 128 : p.rows_per_warp;
@@ -430,7 +501,7 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         e = cached_occupancy(&per_sm, fn, warps * 32, smem);
         if (e != cudaSuccess) return cuda_fail("cudaOccupancyMaxActiveBlocksPerMultiprocessor", e);
         if (per_sm < 1) return HS_ERR_INVALID_ARG;
-        per_sm = env_int("HEINSEN_SCAN_LB_CTAS_PER_SM", per_sm, 1, per_sm);
+        per_sm = knob(kKnobLbCtasPerSm, per_sm, 1, per_sm);
         long long g = (long long)per_sm * dev.sm_count;
         if (g > p.num_tiles) g = p.num_tiles;
         grid = (int)g;
@@ -455,7 +526,7 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         cfg.stream = stream;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = env_int("HEINSEN_SCAN_NO_PDL", 0, 0, 1) ? 0 : 1;
+        attr[0].val.programmaticStreamSerializationAllowed = knob(kKnobNoPdl, 0, 0, 1) ? 0 : 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         e = cudaLaunchKernelExC(&cfg, fn, args);
@@ -535,10 +606,63 @@ hs_status static_scratch_address(void** out) {
     return HS_OK;
 }
 
+// Roofline probe: nothing but MUFU work.  Every thread advances kProbeChains independent chains
+// x <- ex2(x), x <- lg2(x) held in registers; the values stay in (0, 1] x [-1, 0] and never leave the SM
+// (one store per thread at the very end keeps the chains alive).
+constexpr int kProbeChains = 8;
+__global__ void __launch_bounds__(256) mufu_probe_kernel(int iterations, float seed, float* sink) {
+    float x[kProbeChains];
+#pragma unroll
+    for (int c = 0; c < kProbeChains; ++c) x[c] = seed + 0.01f * (float)c + 1e-6f * (float)threadIdx.x;
+#pragma unroll 1
+    for (int i = 0; i < iterations; ++i) {
+#pragma unroll
+        for (int c = 0; c < kProbeChains; ++c) x[c] = hs::ex2(-x[c]);  // (0, 1]
+#pragma unroll
+        for (int c = 0; c < kProbeChains; ++c) x[c] = -hs::lg2(x[c]);  // back to >= 0
+    }
+    float acc = 0.0f;
+#pragma unroll
+    for (int c = 0; c < kProbeChains; ++c) acc += x[c];
+    if (acc == 123456.0f) sink[threadIdx.x] = acc;  // never true in practice
+}
+
 }  // namespace
 
 // =============================================================================================
 extern "C" {
+
+hs_status heinsen_scan_probe_mufu(int iterations, double* results, double* seconds) {
+    if (iterations <= 0 || !results || !seconds) return HS_ERR_INVALID_ARG;
+    DeviceInfo dev;
+    hs_status st = device_info(dev);
+    if (st != HS_OK) return st;
+    if (dev.cc_major != 10) return HS_ERR_UNSUPPORTED_DEVICE;
+    void* scratch = nullptr;
+    st = static_scratch_address(&scratch);
+    if (st != HS_OK) return st;
+    const int threads = 256, blocks = dev.sm_count * 8;  // 64 warps per SM: every MUFU unit has work queued
+    cudaEvent_t e0, e1;
+    cudaError_t e;
+    if ((e = cudaEventCreate(&e0)) != cudaSuccess) return cuda_fail("cudaEventCreate", e);
+    if ((e = cudaEventCreate(&e1)) != cudaSuccess) { cudaEventDestroy(e0); return cuda_fail("cudaEventCreate", e); }
+    // the sink is never written (see the kernel); the library's fixed array only gives it a valid address
+    float* sink = static_cast<float*>(scratch);
+    mufu_probe_kernel<<<blocks, threads>>>(16, 0.5f, sink);  // warm-up
+    cudaEventRecord(e0);
+    mufu_probe_kernel<<<blocks, threads>>>(iterations, 0.5f, sink);
+    cudaEventRecord(e1);
+    e = cudaEventSynchronize(e1);
+    float ms = 0.0f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (e != cudaSuccess) return cuda_fail("mufu probe", e);
+    g_launches.fetch_add(2);
+    *results = (double)blocks * threads * (double)iterations * kProbeChains * 2.0;
+    *seconds = (double)ms * 1e-3;
+    return HS_OK;
+}
 
 hs_status heinsen_scan_linear(const void* a, const void* b, const void* x0, void* x, int64_t rows, int64_t n,
                               hs_dtype dtype, void* workspace, size_t workspace_bytes, void* stream) {
@@ -717,6 +841,17 @@ hs_status heinsen_scan_debug_config(uint32_t lookback_spin_limit, int64_t mute_t
     g_mute_tile.store(mute_tile);
     return HS_OK;
 }
+hs_status heinsen_scan_tune(const char* name, int value) {
+    if (!name) return HS_ERR_INVALID_ARG;
+    std::call_once(g_knobs_once, load_knobs_from_env);
+    for (int k = 0; k < kKnobCount; ++k) {
+        if (std::strcmp(name, kKnobNames[k]) == 0) {
+            g_knobs[k].store(value < 0 ? kKnobUnset : value);
+            return HS_OK;
+        }
+    }
+    return HS_ERR_INVALID_ARG;
+}
 int heinsen_scan_last_path(void) { return g_last_path.load(); }
 int64_t heinsen_scan_launch_count(void) { return g_launches.load(); }
 
@@ -759,6 +894,7 @@ struct HostLanes {
     cudaStream_t side[2] = {nullptr, nullptr};
     cudaEvent_t start = nullptr, done[2] = {nullptr, nullptr};
     bool ok = false;
+    std::mutex busy;  // host-buffer calls on one device share the side streams and events: one at a time
 };
 hs_status host_lanes(HostLanes** out) {
     static std::mutex mu;
@@ -816,6 +952,7 @@ static hs_status host_run(int linear, const void* a, const void* b, const void* 
     HostLanes* hl = nullptr;
     st = host_lanes(&hl);
     if (st != HS_OK) return st;
+    std::lock_guard<std::mutex> one_at_a_time(hl->busy);
     cudaError_t e;
 #define HS_TRY(call)                                          \
     do {                                                      \
@@ -831,16 +968,31 @@ static hs_status host_run(int linear, const void* a, const void* b, const void* 
     HS_TRY(cudaStreamWaitEvent(hl->side[1], hl->start, 0));
     const uint8_t *ha = static_cast<const uint8_t*>(a), *hb = static_cast<const uint8_t*>(b);
     uint8_t* hx = static_cast<uint8_t*>(x);
+    // On an error return nothing may stay in flight to or from the caller's host buffers.
+    auto quiesce = [&]() {
+        cudaStreamSynchronize(hl->side[0]);
+        cudaStreamSynchronize(hl->side[1]);
+        cudaStreamSynchronize(stream);
+    };
+#define HS_TRY_Q(call)                                        \
+    do {                                                      \
+        e = (call);                                           \
+        if (e != cudaSuccess) {                               \
+            quiesce();                                        \
+            return cuda_fail(#call, e);                       \
+        }                                                     \
+    } while (0)
+    int launched = 0;  // row blocks actually launched (the last ones may be empty)
     for (int k = 0; k < nblk; ++k) {
         const int64_t r0 = (int64_t)k * rows_blk;
         const int64_t rb = rows - r0 < rows_blk ? rows - r0 : rows_blk;
         if (rb <= 0) break;
         cudaStream_t s = hl->side[k & 1];
         const size_t e0 = (size_t)r0 * (size_t)n, ec = (size_t)rb * (size_t)n;
-        HS_TRY(cudaMemcpyAsync(d_a + e0 * es_in, ha + e0 * es_in, ec * es_in, cudaMemcpyHostToDevice, s));
-        HS_TRY(cudaMemcpyAsync(d_b + e0 * es_in, hb + e0 * es_in, ec * es_in, cudaMemcpyHostToDevice, s));
-        if (sa) HS_TRY(cudaMemcpyAsync(d_sa + e0, sa + e0, ec, cudaMemcpyHostToDevice, s));
-        if (sb) HS_TRY(cudaMemcpyAsync(d_sb + e0, sb + e0, ec, cudaMemcpyHostToDevice, s));
+        HS_TRY_Q(cudaMemcpyAsync(d_a + e0 * es_in, ha + e0 * es_in, ec * es_in, cudaMemcpyHostToDevice, s));
+        HS_TRY_Q(cudaMemcpyAsync(d_b + e0 * es_in, hb + e0 * es_in, ec * es_in, cudaMemcpyHostToDevice, s));
+        if (sa) HS_TRY_Q(cudaMemcpyAsync(d_sa + e0, sa + e0, ec, cudaMemcpyHostToDevice, s));
+        if (sb) HS_TRY_Q(cudaMemcpyAsync(d_sb + e0, sb + e0, ec, cudaMemcpyHostToDevice, s));
         void* ws = ws0 + (size_t)k * up256(ws_bytes);
         if (linear)
             st = heinsen_scan_linear(d_a + e0 * es_in, d_b + e0 * es_in, d_x0 + (size_t)r0 * es_in, d_x + e0 * es_out, rb, n,
@@ -849,22 +1001,27 @@ static hs_status host_run(int linear, const void* a, const void* b, const void* 
             st = heinsen_scan_log(d_a + e0 * es_in, d_b + e0 * es_in, d_x0 + (size_t)r0 * es_in, d_x + e0 * es_out,
                                   sa ? d_sa + e0 : nullptr, sb ? d_sb + e0 : nullptr, sx0 ? d_sx0 + r0 : nullptr,
                                   with_signs ? d_sx + e0 : nullptr, rb, n, din, dout, ws, ws_bytes, s);
-        if (st != HS_OK) return st;
-        HS_TRY(cudaMemcpyAsync(hx + e0 * es_out, d_x + e0 * es_out, ec * es_out, cudaMemcpyDeviceToHost, s));
-        if (with_signs) HS_TRY(cudaMemcpyAsync(sx + e0, d_sx + e0, ec, cudaMemcpyDeviceToHost, s));
+        if (st != HS_OK) {
+            quiesce();
+            return st;
+        }
+        ++launched;
+        HS_TRY_Q(cudaMemcpyAsync(hx + e0 * es_out, d_x + e0 * es_out, ec * es_out, cudaMemcpyDeviceToHost, s));
+        if (with_signs) HS_TRY_Q(cudaMemcpyAsync(sx + e0, d_sx + e0, ec, cudaMemcpyDeviceToHost, s));
     }
     for (int i = 0; i < 2; ++i) {
-        HS_TRY(cudaEventRecord(hl->done[i], hl->side[i]));
-        HS_TRY(cudaStreamWaitEvent(stream, hl->done[i], 0));
+        HS_TRY_Q(cudaEventRecord(hl->done[i], hl->side[i]));
+        HS_TRY_Q(cudaStreamWaitEvent(stream, hl->done[i], 0));
     }
+#undef HS_TRY_Q
 #undef HS_TRY
-    // one synchronisation and one strided read-back of the row blocks' status words
+    // one synchronisation and one strided read-back of the status words of the row blocks that ran
     e = cudaStreamSynchronize(stream);
     if (e != cudaSuccess) return cuda_fail("cudaStreamSynchronize", e);
     Header heads[kHostBlocks];
-    e = cudaMemcpy2D(heads, sizeof(Header), ws0, up256(ws_bytes), sizeof(Header), (size_t)nblk, cudaMemcpyDeviceToHost);
+    e = cudaMemcpy2D(heads, sizeof(Header), ws0, up256(ws_bytes), sizeof(Header), (size_t)launched, cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return cuda_fail("cudaMemcpy2D", e);
-    for (int k = 0; k < nblk; ++k) {
+    for (int k = 0; k < launched; ++k) {
         const Header& h = heads[k];
         if (h.error_id == h.started_id && h.started_id != 0 &&
             (h.error_code == HS_ERR_LOOKBACK_TIMEOUT || h.error_code == HS_ERR_COPY_TIMEOUT))

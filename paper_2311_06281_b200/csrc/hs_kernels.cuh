@@ -14,6 +14,8 @@
 #pragma once
 #include <cuda.h>
 
+#include <cstddef>
+
 #include "hs_device.cuh"
 
 namespace hs {
@@ -32,9 +34,14 @@ struct Header {
     unsigned long long error_id;    // id of the call that recorded `error_code`
     int error_code;
     int error_where;                // tile or row index, for diagnosis
-    unsigned long long ticket;      // batched kernel: {call id (low 32 bits), next row group} of the running call
-    unsigned long long reserved[28];
+    unsigned long long pad;
+    // batched kernel, one 16-byte word handled with 128-bit accesses: the next row group to hand out and the
+    // id of the call it counts for
+    unsigned long long ticket_next;
+    unsigned long long ticket_call;
+    unsigned long long reserved[26];
 };
+static_assert(offsetof(Header, ticket_next) % 16 == 0, "the ticket word is accessed as 16 bytes");
 static_assert(sizeof(Header) == 256, "workspace header is 256 bytes");
 
 struct Params {
@@ -79,6 +86,33 @@ __device__ __forceinline__ void record_error(const Params& p, int code, long lon
         h->error_code = code;
         h->error_where = (int)where;
     }
+}
+
+// One 16-byte word of global memory, read / written / exchanged as a whole.
+struct Desc { unsigned long long lo, hi; };
+__device__ __forceinline__ Desc ld_desc(const void* p) {
+    Desc d;
+    asm volatile("{\n\t.reg .b128 q;\n\tld.relaxed.gpu.global.b128 q, [%2];\n\tmov.b128 {%0, %1}, q;\n\t}"
+                 : "=l"(d.lo), "=l"(d.hi) : "l"(p) : "memory");
+    return d;
+}
+__device__ __forceinline__ void st_desc(void* p, Desc d) {
+    asm volatile("{\n\t.reg .b128 q;\n\tmov.b128 q, {%1, %2};\n\tst.relaxed.gpu.global.b128 [%0], q;\n\t}"
+                 ::"l"(p), "l"(d.lo), "l"(d.hi) : "memory");
+}
+// Compare-and-swap of a whole 16-byte word; returns what was there.
+__device__ __forceinline__ Desc cas_desc(void* p, Desc expected, Desc desired) {
+    Desc old;
+    asm volatile(
+        "{\n\t.reg .b128 c, d, r;\n\t"
+        "mov.b128 c, {%3, %4};\n\t"
+        "mov.b128 d, {%5, %6};\n\t"
+        "atom.relaxed.gpu.global.cas.b128 r, [%2], c, d;\n\t"
+        "mov.b128 {%0, %1}, r;\n\t}"
+        : "=l"(old.lo), "=l"(old.hi)
+        : "l"(p), "l"(expected.lo), "l"(expected.hi), "l"(desired.lo), "l"(desired.hi)
+        : "memory");
+    return old;
 }
 
 // Neutral padding of a ragged row tail: a = 1 (log a = 0), b = 0 (log b = -inf).
@@ -530,19 +564,22 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
     // an SM that streams faster than another (their shares of the memory system differ by several
     // percent) simply takes more rows.  With few groups per slot greedy hand-out would pile the last
     // round on the SMs that are ahead, and the groups stay with their slots: slot, slot + GW, ...
-    // The counter word carries the low 32
-    // bits of the call id in its upper half: the first CTA to find another call's word there replaces it
-    // by {this call, first ticket = number of warp slots}; the workspace needs no initialisation and no
-    // host-side reset.
-    unsigned long long* const ticket_word = &p.ws->ticket;
-    const unsigned long long ticket_tag = (p.call_id & 0xffffffffull) << 32;
+    // The counter shares a 16-byte word with the id of the call it counts for: the first CTA to find another
+    // call's id there replaces the whole word by {first ticket = number of warp slots, this call} in one
+    // 128-bit compare-and-swap (a CTA that loses the race finds the word already right); the workspace needs
+    // no initialisation and no host-side reset.
+    unsigned long long* const ticket_word = &p.ws->ticket_next;
     const int GW = gridDim.x * nwarps;
     if (threadIdx.x == 0) {
         if (blockIdx.x == 0) p.ws->started_id = p.call_id;
         if (TICKETS) {
-            const unsigned long long seen = *(volatile unsigned long long*)ticket_word;
-            if ((seen & 0xffffffff00000000ull) != ticket_tag)
-                atomicCAS(ticket_word, seen, ticket_tag | (unsigned long long)GW);
+            const Desc seen = ld_desc(ticket_word);
+            if (seen.hi != p.call_id) {
+                Desc fresh;
+                fresh.lo = (unsigned long long)GW;
+                fresh.hi = p.call_id;
+                (void)cas_desc(ticket_word, seen, fresh);
+            }
         }
     }
     if (TICKETS) __syncthreads();  // from here on the word belongs to this call
@@ -728,17 +765,6 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
 // state and payload always belong together:  {A, m, s, tag},  tag = state | parity << 2,
 // state 0 = nothing yet (the descriptor array is zeroed before every launch), 1 = the tile's
 // aggregate, 2 = the value of x after the tile (A = -inf).
-struct Desc { unsigned long long lo, hi; };
-__device__ __forceinline__ Desc ld_desc(const void* p) {
-    Desc d;
-    asm volatile("{\n\t.reg .b128 q;\n\tld.relaxed.gpu.global.b128 q, [%2];\n\tmov.b128 {%0, %1}, q;\n\t}"
-                 : "=l"(d.lo), "=l"(d.hi) : "l"(p) : "memory");
-    return d;
-}
-__device__ __forceinline__ void st_desc(void* p, Desc d) {
-    asm volatile("{\n\t.reg .b128 q;\n\tmov.b128 q, {%1, %2};\n\tst.relaxed.gpu.global.b128 [%0], q;\n\t}"
-                 ::"l"(p), "l"(d.lo), "l"(d.hi) : "memory");
-}
 __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {  // non-blocking
     uint32_t ok;
     asm volatile(
@@ -749,6 +775,16 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {  // n
         : "r"(bar), "r"(parity)
         : "memory");
     return ok != 0;
+}
+// Bounded wait that also gives up when `*abort` becomes non-zero: the flag is looked at between the polls,
+// each of which the hardware suspends for a bounded time of its own.
+__device__ __forceinline__ bool mbar_wait_abortable(uint32_t bar, uint32_t parity, uint32_t limit, const int* abort) {
+#pragma unroll 1
+    for (uint32_t i = 0; i < limit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*(const volatile int*)abort) return false;
+    }
+    return false;
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
@@ -1035,9 +1071,11 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
         const int g_rows_p = (int)G / tpr, g_rem_p = (int)G % tpr;
         for (long long i = 0; i < my_tiles; ++i, cur.advance((int)G, g_rows_p, g_rem_p, tpr)) {
             const int b = (int)(i % kLbRing);
-            if (!mbar_wait_bounded(agg_bar + 8 * b, (uint32_t)((i / kLbRing) & 1), kCopySpinLimit) ||
-                *(volatile int*)&xc->abort) {
-                if (lane == 0) { record_error(p, kErrCopyTimeout, cur.T); xc->abort = 1; }
+            // (the wait watches the CTA's abort flag: once the compute warps have given up, nobody arrives
+            // on this barrier any more, and the publisher must leave at once rather than poll to the limit)
+            const bool arrived = mbar_wait_abortable(agg_bar + 8 * b, (uint32_t)((i / kLbRing) & 1), kCopySpinLimit, &xc->abort);
+            if (!arrived || *(volatile int*)&xc->abort) {
+                if (lane == 0 && !*(volatile int*)&xc->abort) { record_error(p, kErrCopyTimeout, cur.T); xc->abort = 1; }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(total_bar + 8 * b);
                 break;

@@ -24,8 +24,8 @@ PATH_AUTO, PATH_BATCHED, PATH_LOOKBACK = 0, 1, 2
 EXPORTS = [
     "heinsen_scan_linear", "heinsen_scan_log", "heinsen_scan_workspace_bytes", "heinsen_scan_check",
     "heinsen_scan_linear_host", "heinsen_scan_log_host", "heinsen_scan_host_scratch_bytes",
-    "heinsen_scan_set_path", "heinsen_scan_debug_config", "heinsen_scan_last_path",
-    "heinsen_scan_launch_count", "heinsen_scan_strerror",
+    "heinsen_scan_set_path", "heinsen_scan_tune", "heinsen_scan_debug_config", "heinsen_scan_last_path",
+    "heinsen_scan_launch_count", "heinsen_scan_strerror", "heinsen_scan_probe_mufu",
     "heinsen_scan_log_static", "heinsen_scan_check_static", "heinsen_scan_static_max_elements",
     "heinsen_scan_log_complex", "heinsen_scan_complex_workspace_bytes",
     "heinsen_scan_linear_pairs",
@@ -70,6 +70,10 @@ def lib() -> ctypes.CDLL:
         L.heinsen_scan_host_scratch_bytes.restype = sz
         L.heinsen_scan_set_path.argtypes = [ci]
         L.heinsen_scan_set_path.restype = ci
+        L.heinsen_scan_tune.argtypes = [ctypes.c_char_p, ci]
+        L.heinsen_scan_tune.restype = ci
+        L.heinsen_scan_probe_mufu.argtypes = [ci, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
+        L.heinsen_scan_probe_mufu.restype = ci
         L.heinsen_scan_debug_config.argtypes = [ctypes.c_uint32, i64]
         L.heinsen_scan_debug_config.restype = ci
         L.heinsen_scan_last_path.restype = ci
@@ -159,6 +163,18 @@ def new_workspace(rows: int, n: int, device) -> torch.Tensor:
 
 def set_path(path: int):
     _check(lib().heinsen_scan_set_path(int(path)))
+
+
+def tune(name: str, value: int = -1):
+    """Set a tuning knob (see heinsen_scan_tune in the header); value < 0 restores its default."""
+    _check(lib().heinsen_scan_tune(name.encode(), int(value)))
+
+
+def probe_mufu(iterations: int = 4096):
+    """(results, seconds) of the register-only ex2/lg2 probe kernel on the current device; synchronous."""
+    results, seconds = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    _check(lib().heinsen_scan_probe_mufu(int(iterations), ctypes.byref(results), ctypes.byref(seconds)))
+    return results.value, seconds.value
 
 
 def debug_config(lookback_spin_limit: int = 0, mute_tile: int = -1):

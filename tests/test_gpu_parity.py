@@ -173,11 +173,14 @@ def test_rows_of_whole_lines_plus_a_remainder(hs, oracle, rows, n, cid):
             run_log(hs, oracle, w.tensors, path=path, what=f"lines+rest {rows}x{n}/{path}")
 
 
-def test_tickets_forced_on_few_rows(hs, oracle, monkeypatch):
-    monkeypatch.setenv("HEINSEN_SCAN_ROW_TICKETS", "1")
-    for rows, n in ((5, 4100), (300, 515), (2400, 2048)):
-        w = workloads.make(2, rows=rows, n=n, seed=rows)
-        run_log(hs, oracle, w.tensors, path=hs.PATH_BATCHED, what=f"forced tickets {rows}x{n}")
+def test_tickets_forced_on_few_rows(hs, oracle):
+    hs.tune("ROW_TICKETS", 1)
+    try:
+        for rows, n in ((5, 4100), (300, 515), (2400, 2048)):
+            w = workloads.make(2, rows=rows, n=n, seed=rows)
+            run_log(hs, oracle, w.tensors, path=hs.PATH_BATCHED, what=f"forced tickets {rows}x{n}")
+    finally:
+        hs.tune("ROW_TICKETS", -1)
 
 
 @pytest.mark.parametrize("n", [7, 520, 4099])
@@ -500,3 +503,56 @@ def test_repeatability(hs):
     for _ in range(5):
         again = hs.scan_log(la, lb, lx0)
         assert (again - first).abs().max().item() < 1e-5
+
+
+def test_lookback_abort_with_several_tiles_per_cta_returns_promptly(hs):
+    """The same muted tile on a row long enough that every CTA owns several tiles: once the compute warps of a
+    CTA have given up, its publisher warp must leave too instead of polling its barrier to the limit.  The call
+    has to come back within a fraction of a second and report the time-out."""
+    import time
+    n = 1 << 22                                     # 586 tiles on 148 CTAs: about four tiles per CTA
+    w = workloads.make(2, rows=1, n=n)
+    la, lb, lx0 = (to_dev(w.tensors[k]) for k in ("log_a", "log_b", "log_x0"))
+    hs.set_path(hs.PATH_LOOKBACK)
+    ws = hs.new_workspace(1, n, "cuda")
+    hs.debug_config(lookback_spin_limit=2000, mute_tile=3)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    hs.scan_log(la, lb, lx0, workspace=ws)
+    with pytest.raises(hs.HeinsenScanError) as ei:
+        hs.check(ws)
+    elapsed = time.perf_counter() - t0
+    assert ei.value.status == 5
+    assert elapsed < 2.0, f"aborting launch took {elapsed:.2f} s"
+    hs.debug_config(0, -1)
+    good = hs.scan_log(la, lb, lx0, workspace=ws)
+    hs.check(ws)
+    assert torch.isfinite(good).all()
+
+
+def test_lookback_protocol_stress_smallest_tiles(hs, oracle):
+    """Thousands of tiles of the smallest size (8 compute warps, groups of 2 tiles) exercise the descriptor
+    protocol a hundred times over; every repetition must match the oracle (every wait stays bounded)."""
+    n = (1 << 23) + 4096 + 12
+    w = workloads.make(3, rows=1, n=n)
+    t = w.tensors
+    la, lb, lx0 = (to_dev(t[k]) for k in ("log_a", "log_b", "log_x0"))
+    ref, _ = oracle.scan_log(t["log_a"], t["log_b"], t["log_x0"])
+    tol = tol_positive(t["log_a"].astype(np.float64), ref)
+    ref_dev = torch.from_numpy(ref).cuda()
+    tol_dev = torch.from_numpy(tol).cuda()
+    hs.set_path(hs.PATH_LOOKBACK)
+    hs.tune("LB_WARPS", 8)
+    hs.tune("LB_GROUP", 2)
+    try:
+        ws = hs.new_workspace(1, n, "cuda")
+        out = torch.empty_like(la)
+        for rep in range(100):
+            out.fill_(float("nan"))
+            hs.scan_log(la, lb, lx0, log_x=out, workspace=ws)
+            hs.check(ws)
+            worst = ((out.double() - ref_dev).abs() / tol_dev).max().item()
+            assert worst <= 1.0, f"repetition {rep}: {worst:.3g} of the tolerance"
+    finally:
+        hs.tune("LB_WARPS", -1)
+        hs.tune("LB_GROUP", -1)
