@@ -92,6 +92,31 @@ __device__ __forceinline__ float log_abs_fast(float v) {
     return (fabsf(f) < 0.125f) ? near_one : far;
 }
 
+// Packed fp32 pairs (sm_100's f32x2 arithmetic): one instruction, hence one issue slot, for two
+// elements.  The kernels are short of issue slots before they are short of anything else, so all
+// element-wise arithmetic of a lane's run is written on pairs of neighbouring elements.
+__device__ __forceinline__ float2 pk(float x, float y) { return make_float2(x, y); }
+__device__ __forceinline__ float2 pk(float x) { return make_float2(x, x); }
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) { return __ffma2_rn(a, b, c); }
+__device__ __forceinline__ float2 mul2(float2 a, float2 b) { return __fmul2_rn(a, b); }
+__device__ __forceinline__ float2 add2(float2 a, float2 b) { return __fadd2_rn(a, b); }
+
+// log_abs_fast on two values at once.
+__device__ __forceinline__ float2 log_abs_fast2(float2 v) {
+    const float2 av = pk(fabsf(v.x), fabsf(v.y));
+    const float2 f = add2(av, pk(-1.0f));
+    float2 p = fma2(f, pk(-1.0f / 8.0f), pk(1.0f / 7.0f));
+    p = fma2(p, f, pk(-1.0f / 6.0f));
+    p = fma2(p, f, pk(1.0f / 5.0f));
+    p = fma2(p, f, pk(-1.0f / 4.0f));
+    p = fma2(p, f, pk(1.0f / 3.0f));
+    p = fma2(p, f, pk(-0.5f));
+    p = fma2(p, f, pk(1.0f));
+    const float2 near_one = mul2(p, f);
+    const float2 far = mul2(pk(lg2(av.x), lg2(av.y)), pk(kLn2));
+    return pk((fabsf(f.x) < 0.125f) ? near_one.x : far.x, (fabsf(f.y) < 0.125f) ? near_one.y : far.y);
+}
+
 // ------------------------------------------------------------------------------------------
 // The associative element.
 template <bool SIGNED>
@@ -407,45 +432,72 @@ struct Run {
     // va, vb: the stored inputs (log a, log b for the log modes; a, b for kLinear).
     // sa, sb: per-element sign masks for kLogSigned (ignored otherwise).
     __device__ __forceinline__ E pass1(const float* va, const float* vb, const uint32_t* sa, const uint32_t* sb) {
+        static_assert(K % 2 == 0, "runs are processed in pairs of elements");
         float acc = 0.0f;
         uint32_t par = 0u;
         float rr = neg_inf();
+        if (MODE == kLinear) {
+            // The reference of the run is taken from the largest |b_t| and the smallest A_t: it bounds
+            // every u_t = log|b_t| - A_t from above, which is all a log-sum-exp reference has to do, and it
+            // costs one logarithm per run instead of one per element; b_t itself enters the sum linearly.
+            float bmax = 0.0f, amin = 0.0f;
 #pragma unroll
-        for (int t = 0; t < K; ++t) {
-            float la, lbr;
-            if (MODE == kLinear) {
-                la = log_abs_fast(va[t]);
+            for (int t = 0; t < K; t += 2) {
+                const float2 la = log_abs_fast2(pk(va[t], va[t + 1]));
                 par ^= __float_as_uint(va[t]) & kSignBit;
-                lbr = lg2(fabsf(vb[t])) * kLn2;  // rough: only seeds the reference
-            } else {
-                la = va[t];
-                lbr = vb[t];
-                if (MODE == kLogSigned) par ^= sa[t];
+                P[t] = par;
+                par ^= __float_as_uint(va[t + 1]) & kSignBit;
+                P[t + 1] = par;
+                acc += la.x;
+                A[t] = acc;
+                acc += la.y;
+                A[t + 1] = acc;
+                bmax = fmaxf(bmax, fmaxf(fabsf(vb[t]), fabsf(vb[t + 1])));
+                amin = fminf(amin, fminf(A[t], A[t + 1]));
             }
-            acc += la;
-            A[t] = acc;
-            if (SIGNED) P[t] = par;
-            const float u = lbr - acc;
-            s[t] = u;
-            rr = fmaxf(rr, u);
+            // (2^-126 <= bmax keeps the scale factor below 2^127; smaller b_t are zero to ex2/lg2.approx.ftz anyway)
+            rr = (bmax >= 1.17549435e-38f) ? fmaf(lg2(bmax), kLn2, -amin) : neg_inf();
+            bad = !(acc >= -1e30f) || !(bmax <= 3.0e38f) || !(amin >= -1e30f);
+        } else {
+#pragma unroll
+            for (int t = 0; t < K; t += 2) {
+                if (MODE == kLogSigned) {
+                    par ^= sa[t];
+                    P[t] = par;
+                    par ^= sa[t + 1];
+                    P[t + 1] = par;
+                }
+                acc += va[t];
+                A[t] = acc;
+                acc += va[t + 1];
+                A[t + 1] = acc;
+                const float2 u = fma2(pk(A[t], A[t + 1]), pk(-1.0f), pk(vb[t], vb[t + 1]));
+                s[t] = u.x;
+                s[t + 1] = u.y;
+                rr = fmaxf(rr, fmaxf(u.x, u.y));
+            }
+            bad = !(acc >= -1e30f) || !(rr <= 1e30f);
         }
         r = rr;
-        bad = !(acc >= -1e30f) || !(rr <= 1e30f);
         const float ref = (rr == neg_inf()) ? 0.0f : rr;
-        const float c = -ref * kLog2e;
+        const float2 c = pk(-ref * kLog2e);
         float sum = 0.0f;
 #pragma unroll
-        for (int t = 0; t < K; ++t) {
-            float e;
+        for (int t = 0; t < K; t += 2) {
+            float2 e;
             if (MODE == kLinear) {
-                e = vb[t] * ex2(fminf(fmaf(-A[t], kLog2e, c), 126.0f));
-                e = flip(e, P[t]);
+                const float2 arg = fma2(pk(A[t], A[t + 1]), pk(-kLog2e), c);  // <= 126: A_t >= amin, bmax >= 2^-126
+                e = mul2(pk(vb[t], vb[t + 1]), pk(ex2(arg.x), ex2(arg.y)));
+                e = pk(flip(e.x, P[t]), flip(e.y, P[t + 1]));
             } else {
-                e = ex2(fmaf(s[t], kLog2e, c));
-                if (MODE == kLogSigned) e = flip(e, sb[t] ^ P[t]);
+                const float2 arg = fma2(pk(s[t], s[t + 1]), pk(kLog2e), c);
+                e = pk(ex2(arg.x), ex2(arg.y));
+                if (MODE == kLogSigned) e = pk(flip(e.x, sb[t] ^ P[t]), flip(e.y, sb[t + 1] ^ P[t + 1]));
             }
-            sum += e;
+            sum += e.x;
             s[t] = sum;
+            sum += e.y;
+            s[t + 1] = sum;
         }
         E agg;
         agg.A = acc;
@@ -506,17 +558,26 @@ struct Run {
         const float w = (d >= 0.0f) ? ed : 1.0f;
         const float S1 = fmaf(s[0], w, C);
         const bool ok = (fabsf(S1) >= 8.67361738e-19f /* 2^-60 */) || (Sc == 0.0f && r == neg_inf());
+        const float2 w2 = pk(w), C2 = pk(C);
 #pragma unroll
-        for (int t = 0; t < K; ++t) {
-            const float S = fmaf(s[t], w, C);
+        for (int t = 0; t < K; t += 2) {
+            const float2 S = fma2(pk(s[t], s[t + 1]), w2, C2);
             if (MODE == kLinear) {
-                const float h = ex2((A[t] + M) * (0.5f * kLog2e));
-                out_mag[t] = flip((S * h) * h, P[t]);
+                // exp(A_t + M) as the square of exp((A_t + M) / 2): the exponent range of fp32 twice over
+                const float2 arg = fma2(pk(A[t], A[t + 1]), pk(0.5f * kLog2e), pk(M * (0.5f * kLog2e)));
+                const float2 h = pk(ex2(arg.x), ex2(arg.y));
+                const float2 x = mul2(mul2(S, h), h);
+                out_mag[t] = flip(x.x, P[t]);
+                out_mag[t + 1] = flip(x.y, P[t + 1]);
             } else {
-                out_mag[t] = fmaf(lg2(fabsf(S)), kLn2, A[t] + M);
+                const float2 o = fma2(pk(lg2(fabsf(S.x)), lg2(fabsf(S.y))), pk(kLn2), add2(pk(A[t], A[t + 1]), pk(M)));
+                out_mag[t] = o.x;
+                out_mag[t + 1] = o.y;
                 if (MODE == kLogSigned) {
-                    const uint32_t sg = (__float_as_uint(S) ^ P[t]) & kSignBit;
-                    out_sign[t] = (S == 0.0f) ? 0u : sg;
+                    const uint32_t sg0 = (__float_as_uint(S.x) ^ P[t]) & kSignBit;
+                    const uint32_t sg1 = (__float_as_uint(S.y) ^ P[t + 1]) & kSignBit;
+                    out_sign[t] = (S.x == 0.0f) ? 0u : sg0;
+                    out_sign[t + 1] = (S.y == 0.0f) ? 0u : sg1;
                 }
             }
         }
