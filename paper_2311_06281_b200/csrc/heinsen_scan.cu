@@ -227,9 +227,10 @@ KernelEntry entry() {
     e.lookback = reinterpret_cast<const void*>(&lookback_scan_kernel<MODE, TIn, TOut, LBK, TMA>);
     e.lb_K = LBK;
     e.K = K;
-    e.warp_smem_per_stage = 2 * 32 * K * (int)sizeof(TIn);
-    e.warp_smem_out = 2 * 32 * K * (int)sizeof(TOut);
-    e.lb_smem = [](int W, int S) { return lb_total_smem_bytes<TIn, LBK>(W, S); };
+    constexpr int PAD = TMA ? 0 : ChunkEngine<MODE, TIn, TOut, K>::WIDE_PAD;  // chunk buffers without TMA are one line longer
+    e.warp_smem_per_stage = 2 * (32 * K * (int)sizeof(TIn) + PAD);
+    e.warp_smem_out = 2 * (32 * K * (int)sizeof(TOut) + PAD);
+    e.lb_smem = [](int W, int S) { return lb_total_smem_bytes<TIn, LBK, PAD>(W, S); };
     return e;
 }
 
@@ -242,8 +243,9 @@ KernelEntry entry_batched_only() {
     e.lookback = nullptr;
     e.lb_K = K;
     e.K = K;
-    e.warp_smem_per_stage = 2 * 32 * K * (int)sizeof(TIn);
-    e.warp_smem_out = 2 * 32 * K * (int)sizeof(TOut);
+    constexpr int PAD = TMA ? 0 : ChunkEngine<MODE, TIn, TOut, K>::WIDE_PAD;
+    e.warp_smem_per_stage = 2 * (32 * K * (int)sizeof(TIn) + PAD);
+    e.warp_smem_out = 2 * (32 * K * (int)sizeof(TOut) + PAD);
     e.lb_smem = nullptr;
     return e;
 }
@@ -416,7 +418,7 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         const long long groups = (p.rows + R - 1) / R;
         // loads run one chunk ahead of the arithmetic (the kernel keeps one row group ahead): TMA boxes, or
         // asynchronous 4-byte copies where TMA cannot address the rows; 2-byte elements are staged in step
-        stages = (tma || es_in == 4) ? 2 : 1;
+        stages = (tma || es_in == 4 || R == 1) ? 2 : 1;  // (one row per warp: asynchronous 16-byte copies whatever the type)
         if (tma) stages = knob(kKnobStages, stages, 2, kMaxStages);  // deeper TMA pipelines are a knob
         int max_warps = 16;
         while (max_warps > 1 && max_warps * (stages * ke.warp_smem_per_stage + ke.warp_smem_out) + max_warps * 8 * kMaxStages +

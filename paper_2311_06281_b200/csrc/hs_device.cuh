@@ -317,6 +317,110 @@ struct Storage<__nv_bfloat16> {
 };
 
 // ------------------------------------------------------------------------------------------
+// A lane's K elements when the chunk sits `phi` bytes into its buffer (rows whose chunks do not start on a
+// 16-byte boundary of global memory are staged unit for unit, so the misalignment travels with them).
+// `off` holds the shared-memory offsets of the lane's K / kPerUnit units and of the one after them; which
+// words of those units are the lane's depends on phi only, so every shift is a statically indexed variant.
+__device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) {
+    asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ void sts16(uint32_t addr, uint32_t v) {
+    asm volatile("st.shared.b16 [%0], %1;" ::"r"(addr), "h"((unsigned short)v) : "memory");
+}
+template <typename T, int K>
+struct Shifted;
+template <int K>
+struct Shifted<float, K> {
+    static constexpr int UNITS = K / 4;
+    template <int SH>
+    __device__ static __forceinline__ void pick(const float* w, float* v) {
+#pragma unroll
+        for (int t = 0; t < K; ++t) v[t] = w[t + SH];
+    }
+    __device__ static __forceinline__ void read(uint32_t sm, const uint32_t* off, uint32_t phi, float* v) {
+        float w[K + 4];
+#pragma unroll
+        for (int j = 0; j <= UNITS; ++j) Storage<float>::unpack(lds128(sm + off[j]), w + 4 * j);
+        switch (phi >> 2) {
+            case 0: pick<0>(w, v); break;
+            case 1: pick<1>(w, v); break;
+            case 2: pick<2>(w, v); break;
+            default: pick<3>(w, v); break;
+        }
+    }
+    template <int SH>
+    __device__ static __forceinline__ void put(uint32_t sm, const uint32_t* off, const float* v) {
+#pragma unroll
+        for (int t = 0; t < K; ++t) sts32(sm + off[(t + SH) >> 2] + (uint32_t)(((t + SH) & 3) * 4), __float_as_uint(v[t]));
+    }
+    __device__ static __forceinline__ void write(uint32_t sm, const uint32_t* off, uint32_t phi, const float* v) {
+        switch (phi >> 2) {
+            case 0: put<0>(sm, off, v); break;
+            case 1: put<1>(sm, off, v); break;
+            case 2: put<2>(sm, off, v); break;
+            default: put<3>(sm, off, v); break;
+        }
+    }
+};
+template <int K>
+struct Shifted<__nv_bfloat16, K> {
+    static constexpr int UNITS = K / 8;
+    template <int SH>
+    __device__ static __forceinline__ void pick(const uint32_t* w, float* v) {
+#pragma unroll
+        for (int t = 0; t < K; ++t) {
+            const uint32_t word = w[(t + SH) >> 1];
+            v[t] = __uint_as_float(((t + SH) & 1) ? (word & 0xffff0000u) : (word << 16));
+        }
+    }
+    __device__ static __forceinline__ void read(uint32_t sm, const uint32_t* off, uint32_t phi, float* v) {
+        uint32_t w[K / 2 + 4];
+#pragma unroll
+        for (int j = 0; j <= UNITS; ++j) {
+            const uint4 q = lds128(sm + off[j]);
+            w[4 * j] = q.x; w[4 * j + 1] = q.y; w[4 * j + 2] = q.z; w[4 * j + 3] = q.w;
+        }
+        switch (phi >> 1) {
+            case 0: pick<0>(w, v); break;
+            case 1: pick<1>(w, v); break;
+            case 2: pick<2>(w, v); break;
+            case 3: pick<3>(w, v); break;
+            case 4: pick<4>(w, v); break;
+            case 5: pick<5>(w, v); break;
+            case 6: pick<6>(w, v); break;
+            default: pick<7>(w, v); break;
+        }
+    }
+    // element t goes to halfword t + SH of the lane's units
+    template <int SH>
+    __device__ static __forceinline__ void put(uint32_t sm, const uint32_t* off, const float* v) {
+        auto addr = [&](int h) { return sm + off[h >> 3] + (uint32_t)((h & 7) * 2); };
+        if (SH & 1) {
+            // the first and the last element share their words with the neighbouring lanes
+            sts16(addr(SH), Storage<__nv_bfloat16>::pack2(v[0], 0.0f));
+#pragma unroll
+            for (int t = 1; t + 1 < K; t += 2) sts32(addr(t + SH), Storage<__nv_bfloat16>::pack2(v[t], v[t + 1]));
+            sts16(addr(K - 1 + SH), Storage<__nv_bfloat16>::pack2(v[K - 1], 0.0f));
+        } else {
+#pragma unroll
+            for (int t = 0; t < K; t += 2) sts32(addr(t + SH), Storage<__nv_bfloat16>::pack2(v[t], v[t + 1]));
+        }
+    }
+    __device__ static __forceinline__ void write(uint32_t sm, const uint32_t* off, uint32_t phi, const float* v) {
+        switch (phi >> 1) {
+            case 0: put<0>(sm, off, v); break;
+            case 1: put<1>(sm, off, v); break;
+            case 2: put<2>(sm, off, v); break;
+            case 3: put<3>(sm, off, v); break;
+            case 4: put<4>(sm, off, v); break;
+            case 5: put<5>(sm, off, v); break;
+            case 6: put<6>(sm, off, v); break;
+            default: put<7>(sm, off, v); break;
+        }
+    }
+};
+
+// ------------------------------------------------------------------------------------------
 // mbarrier / TMA wrappers (raw PTX).
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
@@ -349,6 +453,10 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 // Asynchronous 4-byte copy global -> shared (for rows that TMA cannot address), with its group bookkeeping.
 __device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
+}
+// ... and 16-byte copy (both addresses 16-byte aligned), past L1.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
@@ -545,43 +653,62 @@ struct Run {
         bad = false;
     }
 
-    // Apply the value entering the run and produce the K outputs.
-    // out_mag: log|x_t| (log modes) or x_t (kLinear);  out_sign: sign masks (kLogSigned).
-    // Returns false when an early prefix is too small relative to the run's reference for the
-    // fast form to be trusted (the caller then redoes the chunk with the tracked form).
-    __device__ __forceinline__ bool apply(const E& entering, float* out_mag, uint32_t* out_sign) const {
+    // Apply the value entering the run and produce the outputs, in two steps so that a caller can store the
+    // outputs piece by piece instead of holding all K of them:
+    //   prepare() : the run's common factors, and whether the fast form can be trusted -- it cannot when an
+    //               early prefix is too small relative to the run's reference (the caller then redoes the chunk
+    //               with the tracked form);
+    //   outputs() : elements T0 .. T0+N-1.  out_mag: log|x_t| (log modes) or x_t (kLinear); out_sign: sign
+    //               masks (kLogSigned).
+    struct Applied {
+        float M, C, w;
+        bool ok;
+    };
+    __device__ __forceinline__ Applied prepare(const E& entering) const {
         const float Mc = entering.m, Sc = entering.s;  // Mc is finite (>= kEmpty); r may be -inf
-        const float M = fmaxf(Mc, r);
+        Applied a;
+        a.M = fmaxf(Mc, r);
         const float d = Mc - r;
         const float ed = ex2(-fabsf(d) * kLog2e);
-        const float C = (d >= 0.0f) ? Sc : Sc * ed;
-        const float w = (d >= 0.0f) ? ed : 1.0f;
-        const float S1 = fmaf(s[0], w, C);
-        const bool ok = (fabsf(S1) >= 8.67361738e-19f /* 2^-60 */) || (Sc == 0.0f && r == neg_inf());
-        const float2 w2 = pk(w), C2 = pk(C);
+        a.C = (d >= 0.0f) ? Sc : Sc * ed;
+        a.w = (d >= 0.0f) ? ed : 1.0f;
+        const float S1 = fmaf(s[0], a.w, a.C);
+        a.ok = (fabsf(S1) >= 8.67361738e-19f /* 2^-60 */) || (Sc == 0.0f && r == neg_inf());
+        return a;
+    }
+    template <int T0, int N>
+    __device__ __forceinline__ void outputs(const Applied& a, float* out_mag, uint32_t* out_sign) const {
+        static_assert(T0 % 2 == 0 && N % 2 == 0, "outputs are produced in pairs");
+        const float2 w2 = pk(a.w), C2 = pk(a.C);
 #pragma unroll
-        for (int t = 0; t < K; t += 2) {
+        for (int i = 0; i < N; i += 2) {
+            const int t = T0 + i;
             const float2 S = fma2(pk(s[t], s[t + 1]), w2, C2);
             if (MODE == kLinear) {
                 // exp(A_t + M) as the square of exp((A_t + M) / 2): the exponent range of fp32 twice over
-                const float2 arg = fma2(pk(A[t], A[t + 1]), pk(0.5f * kLog2e), pk(M * (0.5f * kLog2e)));
+                const float2 arg = fma2(pk(A[t], A[t + 1]), pk(0.5f * kLog2e), pk(a.M * (0.5f * kLog2e)));
                 const float2 h = pk(ex2(arg.x), ex2(arg.y));
                 const float2 x = mul2(mul2(S, h), h);
-                out_mag[t] = flip(x.x, P[t]);
-                out_mag[t + 1] = flip(x.y, P[t + 1]);
+                out_mag[i] = flip(x.x, P[t]);
+                out_mag[i + 1] = flip(x.y, P[t + 1]);
             } else {
-                const float2 o = fma2(pk(lg2(fabsf(S.x)), lg2(fabsf(S.y))), pk(kLn2), add2(pk(A[t], A[t + 1]), pk(M)));
-                out_mag[t] = o.x;
-                out_mag[t + 1] = o.y;
+                const float2 o = fma2(pk(lg2(fabsf(S.x)), lg2(fabsf(S.y))), pk(kLn2), add2(pk(A[t], A[t + 1]), pk(a.M)));
+                out_mag[i] = o.x;
+                out_mag[i + 1] = o.y;
                 if (MODE == kLogSigned) {
                     const uint32_t sg0 = (__float_as_uint(S.x) ^ P[t]) & kSignBit;
                     const uint32_t sg1 = (__float_as_uint(S.y) ^ P[t + 1]) & kSignBit;
-                    out_sign[t] = (S.x == 0.0f) ? 0u : sg0;
-                    out_sign[t + 1] = (S.y == 0.0f) ? 0u : sg1;
+                    out_sign[i] = (S.x == 0.0f) ? 0u : sg0;
+                    out_sign[i + 1] = (S.y == 0.0f) ? 0u : sg1;
                 }
             }
         }
-        return ok;
+    }
+    // all K at once
+    __device__ __forceinline__ bool apply(const E& entering, float* out_mag, uint32_t* out_sign) const {
+        const Applied a = prepare(entering);
+        outputs<0, K>(a, out_mag, out_sign);
+        return a.ok;
     }
 };
 

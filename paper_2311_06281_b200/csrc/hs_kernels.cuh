@@ -142,16 +142,135 @@ struct ChunkEngine {
     static constexpr int OUT_UNITS = R_::OUT_UNITS;
 
     struct Offsets {
-        uint32_t in[IN_UNITS];    // the lane's 16-byte input units inside a stage
-        uint32_t out[OUT_UNITS];  // the lane's 16-byte output units inside an output buffer
+        uint32_t in[IN_UNITS + 1];    // the lane's 16-byte input units inside a stage, and the unit after them
+        uint32_t out[OUT_UNITS + 1];  // the lane's 16-byte output units inside an output buffer, and the one after
     };
     __device__ static __forceinline__ Offsets offsets(const LaneMap& lm) {
         Offsets o;
 #pragma unroll
-        for (int j = 0; j < IN_UNITS; ++j) o.in[j] = chunk_off(lm.R, lm.g, (uint32_t)((lm.i * IN_UNITS + j) * 16));
+        for (int j = 0; j <= IN_UNITS; ++j) o.in[j] = chunk_off(lm.R, lm.g, (uint32_t)((lm.i * IN_UNITS + j) * 16));
 #pragma unroll
-        for (int j = 0; j < OUT_UNITS; ++j) o.out[j] = chunk_off(lm.R, lm.g, (uint32_t)((lm.i * OUT_UNITS + j) * 16));
+        for (int j = 0; j <= OUT_UNITS; ++j) o.out[j] = chunk_off(lm.R, lm.g, (uint32_t)((lm.i * OUT_UNITS + j) * 16));
         return o;
+    }
+
+    // Rows that TMA cannot address, one row per warp ("wide" staging): the 16-byte units of global memory that
+    // hold a chunk are copied as they are, so the chunk's first element sits phi bytes into its buffer, phi =
+    // address of the row's first element modulo 16 (the same for every chunk of the row: a chunk is a whole
+    // number of units wide).  Each tensor has its own phi.  Buffers of these kernels are one 128-byte line longer.
+    struct Wide {
+        bool on;
+        uint32_t phi_a, phi_b, phi_o;
+    };
+    __device__ static __forceinline__ Wide wide_of(const Params& p, long long row, bool on) {
+        Wide w;
+        w.on = on;
+        const size_t e0 = (size_t)row * (size_t)p.n;
+        w.phi_a = on ? (uint32_t)((reinterpret_cast<uintptr_t>(p.in_a) + e0 * sizeof(TIn)) & 15u) : 0u;
+        w.phi_b = on ? (uint32_t)((reinterpret_cast<uintptr_t>(p.in_b) + e0 * sizeof(TIn)) & 15u) : 0u;
+        w.phi_o = on ? (uint32_t)((reinterpret_cast<uintptr_t>(p.out) + e0 * sizeof(TOut)) & 15u) : 0u;
+        return w;
+    }
+    static constexpr int WIDE_PAD = 128;  // bytes added to every chunk buffer of the kernels without TMA
+    // Copy the units that hold columns [colbase, colbase + W) of the row, as far as the row goes (one group of
+    // asynchronous copies per call, committed by the caller).  The first and the last unit may reach a few bytes
+    // beyond the row: they are units that also hold bytes of the row, so they lie in mapped memory.
+    template <typename T>
+    __device__ static __forceinline__ void wide_copy_in(const void* tensor, uint32_t sm, int lane, long long elem0, long long left,
+                                                        int W) {
+        const uintptr_t g0 = reinterpret_cast<uintptr_t>(tensor) + (size_t)elem0 * sizeof(T);
+        const uint32_t phi = (uint32_t)(g0 & 15u);
+        const long long valid = left < W ? left : W;
+        const int nunits = valid > 0 ? (int)((phi + (uint32_t)valid * (uint32_t)sizeof(T) + 15u) >> 4) : 0;
+        const char* src = reinterpret_cast<const char*>(g0 - phi);
+        constexpr int ROUNDS = (32 * K * (int)sizeof(T) / 16 + 1 + 31) / 32;
+#pragma unroll
+        for (int q = 0; q < ROUNDS; ++q) {
+            const int u = q * 32 + lane;
+            if (u < nunits) cp_async16(sm + chunk_off(1, 0, (uint32_t)(u * 16)), src + 16 * u);
+        }
+    }
+    __device__ static __forceinline__ void wide_load_async(const Params& p, uint32_t sm_a, uint32_t sm_b, int lane, long long row,
+                                                           long long colbase, int W) {
+        const long long left = row < p.rows ? p.n - colbase : 0;
+        wide_copy_in<TIn>(p.in_a, sm_a, lane, row * p.n + colbase, left, W);
+        wide_copy_in<TIn>(p.in_b, sm_b, lane, row * p.n + colbase, left, W);
+        cp_async_commit();
+    }
+    // The chunk's outputs, written by the lanes phi_o bytes into the buffer, go out as whole 16-byte units
+    // where they fill one, element by element at the two ends.
+    __device__ static __forceinline__ void wide_store(const Params& p, uint32_t sm_out, int lane, long long row, long long colbase,
+                                                      int W) {
+        const long long left = row < p.rows ? p.n - colbase : 0;
+        const long long valid = left < W ? left : W;
+        if (valid <= 0) return;
+        const uintptr_t g0 = reinterpret_cast<uintptr_t>(p.out) + (size_t)(row * p.n + colbase) * sizeof(TOut);
+        const uint32_t phi = (uint32_t)(g0 & 15u);
+        const uint32_t nbytes = (uint32_t)valid * (uint32_t)sizeof(TOut);
+        const uint32_t head = phi ? ((16u - phi) < nbytes ? (16u - phi) : nbytes) : 0u;  // bytes of the first, partial unit
+        const uint32_t body = (nbytes - head) >> 4;                                     // whole units
+        const uint32_t tail = nbytes - head - (body << 4);                              // bytes of the last, partial unit
+        char* const dst = reinterpret_cast<char*>(g0 - phi);
+        const uint32_t u0 = phi ? 1u : 0u;
+        for (uint32_t u = (uint32_t)lane; u < body; u += 32u)
+            *reinterpret_cast<uint4*>(dst + 16u * (u0 + u)) = lds128(sm_out + chunk_off(1, 0, 16u * (u0 + u)));
+        const uint32_t head_n = head / (uint32_t)sizeof(TOut), tail_n = tail / (uint32_t)sizeof(TOut);
+        if ((uint32_t)lane < head_n) {
+            const uint32_t b = phi + (uint32_t)lane * (uint32_t)sizeof(TOut);
+            Storage<TOut>::store(dst + b, 0, Storage<TOut>::from_smem(sm_out + chunk_off(1, 0, b)));
+        }
+        if ((uint32_t)lane < tail_n) {
+            const uint32_t b = phi + nbytes - tail + (uint32_t)lane * (uint32_t)sizeof(TOut);
+            Storage<TOut>::store(dst + b, 0, Storage<TOut>::from_smem(sm_out + chunk_off(1, 0, b)));
+        }
+    }
+    // The lane's inputs from a stage, whichever way the chunk got there.
+    template <bool PLAIN>
+    __device__ static __forceinline__ void read_inputs(uint32_t sm_a, uint32_t sm_b, const Offsets& off, const Wide& wd,
+                                                       float* va, float* vb) {
+        if (PLAIN && wd.on) {
+            Shifted<TIn, K>::read(sm_a, off.in, wd.phi_a, va);
+            Shifted<TIn, K>::read(sm_b, off.in, wd.phi_b, vb);
+        } else {
+            R_::load(sm_a, sm_b, off.in, va, vb);
+        }
+    }
+    // The outputs of a run whose fast form holds, into the output buffer (and the signs to global memory): unit
+    // by unit, so that no more than one unit's worth of outputs is live at a time.
+    template <bool PLAIN, int J = 0>
+    __device__ static __forceinline__ void emit_units(const R_& run, const typename R_::Applied& ap, uint32_t sm_out,
+                                                      const Offsets& off) {
+        if constexpr (J < OUT_UNITS) {
+            constexpr int PER = Storage<TOut>::kPerUnit;
+            float o[PER];
+            uint32_t sg[1];
+            run.template outputs<J * PER, PER>(ap, o, sg);
+            sts128(sm_out + off.out[J], Storage<TOut>::pack(o));
+            emit_units<PLAIN, J + 1>(run, ap, sm_out, off);
+        }
+    }
+    template <bool PLAIN>
+    __device__ static __forceinline__ void emit_outputs(const Params& p, const R_& run, const typename R_::Applied& ap,
+                                                        uint32_t sm_out, const Offsets& off, const Wide& wd, long long idx0,
+                                                        long long left) {
+        if (MODE == kLogSigned || (PLAIN && wd.on)) {
+            float out_mag[K];
+            uint32_t out_sign[MODE == kLogSigned ? K : 1];
+            run.template outputs<0, K>(ap, out_mag, out_sign);
+            write_outputs<PLAIN>(sm_out, off, wd, out_mag);
+            if (MODE == kLogSigned) store_signs(p.sign_x, idx0, left, p.sign_vec_ok != 0, out_sign);
+        } else {
+            emit_units<PLAIN>(run, ap, sm_out, off);
+        }
+    }
+    template <bool PLAIN>
+    __device__ static __forceinline__ void write_outputs(uint32_t sm_out, const Offsets& off, const Wide& wd, const float* v) {
+        if (PLAIN && wd.on) {
+            Shifted<TOut, K>::write(sm_out, off.out, wd.phi_o, v);
+        } else {
+#pragma unroll
+            for (int j = 0; j < OUT_UNITS; ++j) sts128(sm_out + off.out[j], Storage<TOut>::pack(v + j * Storage<TOut>::kPerUnit));
+        }
     }
 
     // sign masks of the lane's K elements from a uint8 tensor (0/1 per element); idx0 = index of
@@ -195,16 +314,18 @@ struct ChunkEngine {
 
     // Tracked form, pass 1: the lane's run as one part, every step with its own reference.
     // idx0/left as above (`left` <= 0: the run lies wholly beyond the row).
+    // (phi_a, phi_b: where the chunks start in their buffers -- 0 unless staged wide)
     __device__ static __noinline__ E slow_pass1(uint32_t sm_a, uint32_t sm_b, LaneMap lm, const uint8_t* gsa,
-                                                const uint8_t* gsb, long long idx0, long long left) {
+                                                const uint8_t* gsb, long long idx0, long long left, uint32_t phi_a,
+                                                uint32_t phi_b) {
         E e = identity_elem<SIGNED>();
         for (int t = 0; t < K; ++t) {
             if (t < left) {
-                const uint32_t off = chunk_off(lm.R, lm.g, (uint32_t)((lm.i * K + t) * sizeof(TIn)));
+                const uint32_t byte = (uint32_t)((lm.i * K + t) * sizeof(TIn));
                 const uint32_t sa = gsa ? (((uint32_t)gsa[idx0 + t] & 1u) << 31) : 0u;
                 const uint32_t sb = gsb ? (((uint32_t)gsb[idx0 + t] & 1u) << 31) : 0u;
-                e = compose(e, Leaf<MODE, TIn>::get(Storage<TIn>::from_smem(sm_a + off), Storage<TIn>::from_smem(sm_b + off),
-                                                    sa, sb));
+                e = compose(e, Leaf<MODE, TIn>::get(Storage<TIn>::from_smem(sm_a + chunk_off(lm.R, lm.g, phi_a + byte)),
+                                                    Storage<TIn>::from_smem(sm_b + chunk_off(lm.R, lm.g, phi_b + byte)), sa, sb));
             }
         }
         return e;
@@ -216,17 +337,17 @@ struct ChunkEngine {
     // Tracked form, pass 2: step the value through the lane's run; returns outputs (and signs).
     __device__ static __noinline__ SlowOut slow_apply(E st, uint32_t sm_a, uint32_t sm_b, LaneMap lm,
                                                       const uint8_t* gsa, const uint8_t* gsb, long long idx0,
-                                                      long long left) {
+                                                      long long left, uint32_t phi_a, uint32_t phi_b) {
         SlowOut so;
         for (int t = 0; t < K; ++t) {
             float v = 0.0f;
             uint32_t sg = 0u;
             if (t < left) {
-                const uint32_t off = chunk_off(lm.R, lm.g, (uint32_t)((lm.i * K + t) * sizeof(TIn)));
+                const uint32_t byte = (uint32_t)((lm.i * K + t) * sizeof(TIn));
                 const uint32_t sa = gsa ? (((uint32_t)gsa[idx0 + t] & 1u) << 31) : 0u;
                 const uint32_t sb = gsb ? (((uint32_t)gsb[idx0 + t] & 1u) << 31) : 0u;
-                st = compose(st, Leaf<MODE, TIn>::get(Storage<TIn>::from_smem(sm_a + off), Storage<TIn>::from_smem(sm_b + off),
-                                                     sa, sb));
+                st = compose(st, Leaf<MODE, TIn>::get(Storage<TIn>::from_smem(sm_a + chunk_off(lm.R, lm.g, phi_a + byte)),
+                                                     Storage<TIn>::from_smem(sm_b + chunk_off(lm.R, lm.g, phi_b + byte)), sa, sb));
                 renormalise(st);
                 if (MODE == kLinear) {
                     const float h = ex2(st.m * (0.5f * kLog2e));
@@ -252,12 +373,13 @@ struct ChunkEngine {
     // `row` is the lane's row (may be >= rows for a padded group), col0 its first column.
     // `ragged` (warp-uniform): the chunk reaches beyond the row end or the warp's group beyond the
     // last row, so some lanes must pad their run with neutral elements.
+    template <bool PLAIN>
     __device__ static __forceinline__ void phase1(const Params& p, uint32_t sm_a, uint32_t sm_b,
                                                   const Offsets& off, const LaneMap& lm, int lane, long long row,
-                                                  long long col0, bool ragged, Pending& pd, E& total) {
+                                                  long long col0, bool ragged, const Wide& wd, Pending& pd, E& total) {
         float va[K], vb[K];
         uint32_t sa[MODE == kLogSigned ? K : 1], sb[MODE == kLogSigned ? K : 1];
-        R_::load(sm_a, sm_b, off.in, va, vb);
+        read_inputs<PLAIN>(sm_a, sm_b, off, wd, va, vb);
         const long long left = (row < p.rows) ? p.n - col0 : 0;
         if (ragged) {
 #pragma unroll
@@ -273,34 +395,29 @@ struct ChunkEngine {
         pd.slow = __any_sync(0xffffffffu, pd.run.bad);
         if (pd.slow) {
             agg = slow_pass1(sm_a, sm_b, lm, MODE == kLogSigned ? p.sign_a : nullptr,
-                             MODE == kLogSigned ? p.sign_b : nullptr, row * p.n + col0, left);
+                             MODE == kLogSigned ? p.sign_b : nullptr, row * p.n + col0, left, PLAIN ? wd.phi_a : 0u,
+                             PLAIN ? wd.phi_b : 0u);
         }
         row_scan(agg, lane, lm.R, pd.excl, total);
     }
 
     // Phase 2: `entering_row` is the value of x entering this row's piece of the chunk.
+    template <bool PLAIN>
     __device__ static __forceinline__ void phase2(const Params& p, uint32_t sm_a, uint32_t sm_b,
                                                   uint32_t sm_out, const Offsets& off, const LaneMap& lm, long long row,
-                                                  long long col0, const Pending& pd, const E& entering_row) {
+                                                  long long col0, const Wide& wd, const Pending& pd, const E& entering_row) {
         const E entering = compose(entering_row, pd.excl);
         const long long left = (row < p.rows) ? p.n - col0 : 0;
         const uint32_t ob = sm_out;
-        float out_mag[K];
-        uint32_t out_sign[MODE == kLogSigned ? K : 1];
-        bool ok = false;
-        if (!pd.slow) ok = pd.run.apply(entering, out_mag, out_sign);
-        ok = __all_sync(0xffffffffu, ok);
+        const typename R_::Applied ap = pd.run.prepare(entering);
+        const bool ok = __all_sync(0xffffffffu, !pd.slow && ap.ok);
         if (ok) {
-#pragma unroll
-            for (int j = 0; j < OUT_UNITS; ++j)
-                sts128(ob + off.out[j], Storage<TOut>::pack(out_mag + j * Storage<TOut>::kPerUnit));
-            if (MODE == kLogSigned) store_signs(p.sign_x, row * p.n + col0, left, p.sign_vec_ok != 0, out_sign);
+            emit_outputs<PLAIN>(p, pd.run, ap, ob, off, wd, row * p.n + col0, left);
         } else {
             const SlowOut so = slow_apply(entering, sm_a, sm_b, lm, MODE == kLogSigned ? p.sign_a : nullptr,
-                                          MODE == kLogSigned ? p.sign_b : nullptr, row * p.n + col0, left);
-#pragma unroll
-            for (int j = 0; j < OUT_UNITS; ++j)
-                sts128(ob + off.out[j], Storage<TOut>::pack(so.vals + j * Storage<TOut>::kPerUnit));
+                                          MODE == kLogSigned ? p.sign_b : nullptr, row * p.n + col0, left,
+                                          PLAIN ? wd.phi_a : 0u, PLAIN ? wd.phi_b : 0u);
+            write_outputs<PLAIN>(ob, off, wd, so.vals);
             if (MODE == kLogSigned) store_signs(p.sign_x, row * p.n + col0, left, p.sign_vec_ok != 0, so.sgn);
         }
     }
@@ -424,17 +541,20 @@ __device__ __forceinline__ uint8_t* align_1024(uint8_t* p) {
 }
 
 // Per-warp shared-memory footprint (bytes): `stages` input stages of two tensors + two output buffers.
+// (pad: bytes added to every chunk buffer -- 0 with TMA, one 128-byte line without, see ChunkEngine::Wide)
 template <int MODE, typename TIn, typename TOut, int K>
-__host__ __device__ constexpr int warp_smem_bytes(int stages) {
-    return stages * 2 * (32 * K * (int)sizeof(TIn)) + 2 * (32 * K * (int)sizeof(TOut));
+__host__ __device__ constexpr int warp_smem_bytes(int stages, int pad) {
+    return stages * 2 * (32 * K * (int)sizeof(TIn) + pad) + 2 * (32 * K * (int)sizeof(TOut) + pad);
 }
 
 // Per-warp asynchronous chunk pipeline: TMA loads into a ring of input stages, TMA stores from
 // two output buffers.  A chunk is moved as boxes of {128 bytes, R rows}; lane b moves box b.
-template <typename TIn, typename TOut, int K>
+template <typename TIn, typename TOut, int K, int PAD>
 struct WarpPipe {
     static constexpr int IN_BYTES = 32 * K * (int)sizeof(TIn);
     static constexpr int OUT_BYTES = 32 * K * (int)sizeof(TOut);
+    static constexpr int IN_BUF = IN_BYTES + PAD;    // one tensor's chunk buffer
+    static constexpr int OUT_BUF = OUT_BYTES + PAD;
     static constexpr int IN_PER_BOX = 128 / (int)sizeof(TIn);    // elements of a row in one box
     static constexpr int OUT_PER_BOX = 128 / (int)sizeof(TOut);
     uint32_t base;   // this warp's shared memory (32-bit shared address)
@@ -452,9 +572,9 @@ struct WarpPipe {
         in_boxes = flat ? 1 : IN_BYTES / (128 * R);
         out_boxes = flat ? 1 : OUT_BYTES / (128 * R);  // lanes that issue stores
     }
-    __device__ __forceinline__ uint32_t in_a(int s) const { return base + s * 2 * IN_BYTES; }
-    __device__ __forceinline__ uint32_t in_b(int s) const { return base + s * 2 * IN_BYTES + IN_BYTES; }
-    __device__ __forceinline__ uint32_t out(int o) const { return base + stages * 2 * IN_BYTES + o * OUT_BYTES; }
+    __device__ __forceinline__ uint32_t in_a(int s) const { return base + s * 2 * IN_BUF; }
+    __device__ __forceinline__ uint32_t in_b(int s) const { return base + s * 2 * IN_BUF + IN_BUF; }
+    __device__ __forceinline__ uint32_t out(int o) const { return base + stages * 2 * IN_BUF + o * OUT_BUF; }
 
     __device__ __forceinline__ void init() {
         if (lane == 0) {
@@ -533,10 +653,13 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
     uint8_t* smem = align_1024(smem_raw);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     // loads run ahead of the arithmetic: TMA boxes, or groups of asynchronous 4-byte copies
-    constexpr bool AHEAD = TMA || CE::ASYNC_PLAIN;
-    const int S = AHEAD ? p.stages : 1;
-    const int per_warp = warp_smem_bytes<MODE, TIn, TOut, K>(S);
     const int R = p.rows_per_warp;
+    constexpr bool PLAIN = !TMA;
+    constexpr int PAD = PLAIN ? CE::WIDE_PAD : 0;
+    const bool wide = PLAIN && R == 1;  // one row per warp that TMA cannot address: staged as whole 16-byte units
+    const bool AHEAD = TMA || CE::ASYNC_PLAIN || wide;
+    const int S = AHEAD ? p.stages : 1;
+    const int per_warp = warp_smem_bytes<MODE, TIn, TOut, K>(S, PAD);
 
     LaneMap lm;
     lm.R = R;
@@ -545,7 +668,7 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
     lm.W = (32 / R) * K;
     const typename CE::Offsets off = CE::offsets(lm);
 
-    using Pipe = WarpPipe<TIn, TOut, K>;
+    using Pipe = WarpPipe<TIn, TOut, K, PAD>;
     Pipe pipe;
     pipe.base = smem_u32(smem) + warp * per_warp;
     pipe.bars = smem_u32(smem + nwarps * per_warp) + warp * (8 * kMaxStages);
@@ -630,6 +753,7 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
     long long issued = 0, consumed = 0;
     auto issue_chunk = [&]() {
         if (TMA) pipe.issue(&tm_a, &tm_b, pgroup * R, pchunk * lm.W, pstage);
+        else if (wide) CE::wide_load_async(p, pipe.in_a(pstage), pipe.in_b(pstage), lane, pgroup, (long long)pchunk * lm.W, lm.W);
         else CE::generic_load_async(p, pipe.in_a(pstage), pipe.in_b(pstage), lm, lane, (long long)pgroup * R, pchunk * lm.W);
     };
     auto issue_next = [&]() {
@@ -666,6 +790,7 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
     long long row = (long long)group * R + lm.g;
     bool group_ragged = (group + 1) * (long long)R > p.rows;
     E state = CE::row_start(p, row);
+    typename CE::Wide wd = CE::wide_of(p, row, wide);
     int stage = 0;
     uint32_t parity = 0;
     while (TICKETS ? group < groups : consumed < items) {
@@ -698,9 +823,9 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
 
         typename CE::Pending pd;
         E total;
-        CE::phase1(p, sm_a, sm_b, off, lm, lane, row, col0, ragged, pd, total);
+        CE::template phase1<PLAIN>(p, sm_a, sm_b, off, lm, lane, row, col0, ragged, wd, pd, total);
         if (TMA) pipe.acquire_out();
-        CE::phase2(p, sm_a, sm_b, sm_out, off, lm, row, col0, pd, state);
+        CE::template phase2<PLAIN>(p, sm_a, sm_b, sm_out, off, lm, row, col0, wd, pd, state);
         state = compose(state, total);
         renormalise(state);
 
@@ -709,7 +834,8 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
             if (chunk == tail_chunk_out) CE::tail_store(p, sm_out, lane, row, colbase);
         } else {
             __syncwarp();
-            CE::generic_store(p, sm_out, lm, lane, (long long)group * R, colbase);
+            if (wide) CE::wide_store(p, sm_out, lane, row, colbase, lm.W);
+            else CE::generic_store(p, sm_out, lm, lane, (long long)group * R, colbase);
         }
         __syncwarp();  // every lane is done with this input stage
         ++consumed;
@@ -735,6 +861,7 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
             }
             row = (long long)group * R + lm.g;
             group_ragged = (group + 1) * (long long)R > p.rows;
+            wd = CE::wide_of(p, row, wide);
         }
         if (++stage == S) { stage = 0; parity ^= 1u; }
     }
@@ -986,18 +1113,21 @@ struct LanePark {
 // s_t (fp32) of phase 1 are parked over the b-tensor chunk when the input type is 4 bytes wide
 // (in place), else in a region of their own; the outputs of phase 2 are written over the parked
 // sums and stored from there.
-template <typename TIn, int K>
+// (PAD: bytes added to every chunk buffer -- 0 with TMA, one 128-byte line without, see ChunkEngine::Wide)
+template <typename TIn, int K, int PAD>
 struct LbStage {
     static constexpr int IN_BYTES = 32 * K * (int)sizeof(TIn);
+    static constexpr int IN_BUF = IN_BYTES + PAD;
     static constexpr bool IN_PLACE = sizeof(TIn) == 4;
-    static constexpr int PARK_OFF = IN_PLACE ? IN_BYTES : 2 * IN_BYTES;
-    static constexpr int BYTES = IN_PLACE ? 2 * IN_BYTES : 2 * IN_BYTES + 32 * K * 4;
-    static_assert(BYTES % 1024 == 0 && PARK_OFF % 1024 == 0, "swizzled buffers need 1024-byte alignment");
+    static constexpr int PARK_OFF = IN_PLACE ? IN_BUF : 2 * IN_BUF;
+    static constexpr int BYTES = IN_PLACE ? 2 * IN_BUF : 2 * IN_BUF + 32 * K * 4 + PAD;
+    static_assert(PAD != 0 || (BYTES % 1024 == 0 && PARK_OFF % 1024 == 0), "swizzled TMA buffers need 1024-byte alignment");
+    static_assert(BYTES % 128 == 0 && PARK_OFF % 128 == 0, "chunk buffers are made of 128-byte lines");
 };
 // total dynamic shared memory of the look-back kernel for W compute warps and S stages (without alignment slack)
-template <typename TIn, int K>
+template <typename TIn, int K, int PAD>
 __host__ __device__ constexpr int lb_total_smem_bytes(int W, int S) {
-    return W * S * LbStage<TIn, K>::BYTES + (int)sizeof(Exchange) + W * kLbMaxStages * 8;
+    return W * S * LbStage<TIn, K, PAD>::BYTES + (int)sizeof(Exchange) + W * kLbMaxStages * 8;
 }
 
 // Position of a CTA's tile sequence: tile T = tile j of row `row`; advances by a fixed stride
@@ -1025,7 +1155,8 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
     using CE = ChunkEngine<MODE, TIn, TOut, K>;
     using LB = Lookback<MODE, TIn, TOut, K>;
     using R_ = Run<MODE, TIn, TOut, K>;
-    using ST = LbStage<TIn, K>;
+    constexpr bool PLAIN = !TMA;
+    using ST = LbStage<TIn, K, PLAIN ? CE::WIDE_PAD : 0>;
     using E = typename CE::E;
     constexpr bool SIGNED = CE::SIGNED;
     constexpr int CHUNK = 32 * K;
@@ -1132,7 +1263,7 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
 
     const uint32_t wb = smem_u32(smem) + (uint32_t)(warp * S * ST::BYTES);
     auto st_a = [&](int st) { return wb + st * ST::BYTES; };
-    auto st_b = [&](int st) { return wb + st * ST::BYTES + ST::IN_BYTES; };
+    auto st_b = [&](int st) { return wb + st * ST::BYTES + ST::IN_BUF; };
     auto st_park = [&](int st) { return wb + st * ST::BYTES + ST::PARK_OFF; };
     LanePark<SIGNED> lp[4];  // lp[d]: the tile that went through phase 1 d iterations ago
 #pragma unroll
@@ -1158,13 +1289,14 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
     long long issued = 0;
     int istage = 0;
     // loads run a tile ahead of phase 1: TMA boxes, or groups of asynchronous 4-byte copies
-    constexpr bool AHEAD = TMA || CE::ASYNC_PLAIN;
+    // (without TMA: the chunk's 16-byte units copied asynchronously as they are -- see ChunkEngine::Wide)
+    constexpr bool AHEAD = true;
     auto issue_next = [&]() {
         if (issued < my_tiles) {
             const int cb = colbase_of(ci);
             const uint32_t bar = bars + 8 * istage;
             if (!TMA) {
-                CE::generic_load_async(p, st_a(istage), st_b(istage), lm, lane, ci.row, cb);
+                CE::wide_load_async(p, st_a(istage), st_b(istage), lane, ci.row, cb, CHUNK);
             } else if (flat) {
                 if (lane == 0) mbar_expect_tx(bar, 2 * ST::IN_BYTES);
                 __syncwarp();
@@ -1225,17 +1357,17 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                 else cp_async_wait<0>();
                 __syncwarp();
                 ++consumed;
-            } else {
-                CE::generic_load(p, st_a(st), st_b(st), lm, lane, row, colbase);
-                __syncwarp();
             }
             if (!aborted) {
                 const long long col0 = colbase + lane * K;
                 typename CE::Pending pd;
                 E total;
-                CE::phase1(p, st_a(st), st_b(st), off, lm, lane, row, col0, colbase + CHUNK > p.n, pd, total);
+                const typename CE::Wide wd = CE::wide_of(p, row, PLAIN);
+                CE::template phase1<PLAIN>(p, st_a(st), st_b(st), off, lm, lane, row, col0, colbase + CHUNK > p.n, wd, pd, total);
                 if (!pd.slow) {  // park the partial sums (a slow chunk keeps its inputs instead)
                     const uint32_t pb = st_park(st);
+                    // (wide staging: a lane's inputs reach into the unit after its own, where its neighbour parks)
+                    if (PLAIN) __syncwarp();
 #pragma unroll
                     for (int jx = 0; jx < K / 4; ++jx) sts128(pb + park_off[jx], Storage<float>::pack(pd.run.s + 4 * jx));
                     if (MODE == kLinear) {
@@ -1273,6 +1405,7 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
             if (!aborted) {
                 const long long col0 = colbase + lane * K;
                 const long long left = p.n - col0;
+                const typename CE::Wide wd = CE::wide_of(p, row, PLAIN);
                 E carry;
                 carry.A = neg_inf(); carry.m = xc->carry[b].x; carry.s = xc->carry[b].y; carry.p = 0u;
                 const LanePark<SIGNED> mine = (D == 1) ? lp[1] : (D == 2) ? lp[2] : lp[3];
@@ -1281,22 +1414,21 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                 uint32_t sm_a = st_a(st);
                 uint32_t sm_b = st_b(st);
                 const uint32_t pb = st_park(st);
-                float out_mag[K];
-                uint32_t out_sign[MODE == kLogSigned ? K : 1];
                 bool ok = false;
-                const bool was_slow = mine.slow;
+                const bool was_slow = mine.slow;  // (warp-uniform)
                 if (!was_slow) {
+                    R_ run;
                     // rebuild A_t (and the parity of a) from the inputs -- kLinear: fetch the parked A_t --,
                     // fetch the parked s_t, apply
                     float va[K];
                     uint32_t sa[MODE == kLogSigned ? K : 1];
-                    R_ run;
                     if (MODE == kLinear) {
 #pragma unroll
                         for (int jx = 0; jx < K / 4; ++jx) Storage<float>::unpack(lds128(sm_a + park_off[jx]), va + 4 * jx);
                         run.adopt(va, mine.par);
                     } else {
-                        R_::load_a(sm_a, off.in, va);
+                        if (PLAIN) Shifted<TIn, K>::read(sm_a, off.in, wd.phi_a, va);
+                        else R_::load_a(sm_a, off.in, va);
                         if (colbase + CHUNK > p.n) {
 #pragma unroll
                             for (int t = 0; t < K; ++t)
@@ -1308,15 +1440,14 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                     run.r = mine.r;
 #pragma unroll
                     for (int jx = 0; jx < K / 4; ++jx) Storage<float>::unpack(lds128(pb + park_off[jx]), run.s + 4 * jx);
-                    ok = run.apply(entering, out_mag, out_sign);
+                    const typename R_::Applied ap = run.prepare(entering);
+                    ok = __all_sync(0xffffffffu, ap.ok);  // also: every lane has read its parked sums
+                    if (ok) CE::template emit_outputs<PLAIN>(p, run, ap, pb, off, wd, row * p.n + col0, left);
                 }
-                ok = __all_sync(0xffffffffu, ok);  // also: every lane has read its parked sums
-                if (ok) {
-#pragma unroll
-                    for (int jx = 0; jx < CE::OUT_UNITS; ++jx)
-                        sts128(pb + off.out[jx], Storage<TOut>::pack(out_mag + jx * Storage<TOut>::kPerUnit));
-                    if (MODE == kLogSigned) CE::store_signs(p.sign_x, row * p.n + col0, left, p.sign_vec_ok != 0, out_sign);
-                } else {
+                if (!ok) {
+                    // where the lane's inputs are now: as staged (shifted) when the chunk kept them, at the lane's
+                    // own units when they are fetched again below
+                    uint32_t phi_a = PLAIN ? wd.phi_a : 0u, phi_b = PLAIN ? wd.phi_b : 0u;
                     if (!was_slow && ST::IN_PLACE) {
                         // the parked sums replaced the b-tensor chunk: fetch the lane's b values again
 #pragma unroll
@@ -1328,15 +1459,15 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                                 Storage<TIn>::to_smem(sm_a + chunk_off(1, 0, (uint32_t)((lane * K + t) * sizeof(TIn))), u);
                             }
                         }
+                        phi_b = 0u;
+                        if (MODE == kLinear) phi_a = 0u;
                         __syncwarp();
                     }
                     const typename CE::SlowOut so =
                         CE::slow_apply(entering, sm_a, sm_b, lm, MODE == kLogSigned ? p.sign_a : nullptr,
-                                       MODE == kLogSigned ? p.sign_b : nullptr, row * p.n + col0, left);
+                                       MODE == kLogSigned ? p.sign_b : nullptr, row * p.n + col0, left, phi_a, phi_b);
                     __syncwarp();
-#pragma unroll
-                    for (int jx = 0; jx < CE::OUT_UNITS; ++jx)
-                        sts128(pb + off.out[jx], Storage<TOut>::pack(so.vals + jx * Storage<TOut>::kPerUnit));
+                    CE::template write_outputs<PLAIN>(pb, off, wd, so.vals);
                     if (MODE == kLogSigned) CE::store_signs(p.sign_x, row * p.n + col0, left, p.sign_vec_ok != 0, so.sgn);
                 }
                 if (TMA) {
@@ -1356,7 +1487,7 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                     }
                 } else {
                     __syncwarp();
-                    CE::generic_store(p, st_park(st), lm, lane, row, colbase);
+                    CE::wide_store(p, st_park(st), lane, row, colbase, CHUNK);
                 }
                 __syncwarp();  // every lane is done with this tile's stage
             }

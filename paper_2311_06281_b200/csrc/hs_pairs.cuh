@@ -64,11 +64,24 @@ struct ChunkEngine<kPairs, TIn, TOut, K> {
         E excl;
     };
 
+    using Wide = typename Base::Wide;
+    static constexpr int WIDE_PAD = Base::WIDE_PAD;
+    __device__ static __forceinline__ Wide wide_of(const Params& p, long long row, bool on) { return Base::wide_of(p, row, on); }
+    __device__ static __forceinline__ void wide_load_async(const Params& p, uint32_t sm_a, uint32_t sm_b, int lane, long long row,
+                                                           long long colbase, int W) {
+        Base::wide_load_async(p, sm_a, sm_b, lane, row, colbase, W);
+    }
+    __device__ static __forceinline__ void wide_store(const Params& p, uint32_t sm_out, int lane, long long row, long long colbase,
+                                                      int W) {
+        Base::wide_store(p, sm_out, lane, row, colbase, W);
+    }
+
+    template <bool PLAIN>
     __device__ static __forceinline__ void phase1(const Params& p, uint32_t sm_a, uint32_t sm_b, const Offsets& off,
                                                   const LaneMap&, int lane, long long row, long long col0, bool ragged,
-                                                  Pending& pd, E& total) {
+                                                  const Wide& wd, Pending& pd, E& total) {
         float va[K], vb[K];
-        Run<kLinear, TIn, TOut, K>::load(sm_a, sm_b, off.in, va, vb);
+        Base::template read_inputs<PLAIN>(sm_a, sm_b, off, wd, va, vb);
         if (ragged) {
             const long long left = (row < p.rows) ? p.n - col0 : 0;
 #pragma unroll
@@ -90,16 +103,15 @@ struct ChunkEngine<kPairs, TIn, TOut, K> {
         row_scan(agg, lane, p.rows_per_warp, pd.excl, total);
     }
 
+    template <bool PLAIN>
     __device__ static __forceinline__ void phase2(const Params&, uint32_t, uint32_t, uint32_t sm_out, const Offsets& off,
-                                                  const LaneMap&, long long, long long, const Pending& pd,
+                                                  const LaneMap&, long long, long long, const Wide& wd, const Pending& pd,
                                                   const E& entering_row) {
         const float x_in = fmaf(pd.excl.alpha, entering_row.beta, pd.excl.beta);
         float out[K];
 #pragma unroll
         for (int t = 0; t < K; ++t) out[t] = fmaf(pd.P[t], x_in, pd.B[t]);
-#pragma unroll
-        for (int j = 0; j < OUT_UNITS; ++j)
-            sts128(sm_out + off.out[j], Storage<TOut>::pack(out + j * Storage<TOut>::kPerUnit));
+        Base::template write_outputs<PLAIN>(sm_out, off, wd, out);
     }
 
     struct RawX0 { float v; };
