@@ -55,8 +55,9 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--rows", type=int, default=None, help="override the workload's rows (profiling of small cases)")
     ap.add_argument("--n", type=int, default=None, help="override the workload's n (profiling of small cases)")
-    ap.add_argument("--variant", default=None, choices=["linear", "bf16"],
-                    help="with --workload 3: time the linear entry point / bf16 storage on the same sequence")
+    ap.add_argument("--variant", default=None, choices=["linear", "bf16", "complex"],
+                    help="with --workload 3: time the linear entry point / bf16 storage on the same sequence; with "
+                         "--workload 4: the same signed values as complex logarithms (heinsen_scan_log_complex)")
     ap.add_argument("--only-headline", action="store_true",
                     help="skip the per-configuration records, the MUFU probe, the end-to-end leg and the CPU baselines "
                          "(profiling runs)")
@@ -164,6 +165,19 @@ def make_workload(cid, variant=None, rows=None, n=None, seed=0):
         for k in ("log_a", "log_b", "log_x0"):
             w.tensors[k] = workloads.to_bf16_bits(w.tensors[k].astype("float64")).reshape(w.tensors[k].shape)
         w.storage = "bf16"
+    elif variant == "complex":
+        # the signed workload as complex logarithms (log|v|, 0 or pi): the representation the paper names for
+        # negative values; the logarithms are taken on the host in float64 (input preparation, not the method)
+        import numpy as np
+        assert cid == 4
+        with np.errstate(divide="ignore"):
+            for src, dst in (("a", "log_a"), ("b", "log_b"), ("x0", "log_x0")):
+                v = w.tensors.pop(src).astype(np.float64)
+                z = np.empty(v.shape, dtype=np.complex64)
+                z.real = np.log(np.abs(v))
+                z.imag = np.where(v < 0, np.float32(np.pi), np.float32(0))
+                w.tensors[dst] = z
+        w.kind, w.storage = "log", "c64"
     return w
 
 
@@ -177,8 +191,11 @@ def mufu_per_element(w):
     return 4 if w.kind == "linear" else 2
 
 
+ELEMENT_BYTES = {"f32": 4, "bf16": 2, "c64": 8}
+
+
 def algorithmic_bytes(w):
-    es = 4 if w.storage == "f32" else 2
+    es = ELEMENT_BYTES[w.storage]
     return w.rows * w.n * 3 * es + w.rows * es   # two inputs read once, one output written once, x0
 
 
@@ -199,11 +216,17 @@ class DeviceWorkload:
         base = [dev_tensor(w.tensors[k]) for k in input_keys(w)]
         self.sets = [base] + [[x.clone() for x in base] for _ in range(nsets - 1)]
         self.outs = [torch.empty((w.rows, w.n), dtype=base[0].dtype, device=dev) for _ in range(nsets)]
-        self.wss = [hs.new_workspace(w.rows, w.n, dev) for _ in range(nsets)]
+        if w.storage == "c64":
+            nbytes = int(hs.lib().heinsen_scan_complex_workspace_bytes(w.rows, w.n))
+            self.wss = [torch.empty(nbytes, dtype=torch.uint8, device=dev) for _ in range(nsets)]
+        else:
+            self.wss = [hs.new_workspace(w.rows, w.n, dev) for _ in range(nsets)]
 
     def step(self, i):
         s, hs = i % self.nsets, self.hs
-        if self.w.kind == "linear":
+        if self.w.storage == "c64":
+            hs.scan_log_complex(*self.sets[s], log_x=self.outs[s], workspace=self.wss[s])
+        elif self.w.kind == "linear":
             hs.scan_linear(*self.sets[s], x=self.outs[s], workspace=self.wss[s])
         else:
             hs.scan_log(*self.sets[s], log_x=self.outs[s], workspace=self.wss[s])
@@ -242,7 +265,7 @@ def roofline_record(w, us_per_step, clocks, peak, peak_source, mufu_rate, kernel
     achieved = alg_bytes / (us_per_step * 1e-6) / 1e9
     rec = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": t_hbm / us_per_step,
            "traffic": traffic, "peak_source": peak_source, "kernel": kernel,
-           "algorithmic_bytes_per_launch": alg_bytes, "bytes_per_element": 3 * (4 if w.storage == "f32" else 2),
+           "algorithmic_bytes_per_launch": alg_bytes, "bytes_per_element": 3 * ELEMENT_BYTES[w.storage],
            "hbm": {"time_us": t_hbm, "frac": t_hbm / us_per_step},
            "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS}
     if mufu_rate and clocks.get("sm_mhz"):
@@ -505,10 +528,10 @@ def run_ours(args):
         # the headline workload again as repeated batches, then the other configurations
         del dw
         torch.cuda.empty_cache()
-        for c, variant in ((2, None), (4, None), (5, None), (3, None), (3, "linear"), (3, "bf16")):
+        for c, variant in ((2, None), (4, None), (4, "complex"), (5, None), (3, None), (3, "linear"), (3, "bf16")):
             rec, wl = measure_record(c, variant, dev, local, hs, args, peak, peak_source, mufu_rate, torch)
             k = f"cfg{c}" + (f"_{variant}" if variant else "")
-            if not args.no_cpu_baseline and variant != "bf16":
+            if not args.no_cpu_baseline and variant not in ("bf16", "complex"):
                 rec["cpu_baseline_1core"] = cpu_oracle_rate(wl, 1, budget_s=1.5)
             records[k] = rec
             del wl

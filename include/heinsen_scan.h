@@ -209,10 +209,12 @@ size_t heinsen_scan_static_max_elements(void);
  * a negative v (principal branch: log(-r) = log r + i*pi); log 0 = (-inf, anything).
  *   log_a, log_b : device, [rows,n] complex64;  log_x0: device, [rows] complex64.
  *   log_x        : device, [rows,n] complex64 = (log|x_t|, 0 or pi); an exact zero is (-inf, 0).
- *   workspace    : device, at least heinsen_scan_complex_workspace_bytes(rows, n) bytes,
- *                  256-byte aligned (15 bytes per element: the values are split into the
- *                  magnitude and sign planes of the sign+magnitude kernels, scanned there, and
- *                  joined again; the scan itself is the same single-pass kernel).
+ *   workspace    : device, at least heinsen_scan_complex_workspace_bytes(rows, n) bytes, 256-byte
+ *                  aligned: header and look-back descriptors only, as for heinsen_scan_log.  The kernels
+ *                  read the complex elements themselves (magnitude from the real part, sign bit from the
+ *                  parity of the imaginary part over pi) and write complex elements: 24 bytes of traffic
+ *                  per element, nothing staged in between.
+ *   n            : at most half the limit of the other entry points (a row is addressed as 2n floats).
  * Device-side errors: heinsen_scan_check(workspace, stream).
  */
 hs_status heinsen_scan_log_complex(const void* log_a, const void* log_b, const void* log_x0, void* log_x,

@@ -32,7 +32,9 @@ constexpr int kBatchedMinRowsPerSm = 8;  // fewer rows per SM than this: look-ba
 constexpr int kBatchedMinWarpsPerSm = 12; // rows per warp are chosen to keep at least this many warps per SM
 constexpr int kLookbackMinWarps = 8;     // fewest compute warps (= chunks per tile) of the look-back kernel
 constexpr int kLookbackWarps = 14;       // default compute warps of the look-back kernel
-constexpr int kMinChunk = 512;           // smallest chunk (32 lanes x 16 elements)
+constexpr int kMinChunk = 512;           // smallest chunk of the real storage types (32 lanes x 16 elements)
+constexpr int kComplexChunk = 256;       // chunk of the complex-logarithm storage type (32 lanes x 8 elements)
+constexpr hs_dtype kC64 = static_cast<hs_dtype>(2);  // internal: complex64 elements (heinsen_scan_log_complex)
 
 unsigned long long next_call_id() {
     static std::atomic<unsigned long long> counter{[] {
@@ -102,6 +104,8 @@ EncodeFn encode_fn() {
 bool encode_tmap(CUtensorMap* tm, const void* ptr, hs_dtype dt, long long rows, long long n, int box_rows, bool flat) {
     EncodeFn fn = encode_fn();
     if (!fn) return false;
+    // complex64 rows are shown to TMA as rows of 2n floats
+    if (dt == kC64) { dt = HS_F32; n *= 2; }
     const int es = (dt == HS_F32) ? 4 : 2;
     const CUtensorMapDataType type = dt == HS_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
     cuuint32_t estr[3] = {1, 1, 1};
@@ -221,7 +225,7 @@ struct KernelEntry {
 template <int MODE, typename TIn, typename TOut, int K, bool TMA>
 KernelEntry entry() {
     KernelEntry e;
-    constexpr int LBK = 16;  // the look-back kernel parks fp32 partial sums: 16 per lane for every type
+    constexpr int LBK = sizeof(TIn) == 8 ? 8 : 16;  // the look-back kernel parks fp32 partial sums: 16 per lane (8 for complex elements)
     e.batched = reinterpret_cast<const void*>(&batched_scan_kernel<MODE, TIn, TOut, K, TMA, false>);
     e.batched_tk = reinterpret_cast<const void*>(&batched_scan_kernel<MODE, TIn, TOut, K, TMA, true>);
     e.lookback = reinterpret_cast<const void*>(&lookback_scan_kernel<MODE, TIn, TOut, LBK, TMA>);
@@ -276,6 +280,7 @@ bool find_kernel(int mode, hs_dtype din, hs_dtype dout, bool tma, KernelEntry& e
         return false;
     }
     if (mode == kLogSigned) {
+        if (din == kC64 && dout == kC64) HS_PICK(kLogSigned, cplx, cplx, 8);
         if (din == HS_F32 && dout == HS_F32) HS_PICK(kLogSigned, float, float, 16);
         if (din == HS_BF16 && dout == HS_BF16) HS_PICK(kLogSigned, bf16, bf16, 32);
         if (din == HS_F32 && dout == HS_BF16) HS_PICK(kLogSigned, float, bf16, 16);
@@ -296,9 +301,9 @@ int choose_path(long long rows, const DeviceInfo& d) {
     return rows >= (long long)kBatchedMinRowsPerSm * d.sm_count ? HS_PATH_BATCHED : HS_PATH_LOOKBACK;
 }
 
-size_t workspace_bytes_for(long long rows, long long n) {
+size_t workspace_bytes_for(long long rows, long long n, int min_chunk = kMinChunk) {
     // sized for the smallest chunk so that it covers every type
-    const long long tpr = lookback_tiles_per_row(n, kMinChunk, kLookbackMinWarps);
+    const long long tpr = lookback_tiles_per_row(n, min_chunk, kLookbackMinWarps);
     const long long gpr = (tpr + 1) / 2;  // groups hold at least 2 tiles
     return sizeof(Header) + (size_t)(rows * (tpr + gpr)) * 16;
 }
@@ -367,7 +372,8 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
     if (st != HS_OK) return st;
     if (dev.cc_major != 10) return HS_ERR_UNSUPPORTED_DEVICE;
 
-    const int es_in = pr.din == HS_F32 ? 4 : 2, es_out = pr.dout == HS_F32 ? 4 : 2;
+    auto elem_size = [](hs_dtype d) { return d == HS_F32 ? 4 : d == HS_BF16 ? 2 : 8; };
+    const int es_in = elem_size(pr.din), es_out = elem_size(pr.dout);
     bool tma = aligned16(p.in_a) && aligned16(p.in_b) && aligned16(p.out) && (p.n * es_in) % 16 == 0 &&
                (p.n * es_out) % 16 == 0 && p.n <= kMaxTmaDim && encode_fn() != nullptr;
     if (knob(kKnobNoTma, 0, 0, 1)) tma = false;
@@ -413,6 +419,7 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         }
         R = knob(kKnobRowsPerWarp, R, 1, 16);
         while (R & (R - 1)) R &= R - 1;  // power of two
+        if (!tma && es_in == 8) R = 1;   // complex elements without TMA: only the one-row-per-warp staging moves 8-byte elements
         p.rows_per_warp = R;
         p.nchunks = (int)((p.n + (32 / R) * ke.K - 1) / ((32 / R) * ke.K));
         const long long groups = (p.rows + R - 1) / R;
@@ -537,50 +544,6 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
     g_last_path.store(path);
     g_launches.fetch_add(1);
     return HS_OK;
-}
-
-// ---------------------------------------------------------------------------------------------
-// Complex-logarithm interface (Summary, last paragraph: the logarithm of a negative value is
-// complex, log r + i*pi on the principal branch).  Values arrive and leave as complex64; the
-// imaginary part divided by pi, modulo 2, is the sign bit of the sign+magnitude kernels.
-constexpr float kPi = 3.14159265358979323846f;
-
-__global__ void __launch_bounds__(256) split_complex_kernel(const float2* __restrict__ z, float* __restrict__ mag,
-                                                            uint8_t* __restrict__ sign, long long count) {
-    const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += stride) {
-        const float2 v = z[i];
-        mag[i] = v.x;
-        sign[i] = (uint8_t)(__float2int_rn(v.y * (1.0f / kPi)) & 1);
-    }
-}
-__global__ void __launch_bounds__(256) join_complex_kernel(const float* __restrict__ mag, const uint8_t* __restrict__ sign,
-                                                           float2* __restrict__ z, long long count) {
-    const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += stride) {
-        z[i] = make_float2(mag[i], (sign[i] & 1) ? kPi : 0.0f);
-    }
-}
-
-struct ComplexLayout {
-    size_t ws, mag_a, mag_b, mag_x, sign_a, sign_b, sign_x, mag_x0, sign_x0, total;
-};
-ComplexLayout complex_layout(long long rows, long long n) {
-    auto up = [](size_t v) { return (v + 255) & ~size_t(255); };
-    const size_t cnt = (size_t)rows * (size_t)n;
-    ComplexLayout L;
-    size_t o = 0;
-    L.ws = o;      o += up(workspace_bytes_for(rows, n));
-    L.mag_a = o;   o += up(cnt * 4);
-    L.mag_b = o;   o += up(cnt * 4);
-    L.mag_x = o;   o += up(cnt * 4);
-    L.sign_a = o;  o += up(cnt);
-    L.sign_b = o;  o += up(cnt);
-    L.sign_x = o;  o += up(cnt);
-    L.mag_x0 = o;  o += up((size_t)rows * 4);
-    L.sign_x0 = o; o += up((size_t)rows);
-    L.total = o;
-    return L;
 }
 
 // Scratch of heinsen_scan_log_static(): lives in the library image, so every GPU that loads the
@@ -735,9 +698,13 @@ hs_status heinsen_scan_log_static(const void* log_a, const void* log_b, const vo
     return run(pr, scratch, kStaticScratchBytes, static_cast<cudaStream_t>(stream), HS_PATH_LOOKBACK);
 }
 
+// Complex-logarithm interface (Summary, last paragraph: the logarithm of a negative value is complex,
+// log r + i*pi on the principal branch).  Values arrive and leave as complex64; the kernels read the
+// magnitude from the real part and one sign bit from the imaginary part of every element as it comes out of
+// shared memory, and write (log|x|, 0 or pi): 24 bytes per element of traffic, the representation's own.
 size_t heinsen_scan_complex_workspace_bytes(int64_t rows, int64_t n) {
     if (rows <= 0 || n <= 0 || rows > 0x7fffffffll || n > kMaxN || rows > (1ll << 62) / n) return 0;
-    return complex_layout(rows, n).total;
+    return workspace_bytes_for(rows, n, kComplexChunk);
 }
 
 hs_status heinsen_scan_log_complex(const void* log_a, const void* log_b, const void* log_x0, void* log_x, int64_t rows,
@@ -745,34 +712,15 @@ hs_status heinsen_scan_log_complex(const void* log_a, const void* log_b, const v
     hs_status st = validate_common(log_a, log_b, log_x0, log_x, rows, n);
     if (st != HS_OK || rows == 0 || n == 0) return st;
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HS_ERR_INVALID_ARG;
-    const ComplexLayout L = complex_layout(rows, n);
-    if (workspace_bytes < L.total) return HS_ERR_WORKSPACE_TOO_SMALL;
-    DeviceInfo dev;
-    st = device_info(dev);
-    if (st != HS_OK) return st;
-    if (dev.cc_major != 10) return HS_ERR_UNSUPPORTED_DEVICE;
-    uint8_t* w = static_cast<uint8_t*>(workspace);
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const long long cnt = (long long)rows * n;
-    auto blocks = [&](long long c) { long long b = (c + 255) / 256; return (int)(b < 8LL * dev.sm_count ? b : 8LL * dev.sm_count); };
-    split_complex_kernel<<<blocks(cnt), 256, 0, s>>>(static_cast<const float2*>(log_a), reinterpret_cast<float*>(w + L.mag_a),
-                                                     w + L.sign_a, cnt);
-    split_complex_kernel<<<blocks(cnt), 256, 0, s>>>(static_cast<const float2*>(log_b), reinterpret_cast<float*>(w + L.mag_b),
-                                                     w + L.sign_b, cnt);
-    split_complex_kernel<<<blocks(rows), 256, 0, s>>>(static_cast<const float2*>(log_x0), reinterpret_cast<float*>(w + L.mag_x0),
-                                                      w + L.sign_x0, rows);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return cuda_fail("split_complex_kernel", e);
-    g_launches.fetch_add(3);
-    st = heinsen_scan_log(w + L.mag_a, w + L.mag_b, w + L.mag_x0, w + L.mag_x, w + L.sign_a, w + L.sign_b, w + L.sign_x0,
-                          w + L.sign_x, rows, n, HS_F32, HS_F32, w + L.ws, workspace_bytes_for(rows, n), stream);
-    if (st != HS_OK) return st;
-    join_complex_kernel<<<blocks(cnt), 256, 0, s>>>(reinterpret_cast<const float*>(w + L.mag_x), w + L.sign_x,
-                                                    static_cast<float2*>(log_x), cnt);
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return cuda_fail("join_complex_kernel", e);
-    g_launches.fetch_add(1);
-    return HS_OK;
+    if (workspace_bytes < workspace_bytes_for(rows, n, kComplexChunk)) return HS_ERR_WORKSPACE_TOO_SMALL;
+    if (n > kMaxN / 2) return HS_ERR_INVALID_ARG;  // a row of 2n floats must still fit the 32-bit column indices
+    Problem pr;
+    std::memset(&pr, 0, sizeof pr);
+    pr.mode = kLogSigned;
+    pr.din = pr.dout = kC64;
+    pr.p.in_a = log_a; pr.p.in_b = log_b; pr.p.x0 = log_x0; pr.p.out = log_x;
+    pr.p.rows = rows; pr.p.n = n;
+    return run(pr, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
 }
 
 hs_status scan_linear(const void* a, const void* b, const void* x0, void* x, int64_t rows, int64_t n) {

@@ -282,6 +282,16 @@ struct Storage<float> {
     __device__ static __forceinline__ void to_smem(uint32_t addr, float v) {
         asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
     }
+    // A storage type may carry the sign of a value itself (complex logarithms do); these do not.
+    static constexpr bool kCarriesSign = false;
+    static constexpr int kTmaScale = 1;  // tensor-map elements per stored element
+    __device__ static __forceinline__ void unpack_signed(uint4 u, float* o, uint32_t*) { unpack(u, o); }
+    __device__ static __forceinline__ uint4 pack_signed(const float* v, const uint32_t*) { return pack(v); }
+    __device__ static __forceinline__ uint32_t sign_from_smem(uint32_t) { return 0u; }
+    __device__ static __forceinline__ uint32_t load_sign(const void*, int64_t) { return 0u; }
+    // one element moved as it is, global -> shared / shared -> global
+    __device__ static __forceinline__ void copy_in(uint32_t addr, const void* p, int64_t i) { to_smem(addr, load(p, i)); }
+    __device__ static __forceinline__ void copy_out(void* p, int64_t i, uint32_t addr) { store(p, i, from_smem(addr)); }
 };
 template <>
 struct Storage<__nv_bfloat16> {
@@ -313,6 +323,73 @@ struct Storage<__nv_bfloat16> {
     __device__ static __forceinline__ void to_smem(uint32_t addr, float v) {
         const __nv_bfloat16 b = __float2bfloat16_rn(v);
         asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(*reinterpret_cast<const unsigned short*>(&b)) : "memory");
+    }
+    static constexpr bool kCarriesSign = false;
+    static constexpr int kTmaScale = 1;
+    __device__ static __forceinline__ void unpack_signed(uint4 u, float* o, uint32_t*) { unpack(u, o); }
+    __device__ static __forceinline__ uint4 pack_signed(const float* v, const uint32_t*) { return pack(v); }
+    __device__ static __forceinline__ uint32_t sign_from_smem(uint32_t) { return 0u; }
+    __device__ static __forceinline__ uint32_t load_sign(const void*, int64_t) { return 0u; }
+    __device__ static __forceinline__ void copy_in(uint32_t addr, const void* p, int64_t i) {
+        asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(((const unsigned short*)p)[i]) : "memory");
+    }
+    __device__ static __forceinline__ void copy_out(void* p, int64_t i, uint32_t addr) {
+        unsigned short h;
+        asm volatile("ld.shared.u16 %0, [%1];" : "=h"(h) : "r"(addr));
+        ((unsigned short*)p)[i] = h;
+    }
+};
+
+// The logarithm of a real number as the paper writes it for negative values (Summary, last paragraph): a
+// complex number (log|v|, k*pi) on the principal branch, k odd for a negative v.  Stored as two floats; the
+// kernels take the magnitude from the real part and one sign bit from the imaginary part, and write
+// (log|x|, 0) or (log|x|, pi).
+struct cplx {
+    float re, im;
+};
+constexpr float kPi = 3.14159265358979323846f;
+template <>
+struct Storage<cplx> {
+    static constexpr int kPerUnit = 2;
+    static constexpr bool kCarriesSign = true;
+    static constexpr int kTmaScale = 2;
+    // parity of round(im / pi) as a sign mask: adding 1.5 * 2^23 leaves the rounded integer in the low mantissa bits
+    __device__ static __forceinline__ uint32_t sign_of(uint32_t im_bits) {
+        return __float_as_uint(fmaf(__uint_as_float(im_bits), 1.0f / kPi, 12582912.0f)) << 31;
+    }
+    __device__ static __forceinline__ uint32_t imag_of(uint32_t sign_mask) { return sign_mask ? __float_as_uint(kPi) : 0u; }
+    __device__ static __forceinline__ void unpack(uint4 u, float* o) {
+        o[0] = __uint_as_float(u.x); o[1] = __uint_as_float(u.z);
+    }
+    __device__ static __forceinline__ void unpack_signed(uint4 u, float* o, uint32_t* sg) {
+        o[0] = __uint_as_float(u.x); o[1] = __uint_as_float(u.z);
+        sg[0] = sign_of(u.y); sg[1] = sign_of(u.w);
+    }
+    __device__ static __forceinline__ uint4 pack_signed(const float* v, const uint32_t* sg) {
+        return make_uint4(__float_as_uint(v[0]), imag_of(sg[0]), __float_as_uint(v[1]), imag_of(sg[1]));
+    }
+    __device__ static __forceinline__ uint4 pack(const float* v) {
+        return make_uint4(__float_as_uint(v[0]), 0u, __float_as_uint(v[1]), 0u);
+    }
+    __device__ static __forceinline__ float load(const void* p, int64_t i) { return ((const cplx*)p)[i].re; }
+    __device__ static __forceinline__ uint32_t load_sign(const void* p, int64_t i) {
+        return sign_of(__float_as_uint(((const cplx*)p)[i].im));
+    }
+    __device__ static __forceinline__ float from_smem(uint32_t addr) { return Storage<float>::from_smem(addr); }
+    __device__ static __forceinline__ uint32_t sign_from_smem(uint32_t addr) {
+        return sign_of(__float_as_uint(Storage<float>::from_smem(addr + 4u)));
+    }
+    __device__ static __forceinline__ void to_smem(uint32_t addr, float v) {  // a positive value of that magnitude
+        asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(v), "f"(0.0f) : "memory");
+    }
+    __device__ static __forceinline__ void copy_in(uint32_t addr, const void* p, int64_t i) {
+        const float2 v = ((const float2*)p)[i];
+        asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(v.x), "f"(v.y) : "memory");
+    }
+    __device__ static __forceinline__ void copy_out(void* p, int64_t i, uint32_t addr) {
+        float2 v;
+        asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
+        ((float2*)p)[i] = v;
     }
 };
 
@@ -359,6 +436,49 @@ struct Shifted<float, K> {
             case 1: put<1>(sm, off, v); break;
             case 2: put<2>(sm, off, v); break;
             default: put<3>(sm, off, v); break;
+        }
+    }
+    __device__ static __forceinline__ void read_signed(uint32_t sm, const uint32_t* off, uint32_t phi, float* v, uint32_t*) {
+        read(sm, off, phi, v);
+    }
+    __device__ static __forceinline__ void write_signed(uint32_t sm, const uint32_t* off, uint32_t phi, const float* v,
+                                                        const uint32_t*) {
+        write(sm, off, phi, v);
+    }
+};
+template <int K>
+struct Shifted<cplx, K> {
+    static constexpr int UNITS = K / 2;
+    // (the chunk starts 0 or 8 bytes into its buffer: elements are 8 bytes wide and 8-byte aligned)
+    template <int SH>
+    __device__ static __forceinline__ void pick(const uint32_t* w, float* v, uint32_t* sg) {
+#pragma unroll
+        for (int t = 0; t < K; ++t) {
+            v[t] = __uint_as_float(w[2 * t + SH]);
+            sg[t] = Storage<cplx>::sign_of(w[2 * t + 1 + SH]);
+        }
+    }
+    __device__ static __forceinline__ void read_signed(uint32_t sm, const uint32_t* off, uint32_t phi, float* v, uint32_t* sg) {
+        uint32_t w[2 * K + 4];
+#pragma unroll
+        for (int j = 0; j <= UNITS; ++j) {
+            const uint4 q = lds128(sm + off[j]);
+            w[4 * j] = q.x; w[4 * j + 1] = q.y; w[4 * j + 2] = q.z; w[4 * j + 3] = q.w;
+        }
+        if (phi) pick<2>(w, v, sg);
+        else pick<0>(w, v, sg);
+    }
+    __device__ static __forceinline__ void write_signed(uint32_t sm, const uint32_t* off, uint32_t phi, const float* v,
+                                                        const uint32_t* sg) {
+        const int sh = phi ? 2 : 0;
+#pragma unroll
+        for (int t = 0; t < K; ++t) {
+            const uint32_t addr0 = sm + off[t >> 1] + (uint32_t)((t & 1) * 8);        // phi == 0
+            const uint32_t addr8 = sm + off[(t + 1) >> 1] + (uint32_t)(((t + 1) & 1) * 8);  // phi == 8
+            const uint32_t addr = sh ? addr8 : addr0;
+            asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(addr), "r"(__float_as_uint(v[t])),
+                         "r"(Storage<cplx>::imag_of(sg[t]))
+                         : "memory");
         }
     }
 };
@@ -417,6 +537,13 @@ struct Shifted<__nv_bfloat16, K> {
             case 6: put<6>(sm, off, v); break;
             default: put<7>(sm, off, v); break;
         }
+    }
+    __device__ static __forceinline__ void read_signed(uint32_t sm, const uint32_t* off, uint32_t phi, float* v, uint32_t*) {
+        read(sm, off, phi, v);
+    }
+    __device__ static __forceinline__ void write_signed(uint32_t sm, const uint32_t* off, uint32_t phi, const float* v,
+                                                        const uint32_t*) {
+        write(sm, off, phi, v);
     }
 };
 
@@ -535,6 +662,22 @@ struct Run {
     __device__ __forceinline__ static void load_a(uint32_t base_a, const uint32_t* off, float* va) {
 #pragma unroll
         for (int j = 0; j < IN_UNITS; ++j) Storage<TIn>::unpack(lds128(base_a + off[j]), va + j * Storage<TIn>::kPerUnit);
+    }
+    // ... with the sign masks, for storage types that carry the sign in the element (sa, sb untouched otherwise)
+    __device__ __forceinline__ static void load_signed(uint32_t base_a, uint32_t base_b, const uint32_t* off, float* va,
+                                                       float* vb, uint32_t* sa, uint32_t* sb) {
+        constexpr int PER = Storage<TIn>::kPerUnit;
+#pragma unroll
+        for (int j = 0; j < IN_UNITS; ++j) {
+            Storage<TIn>::unpack_signed(lds128(base_a + off[j]), va + j * PER, sa + (Storage<TIn>::kCarriesSign ? j * PER : 0));
+            Storage<TIn>::unpack_signed(lds128(base_b + off[j]), vb + j * PER, sb + (Storage<TIn>::kCarriesSign ? j * PER : 0));
+        }
+    }
+    __device__ __forceinline__ static void load_a_signed(uint32_t base_a, const uint32_t* off, float* va, uint32_t* sa) {
+        constexpr int PER = Storage<TIn>::kPerUnit;
+#pragma unroll
+        for (int j = 0; j < IN_UNITS; ++j)
+            Storage<TIn>::unpack_signed(lds128(base_a + off[j]), va + j * PER, sa + (Storage<TIn>::kCarriesSign ? j * PER : 0));
     }
 
     // va, vb: the stored inputs (log a, log b for the log modes; a, b for kLinear).

@@ -217,24 +217,40 @@ struct ChunkEngine {
         const uint32_t head_n = head / (uint32_t)sizeof(TOut), tail_n = tail / (uint32_t)sizeof(TOut);
         if ((uint32_t)lane < head_n) {
             const uint32_t b = phi + (uint32_t)lane * (uint32_t)sizeof(TOut);
-            Storage<TOut>::store(dst + b, 0, Storage<TOut>::from_smem(sm_out + chunk_off(1, 0, b)));
+            Storage<TOut>::copy_out(dst + b, 0, sm_out + chunk_off(1, 0, b));
         }
         if ((uint32_t)lane < tail_n) {
             const uint32_t b = phi + nbytes - tail + (uint32_t)lane * (uint32_t)sizeof(TOut);
-            Storage<TOut>::store(dst + b, 0, Storage<TOut>::from_smem(sm_out + chunk_off(1, 0, b)));
+            Storage<TOut>::copy_out(dst + b, 0, sm_out + chunk_off(1, 0, b));
         }
     }
-    // The lane's inputs from a stage, whichever way the chunk got there.
+    // The lane's inputs from a stage, whichever way the chunk got there (sa, sb: filled only by storage types that
+    // carry the sign in the element).
     template <bool PLAIN>
     __device__ static __forceinline__ void read_inputs(uint32_t sm_a, uint32_t sm_b, const Offsets& off, const Wide& wd,
-                                                       float* va, float* vb) {
+                                                       float* va, float* vb, uint32_t* sa, uint32_t* sb) {
         if (PLAIN && wd.on) {
-            Shifted<TIn, K>::read(sm_a, off.in, wd.phi_a, va);
-            Shifted<TIn, K>::read(sm_b, off.in, wd.phi_b, vb);
+            Shifted<TIn, K>::read_signed(sm_a, off.in, wd.phi_a, va, sa);
+            Shifted<TIn, K>::read_signed(sm_b, off.in, wd.phi_b, vb, sb);
         } else {
-            R_::load(sm_a, sm_b, off.in, va, vb);
+            R_::load_signed(sm_a, sm_b, off.in, va, vb, sa, sb);
         }
     }
+    template <bool PLAIN>
+    __device__ static __forceinline__ void write_outputs(uint32_t sm_out, const Offsets& off, const Wide& wd, const float* v,
+                                                         const uint32_t* sg) {
+        if (PLAIN && wd.on) {
+            Shifted<TOut, K>::write_signed(sm_out, off.out, wd.phi_o, v, sg);
+        } else {
+            constexpr int PER = Storage<TOut>::kPerUnit;
+#pragma unroll
+            for (int j = 0; j < OUT_UNITS; ++j)
+                sts128(sm_out + off.out[j], Storage<TOut>::pack_signed(v + j * PER, sg + (Storage<TOut>::kCarriesSign ? j * PER : 0)));
+        }
+    }
+    // whether the sign tensors of the call exist (signed mode with a storage type that does not carry the sign)
+    static constexpr bool SIGN_TENSORS = (MODE == kLogSigned) && !Storage<TIn>::kCarriesSign;
+
     // The outputs of a run whose fast form holds, into the output buffer (and the signs to global memory): unit
     // by unit, so that no more than one unit's worth of outputs is live at a time.
     template <bool PLAIN, int J = 0>
@@ -243,9 +259,9 @@ struct ChunkEngine {
         if constexpr (J < OUT_UNITS) {
             constexpr int PER = Storage<TOut>::kPerUnit;
             float o[PER];
-            uint32_t sg[1];
+            uint32_t sg[MODE == kLogSigned ? PER : 1];
             run.template outputs<J * PER, PER>(ap, o, sg);
-            sts128(sm_out + off.out[J], Storage<TOut>::pack(o));
+            sts128(sm_out + off.out[J], Storage<TOut>::pack_signed(o, sg));
             emit_units<PLAIN, J + 1>(run, ap, sm_out, off);
         }
     }
@@ -253,23 +269,14 @@ struct ChunkEngine {
     __device__ static __forceinline__ void emit_outputs(const Params& p, const R_& run, const typename R_::Applied& ap,
                                                         uint32_t sm_out, const Offsets& off, const Wide& wd, long long idx0,
                                                         long long left) {
-        if (MODE == kLogSigned || (PLAIN && wd.on)) {
+        if (SIGN_TENSORS || (PLAIN && wd.on)) {
             float out_mag[K];
             uint32_t out_sign[MODE == kLogSigned ? K : 1];
             run.template outputs<0, K>(ap, out_mag, out_sign);
-            write_outputs<PLAIN>(sm_out, off, wd, out_mag);
-            if (MODE == kLogSigned) store_signs(p.sign_x, idx0, left, p.sign_vec_ok != 0, out_sign);
+            write_outputs<PLAIN>(sm_out, off, wd, out_mag, out_sign);
+            if (SIGN_TENSORS) store_signs(p.sign_x, idx0, left, p.sign_vec_ok != 0, out_sign);
         } else {
             emit_units<PLAIN>(run, ap, sm_out, off);
-        }
-    }
-    template <bool PLAIN>
-    __device__ static __forceinline__ void write_outputs(uint32_t sm_out, const Offsets& off, const Wide& wd, const float* v) {
-        if (PLAIN && wd.on) {
-            Shifted<TOut, K>::write(sm_out, off.out, wd.phi_o, v);
-        } else {
-#pragma unroll
-            for (int j = 0; j < OUT_UNITS; ++j) sts128(sm_out + off.out[j], Storage<TOut>::pack(v + j * Storage<TOut>::kPerUnit));
         }
     }
 
@@ -322,10 +329,10 @@ struct ChunkEngine {
         for (int t = 0; t < K; ++t) {
             if (t < left) {
                 const uint32_t byte = (uint32_t)((lm.i * K + t) * sizeof(TIn));
-                const uint32_t sa = gsa ? (((uint32_t)gsa[idx0 + t] & 1u) << 31) : 0u;
-                const uint32_t sb = gsb ? (((uint32_t)gsb[idx0 + t] & 1u) << 31) : 0u;
-                e = compose(e, Leaf<MODE, TIn>::get(Storage<TIn>::from_smem(sm_a + chunk_off(lm.R, lm.g, phi_a + byte)),
-                                                    Storage<TIn>::from_smem(sm_b + chunk_off(lm.R, lm.g, phi_b + byte)), sa, sb));
+                const uint32_t at_a = sm_a + chunk_off(lm.R, lm.g, phi_a + byte), at_b = sm_b + chunk_off(lm.R, lm.g, phi_b + byte);
+                const uint32_t sa = gsa ? (((uint32_t)gsa[idx0 + t] & 1u) << 31) : Storage<TIn>::sign_from_smem(at_a);
+                const uint32_t sb = gsb ? (((uint32_t)gsb[idx0 + t] & 1u) << 31) : Storage<TIn>::sign_from_smem(at_b);
+                e = compose(e, Leaf<MODE, TIn>::get(Storage<TIn>::from_smem(at_a), Storage<TIn>::from_smem(at_b), sa, sb));
             }
         }
         return e;
@@ -344,10 +351,10 @@ struct ChunkEngine {
             uint32_t sg = 0u;
             if (t < left) {
                 const uint32_t byte = (uint32_t)((lm.i * K + t) * sizeof(TIn));
-                const uint32_t sa = gsa ? (((uint32_t)gsa[idx0 + t] & 1u) << 31) : 0u;
-                const uint32_t sb = gsb ? (((uint32_t)gsb[idx0 + t] & 1u) << 31) : 0u;
-                st = compose(st, Leaf<MODE, TIn>::get(Storage<TIn>::from_smem(sm_a + chunk_off(lm.R, lm.g, phi_a + byte)),
-                                                     Storage<TIn>::from_smem(sm_b + chunk_off(lm.R, lm.g, phi_b + byte)), sa, sb));
+                const uint32_t at_a = sm_a + chunk_off(lm.R, lm.g, phi_a + byte), at_b = sm_b + chunk_off(lm.R, lm.g, phi_b + byte);
+                const uint32_t sa = gsa ? (((uint32_t)gsa[idx0 + t] & 1u) << 31) : Storage<TIn>::sign_from_smem(at_a);
+                const uint32_t sb = gsb ? (((uint32_t)gsb[idx0 + t] & 1u) << 31) : Storage<TIn>::sign_from_smem(at_b);
+                st = compose(st, Leaf<MODE, TIn>::get(Storage<TIn>::from_smem(at_a), Storage<TIn>::from_smem(at_b), sa, sb));
                 renormalise(st);
                 if (MODE == kLinear) {
                     const float h = ex2(st.m * (0.5f * kLog2e));
@@ -379,23 +386,27 @@ struct ChunkEngine {
                                                   long long col0, bool ragged, const Wide& wd, Pending& pd, E& total) {
         float va[K], vb[K];
         uint32_t sa[MODE == kLogSigned ? K : 1], sb[MODE == kLogSigned ? K : 1];
-        read_inputs<PLAIN>(sm_a, sm_b, off, wd, va, vb);
+        read_inputs<PLAIN>(sm_a, sm_b, off, wd, va, vb, sa, sb);
         const long long left = (row < p.rows) ? p.n - col0 : 0;
         if (ragged) {
 #pragma unroll
             for (int t = 0; t < K; ++t) {
-                if (t >= left) { va[t] = neutral_a<MODE>(); vb[t] = neutral_b<MODE>(); }
+                if (t >= left) {
+                    va[t] = neutral_a<MODE>();
+                    vb[t] = neutral_b<MODE>();
+                    if (MODE == kLogSigned) { sa[t] = 0u; sb[t] = 0u; }
+                }
             }
         }
-        if (MODE == kLogSigned) {
+        if (SIGN_TENSORS) {
             load_signs(p.sign_a, row * p.n + col0, left, p.sign_vec_ok != 0, sa);
             load_signs(p.sign_b, row * p.n + col0, left, p.sign_vec_ok != 0, sb);
         }
         E agg = pd.run.pass1(va, vb, sa, sb);
         pd.slow = __any_sync(0xffffffffu, pd.run.bad);
         if (pd.slow) {
-            agg = slow_pass1(sm_a, sm_b, lm, MODE == kLogSigned ? p.sign_a : nullptr,
-                             MODE == kLogSigned ? p.sign_b : nullptr, row * p.n + col0, left, PLAIN ? wd.phi_a : 0u,
+            agg = slow_pass1(sm_a, sm_b, lm, SIGN_TENSORS ? p.sign_a : nullptr,
+                             SIGN_TENSORS ? p.sign_b : nullptr, row * p.n + col0, left, PLAIN ? wd.phi_a : 0u,
                              PLAIN ? wd.phi_b : 0u);
         }
         row_scan(agg, lane, lm.R, pd.excl, total);
@@ -414,11 +425,11 @@ struct ChunkEngine {
         if (ok) {
             emit_outputs<PLAIN>(p, pd.run, ap, ob, off, wd, row * p.n + col0, left);
         } else {
-            const SlowOut so = slow_apply(entering, sm_a, sm_b, lm, MODE == kLogSigned ? p.sign_a : nullptr,
-                                          MODE == kLogSigned ? p.sign_b : nullptr, row * p.n + col0, left,
+            const SlowOut so = slow_apply(entering, sm_a, sm_b, lm, SIGN_TENSORS ? p.sign_a : nullptr,
+                                          SIGN_TENSORS ? p.sign_b : nullptr, row * p.n + col0, left,
                                           PLAIN ? wd.phi_a : 0u, PLAIN ? wd.phi_b : 0u);
-            write_outputs<PLAIN>(ob, off, wd, so.vals);
-            if (MODE == kLogSigned) store_signs(p.sign_x, row * p.n + col0, left, p.sign_vec_ok != 0, so.sgn);
+            write_outputs<PLAIN>(ob, off, wd, so.vals, so.sgn);
+            if (SIGN_TENSORS) store_signs(p.sign_x, row * p.n + col0, left, p.sign_vec_ok != 0, so.sgn);
         }
     }
 
@@ -430,7 +441,8 @@ struct ChunkEngine {
         r.sg = 0u;
         if (row < p.rows) {
             r.v = Storage<TIn>::load(p.x0, row);
-            if (MODE == kLogSigned && p.sign_x0) r.sg = ((uint32_t)p.sign_x0[row] & 1u) << 31;
+            if (SIGN_TENSORS && p.sign_x0) r.sg = ((uint32_t)p.sign_x0[row] & 1u) << 31;
+            if (Storage<TIn>::kCarriesSign) r.sg = Storage<TIn>::load_sign(p.x0, row);
         }
         return r;
     }
@@ -456,8 +468,13 @@ struct ChunkEngine {
             for (int c = lane; c < lm.W; c += 32) {
                 const bool in = c < left;
                 const uint32_t off = chunk_off(lm.R, rg, (uint32_t)(c * sizeof(TIn)));
-                Storage<TIn>::to_smem(sm_a + off, in ? Storage<TIn>::load(p.in_a, base + c) : neutral_a<MODE>());
-                Storage<TIn>::to_smem(sm_b + off, in ? Storage<TIn>::load(p.in_b, base + c) : neutral_b<MODE>());
+                if (in) {
+                    Storage<TIn>::copy_in(sm_a + off, p.in_a, base + c);
+                    Storage<TIn>::copy_in(sm_b + off, p.in_b, base + c);
+                } else {
+                    Storage<TIn>::to_smem(sm_a + off, neutral_a<MODE>());
+                    Storage<TIn>::to_smem(sm_b + off, neutral_b<MODE>());
+                }
             }
         }
     }
@@ -497,7 +514,7 @@ struct ChunkEngine {
             for (int c = lane; c < lm.W; c += 32) {
                 if (c < left) {
                     const uint32_t off = chunk_off(lm.R, rg, (uint32_t)(c * sizeof(TOut)));
-                    Storage<TOut>::store(p.out, base + c, Storage<TOut>::from_smem(sm_out + off));
+                    Storage<TOut>::copy_out(p.out, base + c, sm_out + off);
                 }
             }
         }
@@ -512,15 +529,15 @@ struct ChunkEngine {
                                                        uint32_t sm_b, int lane, long long row, int colbase) {
         for (int col = (int)(n / IN_LINE) * IN_LINE + lane; col < n; col += 32) {
             const uint32_t off = chunk_off(1, 0, (uint32_t)((col - colbase) * sizeof(TIn)));
-            Storage<TIn>::to_smem(sm_a + off, Storage<TIn>::load(in_a, row * n + col));
-            Storage<TIn>::to_smem(sm_b + off, Storage<TIn>::load(in_b, row * n + col));
+            Storage<TIn>::copy_in(sm_a + off, in_a, row * n + col);
+            Storage<TIn>::copy_in(sm_b + off, in_b, row * n + col);
         }
     }
     __device__ static __noinline__ void tail_store_impl(void* out, long long n, uint32_t sm_out, int lane, long long row,
                                                         int colbase) {
         for (int col = (int)(n / OUT_LINE) * OUT_LINE + lane; col < n; col += 32) {
             const uint32_t off = chunk_off(1, 0, (uint32_t)((col - colbase) * sizeof(TOut)));
-            Storage<TOut>::store(out, row * n + col, Storage<TOut>::from_smem(sm_out + off));
+            Storage<TOut>::copy_out(out, row * n + col, sm_out + off);
         }
     }
     __device__ static __forceinline__ void tail_load(const Params& p, uint32_t sm_a, uint32_t sm_b, int lane, long long row,
@@ -596,7 +613,7 @@ struct WarpPipe {
                 tma_load_3d(in_b(s), tm_b, 0, colbase / IN_PER_BOX, row0, bar);
             }
         } else if (lane < in_boxes) {
-            const int x = colbase + lane * IN_PER_BOX;
+            const int x = (colbase + lane * IN_PER_BOX) * Storage<TIn>::kTmaScale;
             const uint32_t dst = (uint32_t)(lane * R * 128);
             tma_load_2d(in_a(s) + dst, tm_a, x, row0, bar);
             tma_load_2d(in_b(s) + dst, tm_b, x, row0, bar);
@@ -620,7 +637,7 @@ struct WarpPipe {
                 bulk_commit();
             }
         } else if (lane < out_boxes) {
-            const int x = colbase + lane * OUT_PER_BOX;
+            const int x = (colbase + lane * OUT_PER_BOX) * Storage<TOut>::kTmaScale;
             tma_store_2d(tm_o, x, row0, src + (uint32_t)(lane * R * 128));
             bulk_commit();
         }
@@ -1118,7 +1135,7 @@ template <typename TIn, int K, int PAD>
 struct LbStage {
     static constexpr int IN_BYTES = 32 * K * (int)sizeof(TIn);
     static constexpr int IN_BUF = IN_BYTES + PAD;
-    static constexpr bool IN_PLACE = sizeof(TIn) == 4;
+    static constexpr bool IN_PLACE = sizeof(TIn) >= 4;  // the parked fp32 sums fit over the b-tensor chunk
     static constexpr int PARK_OFF = IN_PLACE ? IN_BUF : 2 * IN_BUF;
     static constexpr int BYTES = IN_PLACE ? 2 * IN_BUF : 2 * IN_BUF + 32 * K * 4 + PAD;
     static_assert(PAD != 0 || (BYTES % 1024 == 0 && PARK_OFF % 1024 == 0), "swizzled TMA buffers need 1024-byte alignment");
@@ -1308,7 +1325,7 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                 if (lane == 0) mbar_expect_tx(bar, 2 * ST::IN_BYTES);
                 __syncwarp();
                 if (lane < in_boxes) {
-                    const int x = cb + lane * IN_PER_BOX;
+                    const int x = (cb + lane * IN_PER_BOX) * Storage<TIn>::kTmaScale;
                     tma_load_2d(st_a(istage) + lane * 128, &tm_a, x, ci.row, bar);
                     tma_load_2d(st_b(istage) + lane * 128, &tm_b, x, ci.row, bar);
                 }
@@ -1366,8 +1383,9 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                 CE::template phase1<PLAIN>(p, st_a(st), st_b(st), off, lm, lane, row, col0, colbase + CHUNK > p.n, wd, pd, total);
                 if (!pd.slow) {  // park the partial sums (a slow chunk keeps its inputs instead)
                     const uint32_t pb = st_park(st);
-                    // (wide staging: a lane's inputs reach into the unit after its own, where its neighbour parks)
-                    if (PLAIN) __syncwarp();
+                    // (wide staging: a lane's inputs reach into the unit after its own, where its neighbour parks;
+                    // elements wider than the parked sums: a lane parks over other lanes' inputs)
+                    if (PLAIN || sizeof(TIn) > 4) __syncwarp();
 #pragma unroll
                     for (int jx = 0; jx < K / 4; ++jx) sts128(pb + park_off[jx], Storage<float>::pack(pd.run.s + 4 * jx));
                     if (MODE == kLinear) {
@@ -1427,14 +1445,17 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                         for (int jx = 0; jx < K / 4; ++jx) Storage<float>::unpack(lds128(sm_a + park_off[jx]), va + 4 * jx);
                         run.adopt(va, mine.par);
                     } else {
-                        if (PLAIN) Shifted<TIn, K>::read(sm_a, off.in, wd.phi_a, va);
-                        else R_::load_a(sm_a, off.in, va);
+                        if (PLAIN) Shifted<TIn, K>::read_signed(sm_a, off.in, wd.phi_a, va, sa);
+                        else R_::load_a_signed(sm_a, off.in, va, sa);
                         if (colbase + CHUNK > p.n) {
 #pragma unroll
                             for (int t = 0; t < K; ++t)
-                                if (t >= left) va[t] = neutral_a<MODE>();
+                                if (t >= left) {
+                                    va[t] = neutral_a<MODE>();
+                                    if (MODE == kLogSigned) sa[t] = 0u;
+                                }
                         }
-                        if (MODE == kLogSigned) CE::load_signs(p.sign_a, row * p.n + col0, left, p.sign_vec_ok != 0, sa);
+                        if (CE::SIGN_TENSORS) CE::load_signs(p.sign_a, row * p.n + col0, left, p.sign_vec_ok != 0, sa);
                         run.rebuild(va, sa);
                     }
                     run.r = mine.r;
@@ -1450,13 +1471,15 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                     uint32_t phi_a = PLAIN ? wd.phi_a : 0u, phi_b = PLAIN ? wd.phi_b : 0u;
                     if (!was_slow && ST::IN_PLACE) {
                         // the parked sums replaced the b-tensor chunk: fetch the lane's b values again
+                        __syncwarp();
 #pragma unroll
                         for (int t = 0; t < K; ++t) {
-                            const float v = (t < left) ? Storage<TIn>::load(p.in_b, row * p.n + col0 + t) : neutral_b<MODE>();
-                            Storage<TIn>::to_smem(sm_b + chunk_off(1, 0, (uint32_t)((lane * K + t) * sizeof(TIn))), v);
+                            const uint32_t at = chunk_off(1, 0, (uint32_t)((lane * K + t) * sizeof(TIn)));
+                            if (t < left) Storage<TIn>::copy_in(sm_b + at, p.in_b, row * p.n + col0 + t);
+                            else Storage<TIn>::to_smem(sm_b + at, neutral_b<MODE>());
                             if (MODE == kLinear) {  // A_t replaced the a-tensor chunk as well
-                                const float u = (t < left) ? Storage<TIn>::load(p.in_a, row * p.n + col0 + t) : neutral_a<MODE>();
-                                Storage<TIn>::to_smem(sm_a + chunk_off(1, 0, (uint32_t)((lane * K + t) * sizeof(TIn))), u);
+                                if (t < left) Storage<TIn>::copy_in(sm_a + at, p.in_a, row * p.n + col0 + t);
+                                else Storage<TIn>::to_smem(sm_a + at, neutral_a<MODE>());
                             }
                         }
                         phi_b = 0u;
@@ -1464,11 +1487,11 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                         __syncwarp();
                     }
                     const typename CE::SlowOut so =
-                        CE::slow_apply(entering, sm_a, sm_b, lm, MODE == kLogSigned ? p.sign_a : nullptr,
-                                       MODE == kLogSigned ? p.sign_b : nullptr, row * p.n + col0, left, phi_a, phi_b);
+                        CE::slow_apply(entering, sm_a, sm_b, lm, CE::SIGN_TENSORS ? p.sign_a : nullptr,
+                                       CE::SIGN_TENSORS ? p.sign_b : nullptr, row * p.n + col0, left, phi_a, phi_b);
                     __syncwarp();
-                    CE::template write_outputs<PLAIN>(pb, off, wd, so.vals);
-                    if (MODE == kLogSigned) CE::store_signs(p.sign_x, row * p.n + col0, left, p.sign_vec_ok != 0, so.sgn);
+                    CE::template write_outputs<PLAIN>(pb, off, wd, so.vals, so.sgn);
+                    if (CE::SIGN_TENSORS) CE::store_signs(p.sign_x, row * p.n + col0, left, p.sign_vec_ok != 0, so.sgn);
                 }
                 if (TMA) {
                     fence_async_smem();
@@ -1482,7 +1505,8 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                         }
                         if (colbase == tail_colbase_out) CE::tail_store(p, pb, lane, row, colbase);
                     } else if (lane < out_boxes) {
-                        tma_store_2d(&tm_o, colbase + lane * OUT_PER_BOX, (int)row, pb + (uint32_t)(lane * 128));
+                        tma_store_2d(&tm_o, (colbase + lane * OUT_PER_BOX) * Storage<TOut>::kTmaScale, (int)row,
+                                     pb + (uint32_t)(lane * 128));
                         bulk_commit();
                     }
                 } else {

@@ -81,7 +81,8 @@ struct ChunkEngine<kPairs, TIn, TOut, K> {
                                                   const LaneMap&, int lane, long long row, long long col0, bool ragged,
                                                   const Wide& wd, Pending& pd, E& total) {
         float va[K], vb[K];
-        Base::template read_inputs<PLAIN>(sm_a, sm_b, off, wd, va, vb);
+        uint32_t none[1];
+        Base::template read_inputs<PLAIN>(sm_a, sm_b, off, wd, va, vb, none, none);
         if (ragged) {
             const long long left = (row < p.rows) ? p.n - col0 : 0;
 #pragma unroll
@@ -111,7 +112,8 @@ struct ChunkEngine<kPairs, TIn, TOut, K> {
         float out[K];
 #pragma unroll
         for (int t = 0; t < K; ++t) out[t] = fmaf(pd.P[t], x_in, pd.B[t]);
-        Base::template write_outputs<PLAIN>(sm_out, off, wd, out);
+        const uint32_t none[1] = {0u};
+        Base::template write_outputs<PLAIN>(sm_out, off, wd, out, none);
     }
 
     struct RawX0 { float v; };

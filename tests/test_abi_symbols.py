@@ -56,7 +56,9 @@ def test_host_side_validation_needs_no_gpu(lib):
     assert lib.heinsen_scan_log_static(p, p, p, p, 1 << 20, 4096, None) == TOO_SMALL
     assert lib.heinsen_scan_log_complex(None, p, p, p, 2, 8, aligned, 1 << 20, None) == INVALID
     assert lib.heinsen_scan_log_complex(p, p, p, p, 2, 8, aligned, 64, None) == TOO_SMALL
-    assert lib.heinsen_scan_complex_workspace_bytes(2, 8) >= 256 + 15 * 16
+    # the complex entry point needs the header and the look-back descriptors only (the elements are read as they are)
+    assert 256 <= lib.heinsen_scan_complex_workspace_bytes(2, 8) <= 1024
+    assert lib.heinsen_scan_complex_workspace_bytes(1, 1 << 24) >= lib.heinsen_scan_workspace_bytes(1, 1 << 24)
     assert lib.scan_linear(None, p, p, p, 2, 8) == INVALID and lib.scan_linear(p, p, p, p, 0, 8) == OK
     assert lib.scan_log(p, p, p, p, p, None, None, None, 2, 8) == INVALID and lib.scan_log(p, p, p, p, None, None, None, None, 2, 0) == OK
     assert lib.heinsen_scan_set_path(7) == INVALID and lib.heinsen_scan_set_path(0) == OK

@@ -411,22 +411,47 @@ def test_lookback_several_rows_several_groups(hs, oracle):
 
 
 @pytest.mark.parametrize("path", ["batched", "lookback"])
-def test_complex_logarithm_interface(hs, oracle, path):
+@pytest.mark.parametrize("rows,n,offset", [(40, 3000, 0), (37, 3001, 0), (40, 3000, 1), (2000, 100, 0), (1900, 37, 0),
+                                            (3, 70004, 0), (2, 70001, 1), (300, 256, 0), (5, 1, 0)])
+def test_complex_logarithm_interface(hs, oracle, path, rows, n, offset):
     """Negative a, b, x0 as complex logarithms (log r + i*pi): the result is real, i.e. its imaginary part is
-    0 or pi, and exp of it equals the recurrence in the linear domain."""
-    w = workloads.make(4, rows=40, n=3000)
+    0 or pi, and exp of it equals the recurrence in the linear domain.  Shapes: rows of whole 16-byte units with
+    and without a remainder of the last 128-byte line, an odd number of elements per row and a base that is only
+    8-byte aligned (rows TMA cannot address), rows shorter than a chunk (several rows per warp), long rows."""
+    w = workloads.make(4, rows=rows, n=n)
     a, b, x0 = (w.tensors[k].astype(np.float64) for k in ("a", "b", "x0"))
     with np.errstate(divide="ignore"):
         la, lb, lx0 = (np.log(v.astype(np.complex128)).astype(np.complex64) for v in (a, b, x0))
-    la.imag[::3] += np.float32(2 * np.pi)         # any odd/even multiple of pi is the same sign
-    lb.imag[1::5] -= np.float32(2 * np.pi)
+    la.imag[:, ::3] += np.float32(2 * np.pi)         # any odd/even multiple of pi is the same sign
+    lb.imag[:, 1::5] -= np.float32(2 * np.pi)
     hs.set_path(getattr(hs, "PATH_" + path.upper()))
-    out = hs.scan_log_complex(*(torch.from_numpy(v).cuda() for v in (la, lb, lx0)))
+
+    def place(v):   # at `offset` elements into a larger buffer: offset 1 leaves the base 8-byte aligned only
+        buf = torch.empty(v.size + 2, dtype=torch.complex64, device="cuda")
+        view = buf[offset:offset + v.size].view(v.shape)
+        view.copy_(torch.from_numpy(v))
+        return view
+
+    d_la, d_lb, d_lx0 = place(la), place(lb), torch.from_numpy(lx0).cuda()
+    out_buf = torch.full((rows * n + 2,), float("nan"), dtype=torch.complex64, device="cuda")
+    out = out_buf[offset:offset + rows * n].view(rows, n)
+    hs.scan_log_complex(d_la, d_lb, d_lx0, log_x=out)
+    torch.cuda.synchronize()
     z = out.cpu().numpy()
+    edge = out_buf.cpu().numpy()
+    assert np.isnan(edge[:offset].real).all() and np.isnan(edge[offset + rows * n:].real).all(), "wrote outside the output"
     assert np.isin(np.round(z.imag / np.pi), (0, 1)).all() and np.allclose(z.imag, np.round(z.imag / np.pi) * np.pi, atol=1e-6)
     got = np.exp(z.real.astype(np.float64)) * np.where(np.round(z.imag / np.pi) == 1, -1.0, 1.0)
     ref = oracle.scan_linear(w.tensors["a"], w.tensors["b"], w.tensors["x0"])
-    assert_signed_close(got, ref, f"complex interface/{path}")
+    assert_signed_close(got, ref, f"complex interface/{path} {rows}x{n}+{offset}")
+    # the same values through the sign + magnitude entry point: same kernels apart from where the sign bit comes from
+    mag = lambda v: torch.from_numpy(np.ascontiguousarray(v.real)).cuda()
+    sgn = lambda v: torch.from_numpy((np.round(v.imag / np.pi).astype(np.int64) & 1).astype(np.uint8)).cuda()
+    lx2, sx2 = hs.scan_log(mag(la), mag(lb), mag(lx0), sign_a=sgn(la), sign_b=sgn(lb), sign_x0=sgn(lx0))
+    torch.cuda.synchronize()
+    got2 = np.exp(to_f64(lx2)) * np.where(sx2.cpu().numpy() == 1, -1.0, 1.0)
+    assert_signed_close(got2, ref, "sign + magnitude entry point on the same values")
+    assert np.abs(got - got2).max() <= 2e-3 * np.abs(ref).max()   # (near a cancellation log|x| itself is ill-conditioned)
 
 
 def test_short_forms_of_the_two_calls(hs, oracle):
