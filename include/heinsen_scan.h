@@ -246,6 +246,23 @@ hs_status heinsen_scan_set_path(hs_path path);
  */
 hs_status heinsen_scan_debug_config(uint32_t lookback_spin_limit, int64_t mute_tile);
 /*
+ * Checked build (the library compiled with -DHEINSEN_DEBUG; `python -m paper_2311_06281_b200.build_ext --debug`
+ * writes it beside the normal one as libheinsen_scan_debug.so).  In that build every shared-memory access of
+ * the kernels checks its address against the CTA's shared-memory window and its alignment, and the kernels
+ * check the element, row, tile and TMA coordinates they are about to use.  A failed check never traps: it is
+ * recorded and the access is skipped.
+ *   heinsen_scan_debug_build()  : 1 in the checked build, 0 otherwise.
+ *   heinsen_scan_debug_faults() : synchronises the device, copies the first recorded failure of the process to
+ *                                 out[0..3] = {check code, detail (address or index), block, thread}, clears the
+ *                                 record, and returns 1; 0 when nothing was recorded (always, in the normal
+ *                                 build); -1 on a CUDA error.  `out` may be NULL.
+ *   heinsen_scan_debug_window_ok(): the window predicate of those checks (addr, bytes inside [base, base + size),
+ *                                 addr a multiple of align), exported so that it can be tested without a GPU.
+ */
+int heinsen_scan_debug_build(void);
+int heinsen_scan_debug_faults(uint64_t out[4]);
+int heinsen_scan_debug_window_ok(uint64_t addr, uint64_t bytes, uint64_t base, uint64_t size, uint64_t align);
+/*
  * Tuning knobs, for sweeps and for tests that force a variant; every knob has a measured default
  * that is chosen per call.  `name` is one of "NO_TMA", "ROWS_PER_WARP", "WARPS", "STAGES",
  * "ROW_TICKETS", "NO_FLAT", "NO_PDL" (row-batched kernel), "LB_STAGES", "LB_WARPS", "LB_GROUP",

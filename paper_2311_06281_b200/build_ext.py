@@ -21,27 +21,34 @@ def _nvcc() -> str:
     return "nvcc"
 
 
-def is_stale() -> bool:
-    if not os.path.exists(LIB):
+DEBUG_LIB = os.path.join(_HERE, "libheinsen_scan_debug.so")
+
+
+def is_stale(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     deps = [os.path.join(CSRC, f) for f in SOURCES + HEADERS] + [os.path.abspath(__file__)]
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile the library if it is missing or older than its sources; return its path."""
-    if force or is_stale():
-        tmp = f"{LIB}.{os.getpid()}.tmp"
-        cmd = [_nvcc(), *NVCC_FLAGS, "-o", tmp, *[os.path.join(CSRC, s) for s in SOURCES]]
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """Compile the library if it is missing or older than its sources; return its path.
+    debug=True builds the checked variant (-DHEINSEN_DEBUG: index checks that record instead of trapping)
+    beside the normal one."""
+    lib = DEBUG_LIB if debug else LIB
+    if force or is_stale(lib):
+        tmp = f"{lib}.{os.getpid()}.tmp"
+        cmd = [_nvcc(), *NVCC_FLAGS, *(["-DHEINSEN_DEBUG"] if debug else []), "-o", tmp,
+               *[os.path.join(CSRC, s) for s in SOURCES]]
         if verbose:
             cmd.insert(1, "-Xptxas")
             cmd.insert(2, "-v")
             print(" ".join(cmd), file=sys.stderr)
         subprocess.check_call(cmd, cwd=CSRC)
-        os.replace(tmp, LIB)
-    return LIB
+        os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

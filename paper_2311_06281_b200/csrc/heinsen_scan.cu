@@ -791,6 +791,34 @@ hs_status heinsen_scan_debug_config(uint32_t lookback_spin_limit, int64_t mute_t
     g_mute_tile.store(mute_tile);
     return HS_OK;
 }
+int heinsen_scan_debug_faults(uint64_t out[4]) {
+    if (out) out[0] = out[1] = out[2] = out[3] = 0;
+#ifdef HEINSEN_DEBUG
+    unsigned long long f[4] = {0, 0, 0, 0};
+    if (cudaDeviceSynchronize() != cudaSuccess) return -1;
+    if (cudaMemcpyFromSymbol(f, hs::g_debug_fault, sizeof f) != cudaSuccess) return -1;
+    if (f[0] != 0) {
+        const unsigned long long zero[4] = {0, 0, 0, 0};
+        if (cudaMemcpyToSymbol(hs::g_debug_fault, zero, sizeof zero) != cudaSuccess) return -1;
+    }
+    if (out) for (int i = 0; i < 4; ++i) out[i] = f[i];
+    return f[0] != 0 ? 1 : 0;
+#else
+    return 0;
+#endif
+}
+int heinsen_scan_debug_build(void) {
+#ifdef HEINSEN_DEBUG
+    return 1;
+#else
+    return 0;
+#endif
+}
+int heinsen_scan_debug_window_ok(uint64_t addr, uint64_t bytes, uint64_t base, uint64_t size, uint64_t align) {
+    if (align == 0) return 0;
+    return hs::debug_window_ok(addr, bytes, base, size, align) ? 1 : 0;
+}
+
 hs_status heinsen_scan_tune(const char* name, int value) {
     if (!name) return HS_ERR_INVALID_ARG;
     std::call_once(g_knobs_once, load_knobs_from_env);

@@ -251,12 +251,70 @@ __device__ __forceinline__ uint32_t chunk_off(int R, int g, uint32_t byte_in_row
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
+// ------------------------------------------------------------------------------------------
+// Checked build (-DHEINSEN_DEBUG).  compute-sanitizer is not always available where this library runs, so
+// the library can be built with its own index checks: every shared-memory access of the wrappers below
+// verifies that its address lies inside the CTA's dynamic shared memory and is aligned to its width, and the
+// kernels verify the element, row, tile and TMA coordinates they are about to use (HS_DBG_CHECK).  A check
+// that fails never traps: it records {code, detail, block, thread} in g_debug_fault (the first failure of a
+// process wins; heinsen_scan_debug_faults() reads and clears it) and the access is skipped.  In the normal
+// build all of this compiles to nothing.
+// The predicate itself is plain arithmetic, shared with the host so that it can be unit-tested without a GPU.
+__host__ __device__ inline bool debug_window_ok(unsigned long long addr, unsigned long long bytes, unsigned long long base,
+                                                unsigned long long size, unsigned long long align) {
+    return addr >= base && bytes <= size && addr - base <= size - bytes && (addr % align) == 0;
+}
+enum DebugCode : int {
+    kDbgSmemWindow = 1,   // shared-memory address outside the CTA's dynamic shared memory, or misaligned
+    kDbgElement = 2,      // element index outside [0, rows * n)
+    kDbgRow = 3,          // row index outside [0, rows)
+    kDbgTile = 4,         // tile / group descriptor index outside the descriptor arrays
+    kDbgTmaCoord = 5,     // TMA coordinate out of range or not on a 16-byte boundary
+    kDbgUnits = 6         // 16-byte unit copy reaching beyond the units that hold the tensor
+};
+#ifdef HEINSEN_DEBUG
+__device__ unsigned long long g_debug_fault[4];
+__device__ __noinline__ void debug_record(int code, unsigned long long detail) {
+    if (atomicCAS(&g_debug_fault[0], 0ull, (unsigned long long)code) == 0ull) {
+        g_debug_fault[1] = detail;
+        g_debug_fault[2] = blockIdx.x;
+        g_debug_fault[3] = threadIdx.x;
+    }
+}
+__device__ __forceinline__ bool debug_smem_ok(uint32_t addr, uint32_t bytes) {
+    extern __shared__ uint8_t hs_debug_dynamic_smem[];
+    uint32_t size;
+    asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(size));
+    const uint32_t base = smem_u32(hs_debug_dynamic_smem);
+    if (debug_window_ok(addr, bytes, base, size, bytes)) return true;
+    debug_record(kDbgSmemWindow, ((unsigned long long)addr << 32) | bytes);
+    return false;
+}
+#define HS_DBG_SMEM(addr, bytes, fail) \
+    do {                               \
+        if (!debug_smem_ok((addr), (bytes))) fail; \
+    } while (0)
+// `cond` must hold; otherwise the failure is recorded and `fail` runs (skip the access)
+#define HS_DBG_CHECK(cond, code, detail, fail)                               \
+    do {                                                                     \
+        if (!(cond)) {                                                       \
+            debug_record((code), (unsigned long long)(detail));              \
+            fail;                                                            \
+        }                                                                    \
+    } while (0)
+#else
+#define HS_DBG_SMEM(addr, bytes, fail) do { } while (0)
+#define HS_DBG_CHECK(cond, code, detail, fail) do { } while (0)
+#endif
+
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 v;
+    HS_DBG_SMEM(addr, 16u, return make_uint4(0u, 0u, 0u, 0u));
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
     return v;
 }
 __device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
+    HS_DBG_SMEM(addr, 16u, return);
     asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
@@ -276,10 +334,12 @@ struct Storage<float> {
     // addr: 32-bit shared-memory address
     __device__ static __forceinline__ float from_smem(uint32_t addr) {
         float v;
+        HS_DBG_SMEM(addr, 4u, return 0.0f);
         asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
         return v;
     }
     __device__ static __forceinline__ void to_smem(uint32_t addr, float v) {
+        HS_DBG_SMEM(addr, 4u, return);
         asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
     }
     // A storage type may carry the sign of a value itself (complex logarithms do); these do not.
@@ -317,11 +377,13 @@ struct Storage<__nv_bfloat16> {
     }
     __device__ static __forceinline__ float from_smem(uint32_t addr) {
         unsigned short h;
+        HS_DBG_SMEM(addr, 2u, return 0.0f);
         asm volatile("ld.shared.u16 %0, [%1];" : "=h"(h) : "r"(addr));
         return __uint_as_float((uint32_t)h << 16);
     }
     __device__ static __forceinline__ void to_smem(uint32_t addr, float v) {
         const __nv_bfloat16 b = __float2bfloat16_rn(v);
+        HS_DBG_SMEM(addr, 2u, return);
         asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(*reinterpret_cast<const unsigned short*>(&b)) : "memory");
     }
     static constexpr bool kCarriesSign = false;
@@ -331,10 +393,12 @@ struct Storage<__nv_bfloat16> {
     __device__ static __forceinline__ uint32_t sign_from_smem(uint32_t) { return 0u; }
     __device__ static __forceinline__ uint32_t load_sign(const void*, int64_t) { return 0u; }
     __device__ static __forceinline__ void copy_in(uint32_t addr, const void* p, int64_t i) {
+        HS_DBG_SMEM(addr, 2u, return);
         asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(((const unsigned short*)p)[i]) : "memory");
     }
     __device__ static __forceinline__ void copy_out(void* p, int64_t i, uint32_t addr) {
         unsigned short h;
+        HS_DBG_SMEM(addr, 2u, return);
         asm volatile("ld.shared.u16 %0, [%1];" : "=h"(h) : "r"(addr));
         ((unsigned short*)p)[i] = h;
     }
@@ -380,14 +444,17 @@ struct Storage<cplx> {
         return sign_of(__float_as_uint(Storage<float>::from_smem(addr + 4u)));
     }
     __device__ static __forceinline__ void to_smem(uint32_t addr, float v) {  // a positive value of that magnitude
+        HS_DBG_SMEM(addr, 8u, return);
         asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(v), "f"(0.0f) : "memory");
     }
     __device__ static __forceinline__ void copy_in(uint32_t addr, const void* p, int64_t i) {
         const float2 v = ((const float2*)p)[i];
+        HS_DBG_SMEM(addr, 8u, return);
         asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(v.x), "f"(v.y) : "memory");
     }
     __device__ static __forceinline__ void copy_out(void* p, int64_t i, uint32_t addr) {
         float2 v;
+        HS_DBG_SMEM(addr, 8u, return);
         asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
         ((float2*)p)[i] = v;
     }
@@ -399,9 +466,11 @@ struct Storage<cplx> {
 // `off` holds the shared-memory offsets of the lane's K / kPerUnit units and of the one after them; which
 // words of those units are the lane's depends on phi only, so every shift is a statically indexed variant.
 __device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) {
+    HS_DBG_SMEM(addr, 4u, return);
     asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
 __device__ __forceinline__ void sts16(uint32_t addr, uint32_t v) {
+    HS_DBG_SMEM(addr, 2u, return);
     asm volatile("st.shared.b16 [%0], %1;" ::"r"(addr), "h"((unsigned short)v) : "memory");
 }
 template <typename T, int K>
@@ -476,6 +545,7 @@ struct Shifted<cplx, K> {
             const uint32_t addr0 = sm + off[t >> 1] + (uint32_t)((t & 1) * 8);        // phi == 0
             const uint32_t addr8 = sm + off[(t + 1) >> 1] + (uint32_t)(((t + 1) & 1) * 8);  // phi == 8
             const uint32_t addr = sh ? addr8 : addr0;
+            HS_DBG_SMEM(addr, 8u, continue);
             asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(addr), "r"(__float_as_uint(v[t])),
                          "r"(Storage<cplx>::imag_of(sg[t]))
                          : "memory");
@@ -579,10 +649,13 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 
 // Asynchronous 4-byte copy global -> shared (for rows that TMA cannot address), with its group bookkeeping.
 __device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
+    HS_DBG_SMEM(dst, 4u, return);
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
 }
 // ... and 16-byte copy (both addresses 16-byte aligned), past L1.
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    HS_DBG_SMEM(dst, 16u, return);
+    HS_DBG_CHECK((reinterpret_cast<uintptr_t>(src) & 15u) == 0, kDbgUnits, reinterpret_cast<uintptr_t>(src), return);
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }

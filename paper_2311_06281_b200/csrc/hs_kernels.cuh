@@ -176,8 +176,8 @@ struct ChunkEngine {
     // asynchronous copies per call, committed by the caller).  The first and the last unit may reach a few bytes
     // beyond the row: they are units that also hold bytes of the row, so they lie in mapped memory.
     template <typename T>
-    __device__ static __forceinline__ void wide_copy_in(const void* tensor, uint32_t sm, int lane, long long elem0, long long left,
-                                                        int W) {
+    __device__ static __forceinline__ void wide_copy_in(const void* tensor, long long total, uint32_t sm, int lane, long long elem0,
+                                                        long long left, int W) {
         const uintptr_t g0 = reinterpret_cast<uintptr_t>(tensor) + (size_t)elem0 * sizeof(T);
         const uint32_t phi = (uint32_t)(g0 & 15u);
         const long long valid = left < W ? left : W;
@@ -187,14 +187,20 @@ struct ChunkEngine {
 #pragma unroll
         for (int q = 0; q < ROUNDS; ++q) {
             const int u = q * 32 + lane;
-            if (u < nunits) cp_async16(sm + chunk_off(1, 0, (uint32_t)(u * 16)), src + 16 * u);
+            if (u < nunits) {
+                HS_DBG_CHECK(reinterpret_cast<uintptr_t>(src) + 16u * (unsigned)u + 16u > reinterpret_cast<uintptr_t>(tensor) &&
+                                 reinterpret_cast<uintptr_t>(src) + 16u * (unsigned)u <
+                                     reinterpret_cast<uintptr_t>(tensor) + (size_t)total * sizeof(T),
+                             kDbgUnits, elem0, continue);
+                cp_async16(sm + chunk_off(1, 0, (uint32_t)(u * 16)), src + 16 * u);
+            }
         }
     }
     __device__ static __forceinline__ void wide_load_async(const Params& p, uint32_t sm_a, uint32_t sm_b, int lane, long long row,
                                                            long long colbase, int W) {
         const long long left = row < p.rows ? p.n - colbase : 0;
-        wide_copy_in<TIn>(p.in_a, sm_a, lane, row * p.n + colbase, left, W);
-        wide_copy_in<TIn>(p.in_b, sm_b, lane, row * p.n + colbase, left, W);
+        wide_copy_in<TIn>(p.in_a, p.rows * p.n, sm_a, lane, row * p.n + colbase, left, W);
+        wide_copy_in<TIn>(p.in_b, p.rows * p.n, sm_b, lane, row * p.n + colbase, left, W);
         cp_async_commit();
     }
     // The chunk's outputs, written by the lanes phi_o bytes into the buffer, go out as whole 16-byte units
@@ -212,8 +218,12 @@ struct ChunkEngine {
         const uint32_t tail = nbytes - head - (body << 4);                              // bytes of the last, partial unit
         char* const dst = reinterpret_cast<char*>(g0 - phi);
         const uint32_t u0 = phi ? 1u : 0u;
-        for (uint32_t u = (uint32_t)lane; u < body; u += 32u)
+        for (uint32_t u = (uint32_t)lane; u < body; u += 32u) {
+            HS_DBG_CHECK(dst + 16u * (u0 + u) >= reinterpret_cast<char*>(p.out) &&
+                             dst + 16u * (u0 + u) + 16u <= reinterpret_cast<char*>(p.out) + (size_t)(p.rows * p.n) * sizeof(TOut),
+                         kDbgUnits, row * p.n + colbase, continue);
             *reinterpret_cast<uint4*>(dst + 16u * (u0 + u)) = lds128(sm_out + chunk_off(1, 0, 16u * (u0 + u)));
+        }
         const uint32_t head_n = head / (uint32_t)sizeof(TOut), tail_n = tail / (uint32_t)sizeof(TOut);
         if ((uint32_t)lane < head_n) {
             const uint32_t b = phi + (uint32_t)lane * (uint32_t)sizeof(TOut);
@@ -290,6 +300,7 @@ struct ChunkEngine {
             return;
         }
         if (vec && left >= K) {
+            HS_DBG_CHECK(idx0 >= 0 && (idx0 & 15) == 0, kDbgElement, idx0, return);
 #pragma unroll
             for (int j = 0; j < K / 16; ++j) {
                 const uint4 v = __ldg(reinterpret_cast<const uint4*>(g + idx0 + 16 * j));
@@ -305,6 +316,7 @@ struct ChunkEngine {
     __device__ static __forceinline__ void store_signs(uint8_t* g, long long idx0, long long left, bool vec,
                                                        const uint32_t* mask) {
         if (vec && left >= K) {
+            HS_DBG_CHECK(idx0 >= 0 && (idx0 & 15) == 0, kDbgElement, idx0, return);
 #pragma unroll
             for (int j = 0; j < K / 16; ++j) {
                 uint32_t w[4] = {0u, 0u, 0u, 0u};
@@ -468,6 +480,7 @@ struct ChunkEngine {
             for (int c = lane; c < lm.W; c += 32) {
                 const bool in = c < left;
                 const uint32_t off = chunk_off(lm.R, rg, (uint32_t)(c * sizeof(TIn)));
+                HS_DBG_CHECK(!in || (base + c >= 0 && base + c < p.rows * p.n), kDbgElement, base + c, continue);
                 if (in) {
                     Storage<TIn>::copy_in(sm_a + off, p.in_a, base + c);
                     Storage<TIn>::copy_in(sm_b + off, p.in_b, base + c);
@@ -493,6 +506,7 @@ struct ChunkEngine {
             for (int c = lane; c < lm.W; c += 32) {
                 const uint32_t off = chunk_off(lm.R, rg, (uint32_t)(c * sizeof(TIn)));
                 if (c < left) {
+                    HS_DBG_CHECK(row >= 0 && row < p.rows && colbase + c < p.n, kDbgElement, row * p.n + colbase + c, continue);
                     cp_async4(sm_a + off, pa + c);
                     cp_async4(sm_b + off, pb + c);
                 } else {
@@ -514,6 +528,7 @@ struct ChunkEngine {
             for (int c = lane; c < lm.W; c += 32) {
                 if (c < left) {
                     const uint32_t off = chunk_off(lm.R, rg, (uint32_t)(c * sizeof(TOut)));
+                    HS_DBG_CHECK(base + c >= 0 && base + c < p.rows * p.n, kDbgElement, base + c, continue);
                     Storage<TOut>::copy_out(p.out, base + c, sm_out + off);
                 }
             }
@@ -525,27 +540,29 @@ struct ChunkEngine {
     // (one row per warp; colbase: first column of that chunk).
     static constexpr int IN_LINE = 128 / (int)sizeof(TIn), OUT_LINE = 128 / (int)sizeof(TOut);
     // (out of line: rare, and the chunk loop should stay small)
-    __device__ static __noinline__ void tail_load_impl(const void* in_a, const void* in_b, long long n, uint32_t sm_a,
-                                                       uint32_t sm_b, int lane, long long row, int colbase) {
+    __device__ static __noinline__ void tail_load_impl(const void* in_a, const void* in_b, long long n, long long rows,
+                                                       uint32_t sm_a, uint32_t sm_b, int lane, long long row, int colbase) {
         for (int col = (int)(n / IN_LINE) * IN_LINE + lane; col < n; col += 32) {
             const uint32_t off = chunk_off(1, 0, (uint32_t)((col - colbase) * sizeof(TIn)));
+            HS_DBG_CHECK(row >= 0 && row < rows && col >= colbase, kDbgElement, row * n + col, continue);
             Storage<TIn>::copy_in(sm_a + off, in_a, row * n + col);
             Storage<TIn>::copy_in(sm_b + off, in_b, row * n + col);
         }
     }
-    __device__ static __noinline__ void tail_store_impl(void* out, long long n, uint32_t sm_out, int lane, long long row,
-                                                        int colbase) {
+    __device__ static __noinline__ void tail_store_impl(void* out, long long n, long long rows, uint32_t sm_out, int lane,
+                                                        long long row, int colbase) {
         for (int col = (int)(n / OUT_LINE) * OUT_LINE + lane; col < n; col += 32) {
             const uint32_t off = chunk_off(1, 0, (uint32_t)((col - colbase) * sizeof(TOut)));
+            HS_DBG_CHECK(row >= 0 && row < rows && col >= colbase, kDbgElement, row * n + col, continue);
             Storage<TOut>::copy_out(out, row * n + col, sm_out + off);
         }
     }
     __device__ static __forceinline__ void tail_load(const Params& p, uint32_t sm_a, uint32_t sm_b, int lane, long long row,
                                                      int colbase) {
-        tail_load_impl(p.in_a, p.in_b, p.n, sm_a, sm_b, lane, row, colbase);
+        tail_load_impl(p.in_a, p.in_b, p.n, p.rows, sm_a, sm_b, lane, row, colbase);
     }
     __device__ static __forceinline__ void tail_store(const Params& p, uint32_t sm_out, int lane, long long row, int colbase) {
-        tail_store_impl(p.out, p.n, sm_out, lane, row, colbase);
+        tail_store_impl(p.out, p.n, p.rows, sm_out, lane, row, colbase);
     }
 };
 
@@ -769,6 +786,9 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
     bool loading = true;  // the producer still has a row group
     long long issued = 0, consumed = 0;
     auto issue_chunk = [&]() {
+        HS_DBG_CHECK(!TMA || ((long long)pgroup * R < p.rows && (long long)pchunk * lm.W < p.n &&
+                              ((pchunk * lm.W * (int)sizeof(TIn)) & 15) == 0 && pstage < S),
+                     kDbgTmaCoord, ((unsigned long long)pgroup << 32) | (unsigned)pchunk, return);
         if (TMA) pipe.issue(&tm_a, &tm_b, pgroup * R, pchunk * lm.W, pstage);
         else if (wide) CE::wide_load_async(p, pipe.in_a(pstage), pipe.in_b(pstage), lane, pgroup, (long long)pchunk * lm.W, lm.W);
         else CE::generic_load_async(p, pipe.in_a(pstage), pipe.in_b(pstage), lm, lane, (long long)pgroup * R, pchunk * lm.W);
@@ -846,6 +866,8 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
         state = compose(state, total);
         renormalise(state);
 
+        HS_DBG_CHECK(!TMA || ((long long)group * R < p.rows && colbase < p.n && ((colbase * (int)sizeof(TOut)) & 15) == 0),
+                     kDbgTmaCoord, ((unsigned long long)group << 32) | (unsigned)colbase, break);
         if (TMA) {
             pipe.store_from(&tm_o, group * R, colbase, sm_out);
             if (chunk == tail_chunk_out) CE::tail_store(p, sm_out, lane, row, colbase);
@@ -982,6 +1004,7 @@ struct Lookback {
         return e;
     }
     __device__ static __forceinline__ void publish_agg(const Params& p, long long T, const E& e) {
+        HS_DBG_CHECK(T >= 0 && T < p.num_tiles, kDbgTile, T, return);
         st_desc(p.desc + T, pack(e, kAgg));
     }
 
@@ -1036,10 +1059,12 @@ struct Lookback {
 #pragma unroll
                 for (int q = 0; q < kLbPerLane; ++q) {
                     const int dist = kLbPerLane * lane + q + 1;
+                    HS_DBG_CHECK(dist > k || (T - dist >= 0 && T - dist < p.num_tiles), kDbgTile, T - dist, continue);
                     if (dist <= k) td[q] = ld_desc(p.desc + (T - dist));
                 }
             }
             const int gg = g - gwin - lane;
+            HS_DBG_CHECK(groups_done || gg < 0 || gbase + gg < p.rows * p.groups_per_row, kDbgTile, gbase + gg, groups_done = true);
             if (!groups_done && gg >= 0) gd = ld_desc(p.gdesc + gbase + gg);
             ++total_polls;
 
@@ -1067,7 +1092,8 @@ struct Lookback {
             }
             if (own_ready && tiles_done && full_group && publish && !group_agg_sent) {
                 // later groups need only this, not our own carry: publish it at once
-                if (lane == 0) st_desc(p.gdesc + gbase + g, pack(compose(before_in_group, tile_total), kAgg));
+                HS_DBG_CHECK(gbase + g < p.rows * p.groups_per_row, kDbgTile, gbase + g, group_agg_sent = true);
+                if (lane == 0 && !group_agg_sent) st_desc(p.gdesc + gbase + g, pack(compose(before_in_group, tile_total), kAgg));
                 group_agg_sent = true;
             }
             if (!groups_done) {
@@ -1312,6 +1338,9 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
         if (issued < my_tiles) {
             const int cb = colbase_of(ci);
             const uint32_t bar = bars + 8 * istage;
+            // (a chunk of the row's last tile may lie wholly beyond the row: TMA fills it with zeros, the plain path skips it)
+            HS_DBG_CHECK(ci.row >= 0 && ci.row < p.rows && ((cb * (int)sizeof(TIn)) & 15) == 0 && istage < S, kDbgTmaCoord,
+                         ((unsigned long long)ci.row << 32) | (unsigned)cb, return);
             if (!TMA) {
                 CE::wide_load_async(p, st_a(istage), st_b(istage), lane, ci.row, cb, CHUNK);
             } else if (flat) {

@@ -15,7 +15,8 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libheinsen_scan.so")
+# HEINSEN_SCAN_LIBRARY selects another build of the same library (the checked build, libheinsen_scan_debug.so)
+LIB_PATH = os.environ.get("HEINSEN_SCAN_LIBRARY") or os.path.join(_HERE, "libheinsen_scan.so")
 
 HS_F32, HS_BF16 = 0, 1
 HS_OK = 0
@@ -26,6 +27,7 @@ EXPORTS = [
     "heinsen_scan_linear_host", "heinsen_scan_log_host", "heinsen_scan_host_scratch_bytes",
     "heinsen_scan_set_path", "heinsen_scan_tune", "heinsen_scan_debug_config", "heinsen_scan_last_path",
     "heinsen_scan_launch_count", "heinsen_scan_strerror", "heinsen_scan_probe_mufu",
+    "heinsen_scan_debug_build", "heinsen_scan_debug_faults", "heinsen_scan_debug_window_ok",
     "heinsen_scan_log_static", "heinsen_scan_check_static", "heinsen_scan_static_max_elements",
     "heinsen_scan_log_complex", "heinsen_scan_complex_workspace_bytes",
     "heinsen_scan_linear_pairs",
@@ -72,6 +74,12 @@ def lib() -> ctypes.CDLL:
         L.heinsen_scan_set_path.restype = ci
         L.heinsen_scan_tune.argtypes = [ctypes.c_char_p, ci]
         L.heinsen_scan_tune.restype = ci
+        u64 = ctypes.c_uint64
+        L.heinsen_scan_debug_build.restype = ci
+        L.heinsen_scan_debug_faults.argtypes = [ctypes.POINTER(u64)]
+        L.heinsen_scan_debug_faults.restype = ci
+        L.heinsen_scan_debug_window_ok.argtypes = [u64, u64, u64, u64, u64]
+        L.heinsen_scan_debug_window_ok.restype = ci
         L.heinsen_scan_probe_mufu.argtypes = [ci, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
         L.heinsen_scan_probe_mufu.restype = ci
         L.heinsen_scan_debug_config.argtypes = [ctypes.c_uint32, i64]
@@ -168,6 +176,20 @@ def set_path(path: int):
 def tune(name: str, value: int = -1):
     """Set a tuning knob (see heinsen_scan_tune in the header); value < 0 restores its default."""
     _check(lib().heinsen_scan_tune(name.encode(), int(value)))
+
+
+def debug_build() -> bool:
+    """True when the loaded library is the checked build (-DHEINSEN_DEBUG)."""
+    return bool(lib().heinsen_scan_debug_build())
+
+
+def debug_faults():
+    """The first failed check of the checked build since the last call, as (code, detail, block, thread), or None."""
+    out = (ctypes.c_uint64 * 4)()
+    rc = lib().heinsen_scan_debug_faults(out)
+    if rc < 0:
+        raise HeinsenScanError(4, "heinsen_scan_debug_faults: CUDA error")
+    return tuple(int(v) for v in out) if rc else None
 
 
 def probe_mufu(iterations: int = 4096):

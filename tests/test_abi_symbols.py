@@ -88,3 +88,20 @@ def test_without_a_gpu_the_product_path_fails_loudly(lib):
     from paper_2311_06281_b200 import heinsen_scan
     with pytest.raises(ValueError):
         heinsen_scan.scan_log(torch.zeros(2, 8), torch.zeros(2, 8), torch.zeros(2))
+
+
+def test_window_predicate_of_the_checked_build(lib):
+    """The predicate the checked build (-DHEINSEN_DEBUG) applies to every shared-memory access: the access must lie
+    inside [base, base + size) and be aligned to its width.  It is plain arithmetic, exported by both builds."""
+    ok = lib.heinsen_scan_debug_window_ok
+    base, size = 0x1000, 0x400
+    assert ok(base, 16, base, size, 16) == 1 and ok(base + size - 16, 16, base, size, 16) == 1
+    assert ok(base + size - 12, 16, base, size, 4) == 0            # runs over the end
+    assert ok(base + size, 4, base, size, 4) == 0                  # starts at the end
+    assert ok(base - 16, 16, base, size, 16) == 0                  # before the window
+    assert ok(base + 4, 16, base, size, 16) == 0                   # misaligned for its width
+    assert ok(base + 4, 4, base, size, 4) == 1
+    assert ok(base, size + 1, base, size, 1) == 0 and ok(base, size, base, size, 1) == 1
+    assert ok(base, 4, base, size, 0) == 0                         # no alignment given: refused, not divided by
+    assert ok(2**64 - 8, 16, base, size, 8) == 0                   # no wrap-around
+    assert lib.heinsen_scan_debug_build() == 0 and lib.heinsen_scan_debug_faults(None) == 0
