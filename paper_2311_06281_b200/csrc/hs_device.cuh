@@ -45,6 +45,17 @@ __device__ __forceinline__ float rcp_approx(float x) {
     return y;
 }
 __device__ __forceinline__ float flip(float v, uint32_t mask) { return __uint_as_float(__float_as_uint(v) ^ mask); }
+// three-input maximum / minimum: one instruction on sm_100
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float min3(float a, float b, float c) {
+    float d;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 
 // Natural logarithm of |v| accurate to about one ulp also for v close to 1, where lg2.approx's
 // absolute error would be a large relative error of log a_t and would bias a*_t over a long
@@ -72,26 +83,6 @@ __device__ __forceinline__ float log_abs_accurate(float v) {
     return zero ? neg_inf() : fmaf((float)e + bias, kLn2, lm);
 }
 
-// log|v| for the hot path of the linear entry point, about half the cost of log_abs_accurate:
-// near 1 (|v| in (0.875, 1.125)) the Taylor series of log(1+f) in f = |v| - 1 (exact in fp32),
-// relative error <= 1.3e-7; elsewhere lg2.approx, whose absolute error of 2^-22 is there a relative
-// error <= 1.4e-6 of log|v| (inside the 2e-6 |a*_t| term of the tolerance even if it never cancelled).
-// |v| = 0 and denormals give -inf.
-__device__ __forceinline__ float log_abs_fast(float v) {
-    const float av = fabsf(v);
-    const float f = av - 1.0f;
-    float p = fmaf(f, -1.0f / 8.0f, 1.0f / 7.0f);
-    p = fmaf(p, f, -1.0f / 6.0f);
-    p = fmaf(p, f, 1.0f / 5.0f);
-    p = fmaf(p, f, -1.0f / 4.0f);
-    p = fmaf(p, f, 1.0f / 3.0f);
-    p = fmaf(p, f, -0.5f);
-    p = fmaf(p, f, 1.0f);
-    const float near_one = p * f;
-    const float far = lg2(av) * kLn2;
-    return (fabsf(f) < 0.125f) ? near_one : far;
-}
-
 // Packed fp32 pairs (sm_100's f32x2 arithmetic): one instruction, hence one issue slot, for two
 // elements.  The kernels are short of issue slots before they are short of anything else, so all
 // element-wise arithmetic of a lane's run is written on pairs of neighbouring elements.
@@ -101,20 +92,33 @@ __device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) { return __
 __device__ __forceinline__ float2 mul2(float2 a, float2 b) { return __fmul2_rn(a, b); }
 __device__ __forceinline__ float2 add2(float2 a, float2 b) { return __fadd2_rn(a, b); }
 
-// log_abs_fast on two values at once.
-__device__ __forceinline__ float2 log_abs_fast2(float2 v) {
+// log2|v| for the hot path of the linear entry point, about half the cost of log_abs_accurate, in binary
+// logarithms because that is what ex2 / lg2 work in (the linear entry point keeps the A_t of a run in these
+// units): near 1 (|v| in (0.875, 1.125)) the Taylor series of log(1+f) in f = |v| - 1 (exact in fp32) to the
+// sixth power, its coefficients carrying the factor log2(e), relative error <= |f|^6 / 7 <= 5.5e-7; elsewhere
+// lg2.approx, whose absolute error of 2^-22 is there a relative error <= 1.4e-6 of the logarithm (inside the
+// 2e-6 |a*_t| term of the tolerance even if it never cancelled).  |v| = 0 and denormals give -inf.
+__device__ __forceinline__ float log2_abs_fast(float v) {
+    const float av = fabsf(v);
+    const float f = av - 1.0f;
+    float p = fmaf(f, -kLog2e / 6.0f, kLog2e / 5.0f);
+    p = fmaf(p, f, -kLog2e / 4.0f);
+    p = fmaf(p, f, kLog2e / 3.0f);
+    p = fmaf(p, f, -kLog2e / 2.0f);
+    p = fmaf(p, f, kLog2e);
+    return (fabsf(f) < 0.125f) ? p * f : lg2(av);
+}
+// ... on two values at once.
+__device__ __forceinline__ float2 log2_abs_fast2(float2 v) {
     const float2 av = pk(fabsf(v.x), fabsf(v.y));
     const float2 f = add2(av, pk(-1.0f));
-    float2 p = fma2(f, pk(-1.0f / 8.0f), pk(1.0f / 7.0f));
-    p = fma2(p, f, pk(-1.0f / 6.0f));
-    p = fma2(p, f, pk(1.0f / 5.0f));
-    p = fma2(p, f, pk(-1.0f / 4.0f));
-    p = fma2(p, f, pk(1.0f / 3.0f));
-    p = fma2(p, f, pk(-0.5f));
-    p = fma2(p, f, pk(1.0f));
+    float2 p = fma2(f, pk(-kLog2e / 6.0f), pk(kLog2e / 5.0f));
+    p = fma2(p, f, pk(-kLog2e / 4.0f));
+    p = fma2(p, f, pk(kLog2e / 3.0f));
+    p = fma2(p, f, pk(-kLog2e / 2.0f));
+    p = fma2(p, f, pk(kLog2e));
     const float2 near_one = mul2(p, f);
-    const float2 far = mul2(pk(lg2(av.x), lg2(av.y)), pk(kLn2));
-    return pk((fabsf(f.x) < 0.125f) ? near_one.x : far.x, (fabsf(f.y) < 0.125f) ? near_one.y : far.y);
+    return pk((fabsf(f.x) < 0.125f) ? near_one.x : lg2(av.x), (fabsf(f.y) < 0.125f) ? near_one.y : lg2(av.y));
 }
 
 // ------------------------------------------------------------------------------------------
@@ -222,12 +226,14 @@ __device__ __forceinline__ Elem<SIGNED> state_elem(float log_mag, uint32_t sign_
     return e;
 }
 
-// Keep |s| in [1,2) so that a long signed cancellation cannot strand the reference far above
-// the value.  Exact apart from one rounding of m.
+// Bring |s| back into [1,2) once it has drifted 20 binary orders away, so that a long signed cancellation
+// cannot strand the reference far above the value (and s, in the end, below fp32's range).  Exact apart from
+// one rounding of m.
 template <bool SIGNED>
 __device__ __forceinline__ void renormalise(Elem<SIGNED>& e) {
     if (!SIGNED) return;
     const float as = fabsf(e.s);
+    if (as >= 9.5367431640625e-07f /* 2^-20 */ && as <= 1048576.0f /* 2^20 */) return;  // nowhere near fp32's limits
     if (as == 0.0f) { e.m = kEmpty; e.s = 0.0f; return; }
     if (as >= 1.17549435e-38f) {
         const int ex = ((__float_as_int(as) >> 23) & 0xff) - 127;
@@ -715,9 +721,10 @@ struct Run {
     static constexpr int IN_BYTES = CHUNK * (int)sizeof(TIn);
     static constexpr int OUT_BYTES = CHUNK * (int)sizeof(TOut);
 
-    float A[K];     // A_t
+    float A[K];     // A_t (kLinear: in binary logarithms, log2 of the product of |a|)
     float s[K];     // s_t (before that: u_t)
-    uint32_t P[K];  // parity mask of a_1..a_t (SIGNED only)
+    uint32_t P[K];  // parity mask of a_1..a_t (log modes with signs)
+    float Pf[K];    // kLinear: the same parity as a factor, +1.0f or -1.0f (applied by a packed multiply)
     float r;        // reference of the run, -inf when the run has no non-zero b
     bool bad;       // the fast form does not apply to this run (a_t = 0, inf or NaN in it)
 
@@ -764,23 +771,24 @@ struct Run {
             // The reference of the run is taken from the largest |b_t| and the smallest A_t: it bounds
             // every u_t = log|b_t| - A_t from above, which is all a log-sum-exp reference has to do, and it
             // costs one logarithm per run instead of one per element; b_t itself enters the sum linearly.
-            float bmax = 0.0f, amin = 0.0f;
+            float bmax = 0.0f, amin = 0.0f, sgf = 1.0f;
 #pragma unroll
             for (int t = 0; t < K; t += 2) {
-                const float2 la = log_abs_fast2(pk(va[t], va[t + 1]));
-                par ^= __float_as_uint(va[t]) & kSignBit;
-                P[t] = par;
-                par ^= __float_as_uint(va[t + 1]) & kSignBit;
-                P[t + 1] = par;
+                const float2 la = log2_abs_fast2(pk(va[t], va[t + 1]));  // A_t of this mode: binary logarithms
+                sgf = flip(sgf, __float_as_uint(va[t]) & kSignBit);
+                Pf[t] = sgf;
+                sgf = flip(sgf, __float_as_uint(va[t + 1]) & kSignBit);
+                Pf[t + 1] = sgf;
                 acc += la.x;
                 A[t] = acc;
                 acc += la.y;
                 A[t + 1] = acc;
-                bmax = fmaxf(bmax, fmaxf(fabsf(vb[t]), fabsf(vb[t + 1])));
-                amin = fminf(amin, fminf(A[t], A[t + 1]));
+                bmax = max3(bmax, fabsf(vb[t]), fabsf(vb[t + 1]));
+                amin = min3(amin, A[t], A[t + 1]);
             }
+            par = __float_as_uint(sgf) & kSignBit;
             // (2^-126 <= bmax keeps the scale factor below 2^127; smaller b_t are zero to ex2/lg2.approx.ftz anyway)
-            rr = (bmax >= 1.17549435e-38f) ? fmaf(lg2(bmax), kLn2, -amin) : neg_inf();
+            rr = (bmax >= 1.17549435e-38f) ? (lg2(bmax) - amin) * kLn2 : neg_inf();
             bad = !(acc >= -1e30f) || !(bmax <= 3.0e38f) || !(amin >= -1e30f);
         } else {
 #pragma unroll
@@ -798,7 +806,7 @@ struct Run {
                 const float2 u = fma2(pk(A[t], A[t + 1]), pk(-1.0f), pk(vb[t], vb[t + 1]));
                 s[t] = u.x;
                 s[t + 1] = u.y;
-                rr = fmaxf(rr, fmaxf(u.x, u.y));
+                rr = max3(rr, u.x, u.y);
             }
             bad = !(acc >= -1e30f) || !(rr <= 1e30f);
         }
@@ -810,9 +818,8 @@ struct Run {
         for (int t = 0; t < K; t += 2) {
             float2 e;
             if (MODE == kLinear) {
-                const float2 arg = fma2(pk(A[t], A[t + 1]), pk(-kLog2e), c);  // <= 126: A_t >= amin, bmax >= 2^-126
-                e = mul2(pk(vb[t], vb[t + 1]), pk(ex2(arg.x), ex2(arg.y)));
-                e = pk(flip(e.x, P[t]), flip(e.y, P[t + 1]));
+                const float2 arg = fma2(pk(A[t], A[t + 1]), pk(-1.0f), c);  // <= 126: A_t >= amin, bmax >= 2^-126
+                e = mul2(mul2(pk(vb[t], vb[t + 1]), pk(ex2(arg.x), ex2(arg.y))), pk(Pf[t], Pf[t + 1]));
             } else {
                 const float2 arg = fma2(pk(s[t], s[t + 1]), pk(kLog2e), c);
                 e = pk(ex2(arg.x), ex2(arg.y));
@@ -823,6 +830,7 @@ struct Run {
             sum += e.y;
             s[t + 1] = sum;
         }
+        if (MODE == kLinear) acc *= kLn2;  // parts are composed in natural logarithms
         E agg;
         agg.A = acc;
         agg.m = fmaxf(rr + acc, kEmpty);
@@ -839,14 +847,15 @@ struct Run {
 #pragma unroll
         for (int t = 0; t < K; ++t) {
             if (MODE == kLinear) {
-                acc += log_abs_fast(va[t]);
+                acc += log2_abs_fast(va[t]);
                 par ^= __float_as_uint(va[t]) & kSignBit;
             } else {
                 acc += va[t];
                 if (MODE == kLogSigned) par ^= sa[t];
             }
             A[t] = acc;
-            if (SIGNED) P[t] = par;
+            if (MODE == kLinear) Pf[t] = __uint_as_float(0x3f800000u | par);
+            else if (SIGNED) P[t] = par;
         }
         bad = false;
     }
@@ -857,14 +866,16 @@ struct Run {
     __device__ __forceinline__ uint32_t parity_bits() const {
         uint32_t bits = 0u;
 #pragma unroll
-        for (int t = 0; t < K; ++t) bits = (bits >> 1) | (SIGNED ? P[t] : 0u);
+        for (int t = 0; t < K; ++t)
+            bits = (bits >> 1) | (MODE == kLinear ? (__float_as_uint(Pf[t]) & kSignBit) : SIGNED ? P[t] : 0u);
         return bits;
     }
     __device__ __forceinline__ void adopt(const float* a_parked, uint32_t bits) {
 #pragma unroll
         for (int t = 0; t < K; ++t) {
             A[t] = a_parked[t];
-            if (SIGNED) P[t] = (bits << (K - 1 - t)) & kSignBit;
+            if (MODE == kLinear) Pf[t] = __uint_as_float(0x3f800000u | ((bits << (K - 1 - t)) & kSignBit));
+            else if (SIGNED) P[t] = (bits << (K - 1 - t)) & kSignBit;
         }
         bad = false;
     }
@@ -902,11 +913,11 @@ struct Run {
             const float2 S = fma2(pk(s[t], s[t + 1]), w2, C2);
             if (MODE == kLinear) {
                 // exp(A_t + M) as the square of exp((A_t + M) / 2): the exponent range of fp32 twice over
-                const float2 arg = fma2(pk(A[t], A[t + 1]), pk(0.5f * kLog2e), pk(a.M * (0.5f * kLog2e)));
+                const float2 arg = fma2(pk(A[t], A[t + 1]), pk(0.5f), pk(a.M * (0.5f * kLog2e)));  // (A_t: binary logarithms)
                 const float2 h = pk(ex2(arg.x), ex2(arg.y));
-                const float2 x = mul2(mul2(S, h), h);
-                out_mag[i] = flip(x.x, P[t]);
-                out_mag[i + 1] = flip(x.y, P[t + 1]);
+                const float2 x = mul2(mul2(mul2(S, h), h), pk(Pf[t], Pf[t + 1]));
+                out_mag[i] = x.x;
+                out_mag[i + 1] = x.y;
             } else {
                 const float2 o = fma2(pk(lg2(fabsf(S.x)), lg2(fabsf(S.y))), pk(kLn2), add2(pk(A[t], A[t + 1]), pk(a.M)));
                 out_mag[i] = o.x;
