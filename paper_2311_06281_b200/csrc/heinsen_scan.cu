@@ -517,7 +517,20 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         if (p.tiles_per_row == 1) {
             // every row is a single tile: no tile waits for another, so neither the descriptors nor the
             // co-residency guarantee of a cooperative launch are needed
-            e = cudaLaunchKernel(fn, dim3(grid), dim3(warps * 32), args, smem, stream);
+            // (programmatic stream serialisation: back-to-back small calls overlap their set-up with the previous
+            // kernel's tail; the kernel waits before its first access to global memory)
+            cudaLaunchConfig_t cfg;
+            std::memset(&cfg, 0, sizeof cfg);
+            cfg.gridDim = dim3(grid);
+            cfg.blockDim = dim3(warps * 32);
+            cfg.dynamicSmemBytes = (size_t)smem;
+            cfg.stream = stream;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[0].val.programmaticStreamSerializationAllowed = knob(kKnobNoPdl, 0, 0, 1) ? 0 : 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            e = cudaLaunchKernelExC(&cfg, fn, args);
         } else {
             // every descriptor starts as "nothing yet"
             e = cudaMemsetAsync(p.desc, 0, ((size_t)p.num_tiles + (size_t)p.rows * p.groups_per_row) * 16, stream);

@@ -1226,8 +1226,13 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
         }
         for (int i = 0; i < W * kLbMaxStages; ++i) mbar_init(warp_bars + 8 * i, 1);
         fence_mbar_init();
-        if (blockIdx.x == 0) p.ws->started_id = p.call_id;
     }
+    // Programmatic dependent launch, as in the batched kernel: when the host launches the single-tile form with
+    // programmatic stream serialisation, everything above overlaps the end of the previous kernel of the stream
+    // and global memory is touched only from here on; for the cooperative launch both are no-ops.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (threadIdx.x == 0 && blockIdx.x == 0) p.ws->started_id = p.call_id;
     __syncthreads();
 
     const long long G = gridDim.x;
