@@ -105,3 +105,17 @@ def test_window_predicate_of_the_checked_build(lib):
     assert ok(base, 4, base, size, 0) == 0                         # no alignment given: refused, not divided by
     assert ok(2**64 - 8, 16, base, size, 8) == 0                   # no wrap-around
     assert lib.heinsen_scan_debug_build() == 0 and lib.heinsen_scan_debug_faults(None) == 0
+
+
+def test_tuning_and_probe_arguments_are_checked_on_the_host(lib):
+    """heinsen_scan_tune knows its knobs by name (no environment look-up per call) and refuses others; the roofline
+    probe refuses bad arguments before it touches CUDA."""
+    import ctypes
+    assert lib.heinsen_scan_tune(b"WARPS", 12) == 0 and lib.heinsen_scan_tune(b"WARPS", -1) == 0
+    for name in (b"ROWS_PER_WARP", b"STAGES", b"ROW_TICKETS", b"NO_TMA", b"NO_FLAT", b"NO_PDL", b"LB_STAGES", b"LB_WARPS",
+                 b"LB_GROUP", b"LB_SLEEP_IDLE", b"LB_SLEEP_READY", b"LB_CTAS_PER_SM"):
+        assert lib.heinsen_scan_tune(name, -1) == 0, name
+    assert lib.heinsen_scan_tune(b"NO_SUCH_KNOB", 1) == 1 and lib.heinsen_scan_tune(None, 1) == 1
+    r, s = ctypes.c_double(0), ctypes.c_double(0)
+    assert lib.heinsen_scan_probe_mufu(0, ctypes.byref(r), ctypes.byref(s)) == 1
+    assert lib.heinsen_scan_probe_mufu(16, None, ctypes.byref(s)) == 1
