@@ -135,7 +135,8 @@ hs_status heinsen_scan_log(const void* log_a, const void* log_b, const void* log
 /*
  * Scratch size in bytes for a problem of this shape (any path, any type): a 256-byte
  * header (status words) plus 16 bytes per tile and per group of tiles of the look-back
- * kernel -- the carry between parts that the associativity of prefix sums allows
+ * kernel, or per warp slot of the batched kernel when it shares rows out among its
+ * slots -- the carry between parts that the associativity of prefix sums allows
  * (Summary, footnote on associativity).  Returns 0 only for invalid sizes.
  */
 size_t heinsen_scan_workspace_bytes(int64_t rows, int64_t n);
@@ -265,7 +266,7 @@ int heinsen_scan_debug_window_ok(uint64_t addr, uint64_t bytes, uint64_t base, u
 /*
  * Tuning knobs, for sweeps and for tests that force a variant; every knob has a measured default
  * that is chosen per call.  `name` is one of "NO_TMA", "ROWS_PER_WARP", "WARPS", "STAGES",
- * "ROW_TICKETS", "NO_FLAT", "NO_PDL" (row-batched kernel), "LB_STAGES", "LB_WARPS", "LB_GROUP",
+ * "ROW_TICKETS", "SPANS", "NO_FLAT", "NO_PDL" (row-batched kernel), "LB_STAGES", "LB_WARPS", "LB_GROUP",
  * "LB_SLEEP_IDLE", "LB_SLEEP_READY", "LB_CTAS_PER_SM" (look-back kernel); value >= 0 sets the knob
  * (clamped to its range), value < 0 returns it to its default.  The environment variables
  * HEINSEN_SCAN_<name> give the initial values; they are read once per process, not per call.

@@ -32,6 +32,7 @@ constexpr int kBatchedMinRowsPerSm = 8;  // fewer rows per SM than this: look-ba
 constexpr int kBatchedMinWarpsPerSm = 12; // rows per warp are chosen to keep at least this many warps per SM
 constexpr int kLookbackMinWarps = 8;     // fewest compute warps (= chunks per tile) of the look-back kernel
 constexpr int kLookbackWarps = 14;       // default compute warps of the look-back kernel
+constexpr size_t kMaxWarpSlots = 16 * 256;  // warp slots of the batched kernel, at most
 constexpr int kMinChunk = 512;           // smallest chunk of the real storage types (32 lanes x 16 elements)
 constexpr int kComplexChunk = 256;       // chunk of the complex-logarithm storage type (32 lanes x 8 elements)
 constexpr hs_dtype kC64 = static_cast<hs_dtype>(2);  // internal: complex64 elements (heinsen_scan_log_complex)
@@ -177,11 +178,11 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 // heinsen_scan_tune() changes a knob, so that a launch costs no getenv().
 enum Knob : int {
     kKnobNoTma = 0, kKnobRowsPerWarp, kKnobWarps, kKnobRowTickets, kKnobNoFlat, kKnobNoPdl, kKnobLbStages,
-    kKnobLbWarps, kKnobLbGroup, kKnobLbSleepIdle, kKnobLbSleepReady, kKnobLbCtasPerSm, kKnobStages, kKnobCount
+    kKnobLbWarps, kKnobLbGroup, kKnobLbSleepIdle, kKnobLbSleepReady, kKnobLbCtasPerSm, kKnobStages, kKnobSpans, kKnobCount
 };
 const char* const kKnobNames[kKnobCount] = {
     "NO_TMA", "ROWS_PER_WARP", "WARPS", "ROW_TICKETS", "NO_FLAT", "NO_PDL", "LB_STAGES",
-    "LB_WARPS", "LB_GROUP", "LB_SLEEP_IDLE", "LB_SLEEP_READY", "LB_CTAS_PER_SM", "STAGES"};
+    "LB_WARPS", "LB_GROUP", "LB_SLEEP_IDLE", "LB_SLEEP_READY", "LB_CTAS_PER_SM", "STAGES", "SPANS"};
 constexpr int kKnobUnset = INT_MIN;
 std::atomic<int> g_knobs[kKnobCount];
 std::once_flag g_knobs_once;
@@ -214,6 +215,7 @@ struct Problem {
 struct KernelEntry {
     const void* batched;      // row groups stay with their warp slots
     const void* batched_tk;   // row groups handed out by tickets
+    const void* batched_span; // one row per warp, the rows' chunks shared out evenly among the warp slots (or null)
     const void* lookback;
     int K;
     int warp_smem_per_stage;  // bytes of one input stage (both tensors) of one warp
@@ -228,6 +230,7 @@ KernelEntry entry() {
     constexpr int LBK = sizeof(TIn) == 8 ? 8 : 16;  // the look-back kernel parks fp32 partial sums: 16 per lane (8 for complex elements)
     e.batched = reinterpret_cast<const void*>(&batched_scan_kernel<MODE, TIn, TOut, K, TMA, false>);
     e.batched_tk = reinterpret_cast<const void*>(&batched_scan_kernel<MODE, TIn, TOut, K, TMA, true>);
+    e.batched_span = reinterpret_cast<const void*>(&batched_span_kernel<MODE, TIn, TOut, K, TMA>);
     e.lookback = reinterpret_cast<const void*>(&lookback_scan_kernel<MODE, TIn, TOut, LBK, TMA>);
     e.lb_K = LBK;
     e.K = K;
@@ -244,6 +247,7 @@ KernelEntry entry_batched_only() {
     KernelEntry e;
     e.batched = reinterpret_cast<const void*>(&batched_scan_kernel<MODE, TIn, TOut, K, TMA, false>);
     e.batched_tk = reinterpret_cast<const void*>(&batched_scan_kernel<MODE, TIn, TOut, K, TMA, true>);
+    e.batched_span = nullptr;
     e.lookback = nullptr;
     e.lb_K = K;
     e.K = K;
@@ -305,7 +309,11 @@ size_t workspace_bytes_for(long long rows, long long n, int min_chunk = kMinChun
     // sized for the smallest chunk so that it covers every type
     const long long tpr = lookback_tiles_per_row(n, min_chunk, kLookbackMinWarps);
     const long long gpr = (tpr + 1) / 2;  // groups hold at least 2 tiles
-    return sizeof(Header) + (size_t)(rows * (tpr + gpr)) * 16;
+    size_t words = (size_t)(rows * (tpr + gpr));
+    // ... or, for the batched kernel that shares the rows' chunks out among its warp slots, one word per slot
+    // (at most 16 warps on each of at most 256 SMs; only shapes with at least one row per slot use it)
+    if (rows >= 128 && words < kMaxWarpSlots) words = kMaxWarpSlots;
+    return sizeof(Header) + words * 16;
 }
 
 // cudaFuncSetAttribute and the occupancy query cost microseconds per call; remember what was set.
@@ -442,6 +450,25 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         int tickets = (groups >= 4ll * grid * warps && p.nchunks >= 4) ? 1 : 0;
         tickets = knob(kKnobRowTickets, tickets, 0, 1);
         fn = tickets ? ke.batched_tk : ke.batched;
+        // Between one and a few rows per warp slot, whole rows per slot leave the last round of slots partly idle:
+        // share the rows' chunks out evenly instead (one row per warp, rows of at least two chunks, at least one row
+        // per slot so that every share begins or ends inside a row at most once; the hand-over words need 16 bytes
+        // per slot behind the workspace header).
+        const long long slots = (long long)grid * warps;
+        const long long rounds = (groups + slots - 1) / slots;
+        // (worth it when whole rows per slot would keep the slots busy less than four fifths of the time; closer to
+        // full rounds than that, the plain assignment is as fast while HBM is the limit and its loop is a little shorter)
+        int spans = (!tickets && R == 1 && ke.batched_span && p.nchunks >= 2 && groups >= slots && stages == 2 &&
+                     groups * 5 <= rounds * slots * 4 && workspace_bytes >= sizeof(Header) + (size_t)slots * 16)
+                        ? 1 : 0;
+        spans = knob(kKnobSpans, spans, 0, 1);
+        if (spans && !(R == 1 && ke.batched_span && groups >= slots && !tickets && stages == 2 &&
+                       workspace_bytes >= sizeof(Header) + (size_t)slots * 16))
+            spans = 0;  // (the knob cannot force it onto shapes it does not cover)
+        if (spans) {
+            fn = ke.batched_span;
+            p.desc = reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(workspace) + sizeof(Header));
+        }
     } else {
         p.rows_per_warp = 1;
         // S input stages per compute warp (phase 2 of a tile runs S-2 iterations after its phase 1),

@@ -908,6 +908,202 @@ batched_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
 }
 
 // ------------------------------------------------------------------------------------------
+// (a') Row-batched kernel with the rows cut to measure: for a number of rows between one and a few per warp slot,
+// whole rows per slot leave the last round of slots partly idle (4096 rows on 2368 slots: 1.73 rounds, which costs
+// nothing while the kernel is bound by HBM and 13 % once it is bound by the SM clock under the board's power cap).
+// Here the rows' chunks form one sequence, (row 0, chunk 0), (row 0, chunk 1), ..., and every slot takes an equal
+// share of it.  With at least one row per slot a share is
+//     [the rest of a row that the slot before began] [whole rows] [the beginning of a row that the next slot ends],
+// and the slot walks it in the order beginning - whole rows - rest: the beginning of a row needs nothing but x_0,
+// and the value of x after it goes to the next slot through a 16-byte word in the workspace, {m, s, call id},
+// long before that slot, which walks its own beginning and whole rows first, asks for it (bounded wait).
+// One row per warp, any staging (TMA boxes or whole 16-byte units); the arithmetic is the batched kernel's.
+template <int MODE, typename TIn, typename TOut, int K, bool TMA>
+__global__ void __launch_bounds__(512, 1)
+batched_span_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+                    const __grid_constant__ CUtensorMap tm_o) {
+    using CE = ChunkEngine<MODE, TIn, TOut, K>;
+    using E = typename CE::E;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = align_1024(smem_raw);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    constexpr bool PLAIN = !TMA;
+    constexpr int PAD = PLAIN ? CE::WIDE_PAD : 0;
+    constexpr int S = 2;  // input stages per warp: one chunk being worked on, one in flight
+    const int per_warp = warp_smem_bytes<MODE, TIn, TOut, K>(S, PAD);
+
+    LaneMap lm;
+    lm.R = 1; lm.g = 0; lm.i = lane; lm.W = 32 * K;
+    const typename CE::Offsets off = CE::offsets(lm);
+    using Pipe = WarpPipe<TIn, TOut, K, PAD>;
+    Pipe pipe;
+    pipe.base = smem_u32(smem) + warp * per_warp;
+    pipe.bars = smem_u32(smem + nwarps * per_warp) + warp * (8 * kMaxStages);
+    pipe.stages = S;
+    pipe.lane = lane;
+    pipe.setup(1, p.flat_boxes != 0);
+    if (TMA) pipe.init();
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (threadIdx.x == 0 && blockIdx.x == 0) p.ws->started_id = p.call_id;
+
+    // the slot's share of the chunk sequence (slots numbered CTA-fastest, as in the batched kernel)
+    const int GW = gridDim.x * nwarps;
+    const int gw = warp * (int)gridDim.x + (int)blockIdx.x;
+    const int nchunks = p.nchunks;
+    const long long total = p.rows * (long long)nchunks;
+    const long long q0 = total / GW, rem = total % GW;
+    const long long lo = gw * q0 + (gw < rem ? gw : rem), hi = lo + q0 + (gw < rem ? 1 : 0);
+    const int len = (int)(hi - lo);  // (the host sends shapes with at least one row per slot: q0 >= nchunks)
+    if (len <= 0) return;
+    const int row_lo = (int)(lo / nchunks), c_lo = (int)(lo % nchunks);
+    const int row_hi = (int)(hi / nchunks), c_hi = (int)(hi % nchunks);
+    const int n_head = c_hi;                         // chunks [0, c_hi) of row_hi, walked first
+    const int n_rest = c_lo ? nchunks - c_lo : 0;    // chunks [c_lo, nchunks) of row_lo, walked last
+    const int first_whole = row_lo + (c_lo ? 1 : 0);
+    // position q of the walk -> (row, chunk)
+    struct Cursor {
+        int q, row, chunk;
+    };
+    auto start = [&]() {
+        Cursor c;
+        c.q = 0;
+        if (n_head) { c.row = row_hi; c.chunk = 0; }
+        else if (len > n_rest) { c.row = first_whole; c.chunk = 0; }
+        else { c.row = row_lo; c.chunk = c_lo; }
+        return c;
+    };
+    auto advance = [&](Cursor& c) {
+        ++c.q;
+        ++c.chunk;
+        if (c.q == n_head) {                       // the beginning is done: on to the whole rows, or to the rest
+            if (len - n_rest > n_head) { c.row = first_whole; c.chunk = 0; }
+            else { c.row = row_lo; c.chunk = c_lo; }
+        } else if (c.q == len - n_rest) {          // the whole rows are done: the rest of the first row
+            c.row = row_lo; c.chunk = c_lo;
+        } else if (c.chunk == nchunks) {
+            c.chunk = 0; ++c.row;
+        }
+    };
+    const bool tail_ragged = (p.n % lm.W) != 0;
+    const int tail_chunk_in = (pipe.flat && p.n % CE::IN_LINE) ? (int)(p.n / CE::IN_LINE) * CE::IN_LINE / lm.W : -1;
+    const int tail_chunk_out = sizeof(TIn) == sizeof(TOut) ? tail_chunk_in
+                               : (pipe.flat && p.n % CE::OUT_LINE) ? (int)(p.n / CE::OUT_LINE) * CE::OUT_LINE / lm.W : -1;
+
+    // Loads run one chunk ahead of the arithmetic (two stages): the chunk after the one being worked on is issued
+    // at the top of every step, from the same cursor.
+    auto issue = [&](const Cursor& c, int stg) {
+        HS_DBG_CHECK(c.row >= 0 && c.row < p.rows && c.chunk >= 0 && c.chunk < nchunks && stg < S, kDbgTmaCoord,
+                     ((unsigned long long)c.row << 32) | (unsigned)c.chunk, return);
+        if (TMA) pipe.issue(&tm_a, &tm_b, c.row, c.chunk * lm.W, stg);
+        else CE::wide_load_async(p, pipe.in_a(stg), pipe.in_b(stg), lane, c.row, (long long)c.chunk * lm.W, lm.W);
+    };
+
+    uint4* const handoff = p.desc;  // [GW]: the value of x after a slot's beginning of a row
+    // x_0 of the next row that starts in the walk, in flight while the current row is worked on
+    auto row_start_after = [&](int r) {
+        if (n_head && r == row_hi) return (len - n_rest > n_head) ? first_whole : -1;
+        return (r + 1 < row_hi) ? r + 1 : -1;
+    };
+    int x0_row = n_head ? row_hi : (len > n_rest ? first_whole : -1);
+    typename CE::RawX0 x0_next = CE::load_x0(p, x0_row >= 0 ? (long long)x0_row : p.rows);
+    Cursor cur = start();
+    issue(cur, 0);
+    Desc early;  // the previous slot's hand-over word, read ahead of its use
+    early.lo = 0ull; early.hi = 0ull;
+    if (n_rest && len - n_rest <= 1) early = ld_desc(handoff + (gw - 1));
+    typename CE::Wide wd = CE::wide_of(p, cur.row, PLAIN);
+    E state = identity_elem<CE::SIGNED>();
+    bool fresh = true;          // the next chunk starts a segment (a row from x_0, or the rest of a row)
+    int stage = 0;
+    uint32_t parity = 0;
+    for (int consumed = 0; consumed < len; ++consumed) {
+        const int row = cur.row, chunk = cur.chunk, colbase = chunk * lm.W;
+        Cursor nxt = cur;
+        advance(nxt);
+        const bool more = consumed + 1 < len;
+        if (more) issue(nxt, stage ^ 1);
+        if (TMA) {
+            if (!pipe.wait(stage, parity)) {
+                if (lane == 0) record_error(p, kErrCopyTimeout, row);
+                if (more) (void)pipe.wait(stage ^ 1, stage ? parity ^ 1u : parity);
+                break;
+            }
+        } else {
+            if (more) cp_async_wait<1>();
+            else cp_async_wait<0>();
+            __syncwarp();
+        }
+        if (fresh) {
+            wd = CE::wide_of(p, row, PLAIN);
+            if (chunk == 0) {
+                state = CE::x0_elem(x0_next);   // (x0_row == row here)
+                x0_row = row_start_after(row);
+                x0_next = CE::load_x0(p, x0_row >= 0 ? (long long)x0_row : p.rows);
+            } else {
+                // the rest of a row: its beginning is the previous slot's, walked first there (the word was asked
+                // for a chunk ago, so that its way through L2 is not waited for here)
+                Desc d = early;
+                bool got = d.hi == p.call_id;
+                for (unsigned int polls = 0; !got && polls < p.spin_limit; ++polls) {
+                    __nanosleep(200);
+                    d = ld_desc(handoff + (gw - 1));
+                    got = d.hi == p.call_id;
+                }
+                if (!got) {
+                    if (lane == 0) record_error(p, kErrLookbackTimeout, row);
+                    if (TMA && more) (void)pipe.wait(stage ^ 1, stage ? parity ^ 1u : parity);
+                    break;
+                }
+                state.A = neg_inf();
+                state.m = __uint_as_float((uint32_t)d.lo);
+                state.s = __uint_as_float((uint32_t)(d.lo >> 32));
+                state.p = 0u;
+            }
+        }
+        const uint32_t sm_a = pipe.in_a(stage), sm_b = pipe.in_b(stage), sm_out = pipe.out(stage);
+        if (TMA && chunk == tail_chunk_in) {
+            CE::tail_load(p, sm_a, sm_b, lane, row, colbase);
+            __syncwarp();
+        }
+        const int col0 = colbase + lane * K;
+        const bool ragged = tail_ragged && chunk == nchunks - 1;
+        typename CE::Pending pd;
+        E total_e;
+        CE::template phase1<PLAIN>(p, sm_a, sm_b, off, lm, lane, row, col0, ragged, wd, pd, total_e);
+        if (TMA) pipe.acquire_out();
+        CE::template phase2<PLAIN>(p, sm_a, sm_b, sm_out, off, lm, row, col0, wd, pd, state);
+        state = compose(state, total_e);
+        renormalise(state);
+        if (TMA) {
+            pipe.store_from(&tm_o, row, colbase, sm_out);
+            if (chunk == tail_chunk_out) CE::tail_store(p, sm_out, lane, row, colbase);
+        } else {
+            __syncwarp();
+            CE::wide_store(p, sm_out, lane, row, colbase, lm.W);
+        }
+        __syncwarp();
+        fresh = nxt.chunk == 0;           // the next chunk starts a row ...
+        if (consumed + 1 == n_head) {
+            // the beginning of the last row of the share is done: hand the value of x to the slot that has the rest
+            if (lane == 0) {
+                Desc d;
+                d.lo = (unsigned long long)__float_as_uint(state.m) | ((unsigned long long)__float_as_uint(state.s) << 32);
+                d.hi = p.call_id;
+                st_desc(handoff + gw, d);
+            }
+            fresh = true;
+        }
+        if (consumed + 1 == len - n_rest) fresh = true;   // ... or the rest of the share's first row
+        if (n_rest && consumed + 2 == len - n_rest) early = ld_desc(handoff + (gw - 1));
+        cur = nxt;
+        stage ^= 1;
+        if (stage == 0) parity ^= 1u;
+    }
+    if (TMA) pipe.drain();
+}
+
+// ------------------------------------------------------------------------------------------
 // (b) Single-pass kernel with decoupled look-back, for few long rows.
 //
 // A row is cut into tiles of W chunks (W = compute warps per CTA).  CTA c handles tiles c, c+G,

@@ -581,3 +581,50 @@ def test_lookback_protocol_stress_smallest_tiles(hs, oracle):
     finally:
         hs.tune("LB_WARPS", -1)
         hs.tune("LB_GROUP", -1)
+
+
+@pytest.mark.parametrize("rows,n,kind", [
+    (2500, 2048, "log"), (3000, 1536, "log"), (2369, 1024, "log"), (3001, 5000, "log"), (2600, 4090, "log"),
+    (2500, 2048, "linear"), (3000, 3001, "linear"), (2500, 4096, "bf16"), (2900, 1500, "bf16"), (2450, 2050, "complex"),
+    (7000, 1030, "log"),
+])
+def test_rows_shared_out_by_chunks(hs, oracle, rows, n, kind):
+    """Between one and a few rows per warp slot the batched kernel cuts the rows to measure: every slot takes an equal
+    share of the rows' chunks -- the rest of a row, whole rows, the beginning of a row -- and the value of x crosses
+    from slot to slot through the workspace.  Forced on (the automatic choice takes it only where whole rows per slot
+    would leave slots idle) and compared with the oracle; forced off, the results must be the same bits."""
+    hs.set_path(hs.PATH_BATCHED)
+    outs = []
+    for spans in (1, 0):
+        hs.tune("SPANS", spans)
+        try:
+            if kind == "linear":
+                w = workloads.make(4, rows=rows, n=n, seed=rows)
+                x = hs.scan_linear(*(to_dev(w.tensors[k]) for k in ("a", "b", "x0")))
+                torch.cuda.synchronize()
+                if spans:
+                    assert_signed_close(to_f64(x), oracle.scan_linear(w.tensors["a"], w.tensors["b"], w.tensors["x0"]), f"spans {rows}x{n}")
+                outs.append(x)
+            elif kind == "complex":
+                w = workloads.make(4, rows=rows, n=n, seed=rows)
+                with np.errstate(divide="ignore"):
+                    z = [np.log(w.tensors[k].astype(np.complex128)).astype(np.complex64) for k in ("a", "b", "x0")]
+                zo = hs.scan_log_complex(*(torch.from_numpy(v).cuda() for v in z))
+                torch.cuda.synchronize()
+                if spans:
+                    zz = zo.cpu().numpy()
+                    got = np.exp(zz.real.astype(np.float64)) * np.where(np.round(zz.imag / np.pi) == 1, -1.0, 1.0)
+                    assert_signed_close(got, oracle.scan_linear(w.tensors["a"], w.tensors["b"], w.tensors["x0"]), f"spans complex {rows}x{n}")
+                outs.append(torch.view_as_real(zo))
+            else:
+                w = workloads.make(5 if kind == "bf16" else 2, rows=rows, n=n, seed=rows)
+                if spans:
+                    run_log(hs, oracle, w.tensors, path=hs.PATH_BATCHED, what=f"spans {kind} {rows}x{n}")
+                out = hs.scan_log(*(to_dev(w.tensors[k]) for k in ("log_a", "log_b", "log_x0")))
+                torch.cuda.synchronize()
+                outs.append(out)
+        finally:
+            hs.tune("SPANS", -1)
+    a, b = outs
+    same = (a == b) | (torch.isnan(a) & torch.isnan(b))
+    assert same.all(), "the same chunks in another order of slots must give the same bits"
