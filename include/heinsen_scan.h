@@ -77,7 +77,7 @@ typedef enum {
 typedef enum {
     HS_PATH_AUTO = 0,     /* rows >= a few per SM: batched kernel; else look-back kernel */
     HS_PATH_BATCHED = 1,  /* one warp walks one row, carry in registers */
-    HS_PATH_LOOKBACK = 2  /* rows cut into tiles, single pass with decoupled look-back */
+    HS_PATH_LOOKBACK = 2  /* rows cut into tiles, single pass, the carry between tiles propagated beside the tiles' arithmetic */
 } hs_path;
 
 /*
@@ -134,9 +134,10 @@ hs_status heinsen_scan_log(const void* log_a, const void* log_b, const void* log
 
 /*
  * Scratch size in bytes for a problem of this shape (any path, any type): a 256-byte
- * header (status words) plus 16 bytes per tile and per group of tiles of the look-back
- * kernel, or per warp slot of the batched kernel when it shares rows out among its
- * slots -- the carry between parts that the associativity of prefix sums allows
+ * header (status words) plus two 16-byte words per tile of the look-back kernel (the
+ * tile's aggregate, the value entering the tile), or one per warp slot of the batched
+ * kernel when it shares rows out among its slots -- the carry between parts that the
+ * associativity of prefix sums allows
  * (Summary, footnote on associativity).  Returns 0 only for invalid sizes.
  */
 size_t heinsen_scan_workspace_bytes(int64_t rows, int64_t n);
@@ -239,10 +240,11 @@ hs_status scan_log(const void* log_a, const void* log_b, const void* log_x0, voi
 /* Process-wide kernel selection (default HS_PATH_AUTO); for tests and benchmarks. */
 hs_status heinsen_scan_set_path(hs_path path);
 /*
- * Test hook for the bounded wait of the look-back kernel (the only device-side wait on another
- * CTA).  `lookback_spin_limit` bounds the polls of predecessor descriptors (0 restores the
- * default); `mute_tile` >= 0 makes that tile skip publishing its descriptors, so that its
- * successors run out of polls, record HS_ERR_LOOKBACK_TIMEOUT in the workspace and leave;
+ * Test hook for the bounded waits of the look-back kernel (the only device-side waits on another
+ * CTA).  `lookback_spin_limit` bounds the polls of a descriptor (0 restores the default);
+ * `mute_tile` >= 0 makes that tile skip publishing its aggregate, so that the CTA that propagates
+ * the carries and the tiles waiting for it run out of polls, record HS_ERR_LOOKBACK_TIMEOUT in the
+ * workspace and leave;
  * -1 disables it.  Nothing faults or hangs: the kernel returns and the context stays usable.
  */
 hs_status heinsen_scan_debug_config(uint32_t lookback_spin_limit, int64_t mute_tile);
@@ -266,7 +268,7 @@ int heinsen_scan_debug_window_ok(uint64_t addr, uint64_t bytes, uint64_t base, u
 /*
  * Tuning knobs, for sweeps and for tests that force a variant; every knob has a measured default
  * that is chosen per call.  `name` is one of "NO_TMA", "ROWS_PER_WARP", "WARPS", "STAGES",
- * "ROW_TICKETS", "SPANS", "NO_FLAT", "NO_PDL" (row-batched kernel), "LB_STAGES", "LB_WARPS", "LB_GROUP",
+ * "ROW_TICKETS", "SPANS", "NO_FLAT", "NO_PDL" (row-batched kernel), "LB_STAGES", "LB_WARPS",
  * "LB_SLEEP_IDLE", "LB_SLEEP_READY", "LB_CTAS_PER_SM" (look-back kernel); value >= 0 sets the knob
  * (clamped to its range), value < 0 returns it to its default.  The environment variables
  * HEINSEN_SCAN_<name> give the initial values; they are read once per process, not per call.

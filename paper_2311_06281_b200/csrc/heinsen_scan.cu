@@ -178,11 +178,11 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 // heinsen_scan_tune() changes a knob, so that a launch costs no getenv().
 enum Knob : int {
     kKnobNoTma = 0, kKnobRowsPerWarp, kKnobWarps, kKnobRowTickets, kKnobNoFlat, kKnobNoPdl, kKnobLbStages,
-    kKnobLbWarps, kKnobLbGroup, kKnobLbSleepIdle, kKnobLbSleepReady, kKnobLbCtasPerSm, kKnobStages, kKnobSpans, kKnobCount
+    kKnobLbWarps, kKnobLbSleepIdle, kKnobLbSleepReady, kKnobLbCtasPerSm, kKnobStages, kKnobSpans, kKnobCount
 };
 const char* const kKnobNames[kKnobCount] = {
     "NO_TMA", "ROWS_PER_WARP", "WARPS", "ROW_TICKETS", "NO_FLAT", "NO_PDL", "LB_STAGES",
-    "LB_WARPS", "LB_GROUP", "LB_SLEEP_IDLE", "LB_SLEEP_READY", "LB_CTAS_PER_SM", "STAGES", "SPANS"};
+    "LB_WARPS", "LB_SLEEP_IDLE", "LB_SLEEP_READY", "LB_CTAS_PER_SM", "STAGES", "SPANS"};
 constexpr int kKnobUnset = INT_MIN;
 std::atomic<int> g_knobs[kKnobCount];
 std::once_flag g_knobs_once;
@@ -308,8 +308,7 @@ int choose_path(long long rows, const DeviceInfo& d) {
 size_t workspace_bytes_for(long long rows, long long n, int min_chunk = kMinChunk) {
     // sized for the smallest chunk so that it covers every type
     const long long tpr = lookback_tiles_per_row(n, min_chunk, kLookbackMinWarps);
-    const long long gpr = (tpr + 1) / 2;  // groups hold at least 2 tiles
-    size_t words = (size_t)(rows * (tpr + gpr));
+    size_t words = (size_t)(rows * tpr * 2);  // a tile's aggregate, and the value entering it
     // ... or, for the batched kernel that shares the rows' chunks out among its warp slots, one word per slot
     // (at most 16 warps on each of at most 256 SMs; only shapes with at least one row per slot use it)
     if (rows >= 128 && words < kMaxWarpSlots) words = kMaxWarpSlots;
@@ -485,20 +484,12 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         warps = W + nlb + 1;  // + the publisher warp
         p.tiles_per_row = (int)lookback_tiles_per_row(p.n, chunk, W);
         p.num_tiles = p.rows * p.tiles_per_row;
-        // group = a little less than the tiles one wave of CTAs processes (the grid is sm_count CTAs, one
-        // per SM).  With exactly one wave per group the group's last tile always sits on the last CTA and
-        // the group closes only after the slowest CTA of the wave; 11/12 of a wave lets the closing position
-        // move through the CTAs and the bulk of a wave close before its stragglers (measured on cfg3:
-        // 148 tiles per group 157 us, 136: 149 us, 128: 150 us, 112: 154 us, 74: 154 us).
-        p.lb_group = dev.sm_count - dev.sm_count / 12;
-        if (p.lb_group > kLbMaxGroup) p.lb_group = kLbMaxGroup;
-        if (p.lb_group < 2) p.lb_group = 2;
-        p.lb_group = knob(kKnobLbGroup, p.lb_group, 2, kLbMaxGroup);
-        p.groups_per_row = (p.tiles_per_row + p.lb_group - 1) / p.lb_group;
-        const size_t need = sizeof(Header) + ((size_t)p.num_tiles + (size_t)p.rows * p.groups_per_row) * 16;
+        // rows of several tiles: a word per tile for its aggregate and one for the value entering it
+        p.lb_server = p.tiles_per_row > 1 ? 1 : 0;
+        const size_t need = sizeof(Header) + (p.lb_server ? (size_t)p.num_tiles * 2 * 16 : 0);
         if (workspace_bytes < need) return HS_ERR_WORKSPACE_TOO_SMALL;
         p.desc = reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(workspace) + sizeof(Header));
-        p.gdesc = p.desc + p.num_tiles;
+        p.edesc = p.desc + p.num_tiles;
         fn = ke.lookback;
         grid = 0;  // set below from occupancy
     }
@@ -538,8 +529,9 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         if (e != cudaSuccess) return cuda_fail("cudaOccupancyMaxActiveBlocksPerMultiprocessor", e);
         if (per_sm < 1) return HS_ERR_INVALID_ARG;
         per_sm = knob(kKnobLbCtasPerSm, per_sm, 1, per_sm);
+        // (with the carry server: one CTA of the grid is the server, the others take the tiles)
         long long g = (long long)per_sm * dev.sm_count;
-        if (g > p.num_tiles) g = p.num_tiles;
+        if (g > p.num_tiles + p.lb_server) g = p.num_tiles + p.lb_server;
         grid = (int)g;
         if (p.tiles_per_row == 1) {
             // every row is a single tile: no tile waits for another, so neither the descriptors nor the
@@ -560,7 +552,7 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
             e = cudaLaunchKernelExC(&cfg, fn, args);
         } else {
             // every descriptor starts as "nothing yet"
-            e = cudaMemsetAsync(p.desc, 0, ((size_t)p.num_tiles + (size_t)p.rows * p.groups_per_row) * 16, stream);
+            e = cudaMemsetAsync(p.desc, 0, (size_t)p.num_tiles * 2 * 16, stream);
             if (e != cudaSuccess) return cuda_fail("cudaMemsetAsync", e);
             e = cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(warps * 32), args, smem, stream);
         }

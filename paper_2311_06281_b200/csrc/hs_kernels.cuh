@@ -4,8 +4,9 @@
 //                          the value of x carried in registers from chunk to chunk (rows >= a few
 //                          per SM); rows are handed out to the warps by slot or by ticket.
 //   lookback_scan_kernel : rows are cut into tiles of WARPS chunks; one CTA per tile, single
-//                          pass, the carry between tiles found by decoupled look-back over
-//                          per-tile descriptors in the caller's workspace (few, long rows).
+//                          pass, the carry between tiles propagated by one CTA of the grid (the
+//                          carry server) through per-tile descriptors in the caller's workspace
+//                          (few, long rows).
 //
 // Both read every input element once and write every output element once.  Chunks travel
 // HBM -> shared memory by TMA (per-warp mbarrier pipelines, 128-byte swizzle) and back by TMA
@@ -68,12 +69,11 @@ struct Params {
     int tiles_per_row;
     long long num_tiles;
     uint4* desc;                // [num_tiles] tile descriptors, zeroed before the launch
-    uint4* gdesc;               // [rows * groups_per_row] group descriptors, zeroed before the launch
-    int groups_per_row;         // ceil(tiles_per_row / lb_group)
-    int lb_group;               // tiles per group: the CTAs of the launch, at most kLbMaxGroup
+    uint4* edesc;               // [num_tiles] values entering the tiles, zeroed before the launch
+    int lb_server;              // rows of several tiles: the grid's last CTA propagates the carries
     int lb_warps;               // look-back warps per CTA
-    unsigned int lb_sleep_idle;   // ns between polls while the tile's own aggregate is not in yet
-    unsigned int lb_sleep_ready;  // ns between polls afterwards
+    unsigned int lb_sleep_idle;   // ns between the carry server's polls of a batch of tile aggregates
+    unsigned int lb_sleep_ready;  // ns between a tile's polls of the value entering it
     unsigned int spin_limit;    // bound on polls of predecessor flags
     long long mute_tile;        // test hook: this tile never publishes (-1: none)
 };
@@ -1104,40 +1104,29 @@ batched_span_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
 }
 
 // ------------------------------------------------------------------------------------------
-// (b) Single-pass kernel with decoupled look-back, for few long rows.
+// (b) Single-pass kernel for few long rows, the carry between tiles decoupled from the tiles' arithmetic.
 //
 // A row is cut into tiles of W chunks (W = compute warps per CTA).  CTA c handles tiles c, c+G,
 // c+2G, ... (all CTAs are resident: cooperative launch); compute warp w owns the w-th chunk of
-// each tile, and one more warp does nothing but carry propagation.  The kernel is software
-// pipelined so that the latency of the look-back never stalls the arithmetic:
+// each tile, and two more warps do nothing but carry propagation.  The kernel is software
+// pipelined so that the latency of the carry never stalls the arithmetic:
 //
 //   compute warp, iteration i :  phase 1 of tile i   (inputs -> partial sums s_t parked in shared
-//                                                     memory, chunk aggregate handed to a
-//                                                     look-back warp)
+//                                                     memory, chunk aggregate handed to the
+//                                                     publisher warp)
 //                                phase 2 of tile i-D (whose entering value has arrived meanwhile:
 //                                                     outputs, TMA store), D = stages - 2
-//   look-back warp, tile i    :  scan of the W chunk aggregates, publish the tile aggregate,
-//                                assemble the value of x entering the tile from the descriptors
-//                                of the preceding tiles (aggregates until a tile whose value is
-//                                known), publish the tile's own value, hand the carry back.
+//   publisher warp, tile i    :  scan of the W chunk aggregates, publish the tile's aggregate
+//   carry server (last CTA)   :  prefix over the tiles' aggregates in tile order, 32 tiles per
+//                                warp at a time: the value of x entering each tile
+//   look-back warp, tile i    :  wait for that value, hand it to the compute warps.
 //
 // This is the "by parts" evaluation that the associativity of prefix sums allows, done in one
 // pass over HBM.  Every wait is bounded; when one runs out the CTA records an error and leaves.
-// A tile's descriptor is one 16-byte word, read and written with single 128-bit accesses so that
+// A descriptor is one 16-byte word, read and written with single 128-bit accesses so that
 // state and payload always belong together:  {A, m, s, tag},  tag = state | parity << 2,
-// state 0 = nothing yet (the descriptor array is zeroed before every launch), 1 = the tile's
-// aggregate, 2 = the value of x after the tile (A = -inf).
-__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {  // non-blocking
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
+// state 0 = nothing yet (the descriptor arrays are zeroed before every launch), 1 = a tile's
+// aggregate, 2 = the value of x entering a tile (A = -inf).
 // Bounded wait that also gives up when `*abort` becomes non-zero: the flag is looked at between the polls,
 // each of which the hardware suspends for a bounded time of its own.
 __device__ __forceinline__ bool mbar_wait_abortable(uint32_t bar, uint32_t parity, uint32_t limit, const int* abort) {
@@ -1163,20 +1152,21 @@ __device__ __forceinline__ Elem<SIGNED> unpack_elem(const float4 v) {
     return e;
 }
 
-constexpr int kLbPerLane = 5;                       // tile descriptors polled by each lane per round
-constexpr int kLbMaxGroup = 32 * kLbPerLane;        // tiles per group, at most
 constexpr int kLbMaxWarps = 16;                     // compute warps per CTA, at most
+constexpr int kSrvRing = 32;                        // hand-over slots between the batches of the carry server
 
-// Two levels of descriptors keep a look-back to one round trip however long the row is:
-//   tile level  : desc[T]   = aggregate of tile T (state 1), written right after its phase 1;
-//   group level : gdesc[g]  = aggregate of the tiles of group g (state 1), written by the
-//                 look-back of the group's last tile as soon as it has seen the others, and
-//                 later replaced by the value of x after the group (state 2).
-// A group is p.lb_group consecutive tiles of a row -- the tiles that the resident CTAs process at
-// the same time -- so the group descriptors a tile needs are those of earlier waves, already
-// visible when it looks.  The value entering tile j = (value before its group: group aggregates
-// back to the nearest known value) composed with (the aggregates of the tiles of its own group
-// before it).  Both levels are polled together, every load of a round in flight at once.
+// The carry between tiles goes through two arrays of 16-byte descriptors, one word per tile:
+//   desc[T]  = aggregate of tile T (state 1), written by the tile's CTA right after its phase 1;
+//   edesc[T] = value of x entering tile T (state 2), written by the carry server.
+// The carry server is the last CTA of the grid; it computes no tile.  Its warps take batches of 32 consecutive
+// tiles in turn (lane l <-> tile 32q + l): wait for the 32 aggregates, scan them, take the value entering the
+// batch from the batch before (through the server's shared memory: the only sequential step, a compose and a
+// flag per 32 tiles), write the 32 entering values.  A tile's CTA then waits for ONE word that only it reads.
+// Against a look-back in which every tile reads its predecessors' descriptors and composes them itself:
+// each descriptor is read once instead of by every tile of its round (no lines of L2 that all SMs poll at
+// once), a tile's warp has nothing to reduce (the look-back warp's reductions, ~4400 cycles per tile, paced
+// the whole kernel), and nothing a tile waits for depends on what a tile of the same round publishes after
+// a look-back of its own.
 template <int MODE, typename TIn, typename TOut, int K>
 struct Lookback {
     using CE = ChunkEngine<MODE, TIn, TOut, K>;
@@ -1204,122 +1194,113 @@ struct Lookback {
         st_desc(p.desc + T, pack(e, kAgg));
     }
 
-    // lane 0 holds the newest part, higher lanes older ones; returns their composition in every lane
-    __device__ static __forceinline__ E reduce_newest_first(E part, int lane) {
-#pragma unroll
-        for (int dd = 1; dd < 32; dd <<= 1) {
-            E other = shfl_down_elem(part, dd);
-            E c = compose(other, part);
-            if (lane + dd < 32) part = c;
-        }
-        return shfl_elem(part, 0);
-    }
     __device__ static __forceinline__ bool give_up(const Params& p, unsigned int& polls) {
         return ++polls >= p.spin_limit ||
                ((polls & 255u) == 0u && *(volatile unsigned long long*)&p.ws->error_id == p.call_id);
     }
 
-    // Warp-collective: everything a look-back warp does for tile T (tile j of `row`).  It starts
-    // reading the predecessors' descriptors at once and in the same loop watches for the tile's own
-    // aggregate (mbarrier `agg_bar`, value at `total_src`; the compute warps have already published
-    // it); once both are there it returns the value of x entering the tile.  Publishes the group
-    // descriptors the tile is responsible for.
-    __device__ static __forceinline__ E run(const Params& p, long long T, int j, long long row, int lane,
-                                            uint32_t agg_bar, uint32_t agg_parity, const float4* total_src,
-                                            const volatile int* abort_flag, bool& failed,
-                                            unsigned int& total_polls) {
+    // Warp-collective, in a tile's CTA: waits for the value of x entering tile T (every lane reads the same word).
+    __device__ static __forceinline__ E await_entering(const Params& p, long long T, const volatile int* abort_flag,
+                                                       bool& failed, unsigned int& total_polls) {
         failed = false;
-        const int gsz = p.lb_group;
-        const int g = j / gsz, k = j - g * gsz;                    // group, position in group
-        const long long gbase = row * p.groups_per_row;            // first group descriptor of the row
-        const bool closes_group = (k == gsz - 1) || (j == p.tiles_per_row - 1);
-        const bool full_group = (k == gsz - 1);
-        const bool publish = (T != p.mute_tile);
         unsigned int polls = 0;
-        const E x0e = CE::row_start(p, row);
-
-        // tiles of the own group before this one: lane l looks at tiles j-1-5l .. j-5-5l (dist <= k);
-        // groups before the own one: lane l looks at group g-1-l; group -1 is x_0
-        Desc td[kLbPerLane];
-#pragma unroll
-        for (int q = 0; q < kLbPerLane; ++q) { td[q].lo = 0ull; td[q].hi = 0ull; }
-        Desc gd;
-        gd.lo = 0ull; gd.hi = 0ull;
-        bool own_ready = false, tiles_done = (k == 0), groups_done = false, group_agg_sent = false;
-        E tile_total = identity_elem<SIGNED>();
-        E before_in_group = identity_elem<SIGNED>();
-        E acc = identity_elem<SIGNED>();
-        int gwin = 1;  // distance of the nearest group of the current group window
-        while (true) {
-            if (!tiles_done) {
-#pragma unroll
-                for (int q = 0; q < kLbPerLane; ++q) {
-                    const int dist = kLbPerLane * lane + q + 1;
-                    HS_DBG_CHECK(dist > k || (T - dist >= 0 && T - dist < p.num_tiles), kDbgTile, T - dist, continue);
-                    if (dist <= k) td[q] = ld_desc(p.desc + (T - dist));
-                }
-            }
-            const int gg = g - gwin - lane;
-            HS_DBG_CHECK(groups_done || gg < 0 || gbase + gg < p.rows * p.groups_per_row, kDbgTile, gbase + gg, groups_done = true);
-            if (!groups_done && gg >= 0) gd = ld_desc(p.gdesc + gbase + gg);
+        HS_DBG_CHECK(T >= 0 && T < p.num_tiles, kDbgTile, T, failed = true);
+        Desc d;
+        d.lo = 0ull; d.hi = 0ull;
+        while (!failed) {
+            d = ld_desc(p.edesc + T);
             ++total_polls;
+            d.lo = __shfl_sync(0xffffffffu, d.lo, 0);
+            d.hi = __shfl_sync(0xffffffffu, d.hi, 0);
+            if (state_of(d) == kInc) break;
+            if (__any_sync(0xffffffffu, *abort_flag || give_up(p, polls))) { failed = true; break; }
+            __nanosleep(p.lb_sleep_ready);
+        }
+        return unpack(d);
+    }
 
-            if (!own_ready && mbar_test(agg_bar, agg_parity)) {
-                own_ready = true;
-                tile_total = unpack_elem<SIGNED>(*total_src);  // scanned and published by the compute warps
+    // The carry server (all warps of the grid's last CTA).  `ring` is kSrvRing hand-over slots in its shared memory.
+    struct ServerRing {
+        float2 value[kSrvRing];             // (m, s) of x after batch q, in slot q % kSrvRing
+        unsigned long long done[kSrvRing];  // q + 1 once it is there
+        int abort;
+    };
+    __device__ static __forceinline__ void serve(const Params& p, ServerRing* ring, int lane, int warp, int nwarps) {
+        if (threadIdx.x < kSrvRing) ring->done[threadIdx.x] = 0ull;
+        if (threadIdx.x == 0) ring->abort = 0;
+        __syncthreads();
+        const long long nb = (p.num_tiles + 31) / 32;
+        for (long long q = warp; q < nb; q += nwarps) {
+            const long long T = q * 32 + lane;
+            const bool active = T < p.num_tiles;
+            long long row = 0;
+            int j = 0;
+            if (active) {
+                row = T / p.tiles_per_row;
+                j = (int)(T - row * p.tiles_per_row);
             }
-            if (!tiles_done) {
-                bool ready = true;
-#pragma unroll
-                for (int q = 0; q < kLbPerLane; ++q) {
-                    const int dist = kLbPerLane * lane + q + 1;
-                    if (dist <= k && state_of(td[q]) != kAgg) ready = false;
+            HS_DBG_CHECK(!active || (row >= 0 && row < p.rows), kDbgTile, T, (void)0);
+            const bool starts_row = active && j == 0;
+            E x0e = identity_elem<SIGNED>();
+            if (starts_row) x0e = CE::row_start(p, row);
+            // the batch's aggregates
+            Desc d;
+            d.lo = 0ull; d.hi = 0ull;
+            unsigned int polls = 0;
+            bool ok = true;
+            while (true) {
+                if (active && state_of(d) != kAgg) d = ld_desc(p.desc + T);
+                if (__all_sync(0xffffffffu, !active || state_of(d) == kAgg)) break;
+                if (__any_sync(0xffffffffu, *(volatile int*)&ring->abort || give_up(p, polls))) { ok = false; break; }
+                __nanosleep(p.lb_sleep_idle);
+            }
+            E part = identity_elem<SIGNED>();
+            if (ok) {
+                if (active) part = unpack(d);
+                if (starts_row) part = compose(x0e, part);  // a value (A = -inf): forgets what came before the row
+            }
+            E wex, total;
+            warp_scan(part, lane, wex, total);
+            // the value entering the batch: from the batch before
+            E cin = identity_elem<SIGNED>();
+            if (ok && q > 0) {
+                const int slot = (int)((q - 1) % kSrvRing);
+                polls = 0;
+                while (!__all_sync(0xffffffffu, *(volatile unsigned long long*)&ring->done[slot] == (unsigned long long)q)) {
+                    if (__any_sync(0xffffffffu, *(volatile int*)&ring->abort || give_up(p, polls))) { ok = false; break; }
                 }
-                if (__all_sync(0xffffffffu, ready)) {
-                    E part = identity_elem<SIGNED>();
-#pragma unroll
-                    for (int q = 0; q < kLbPerLane; ++q) {
-                        const int dist = kLbPerLane * lane + q + 1;
-                        if (dist <= k) part = compose(unpack(td[q]), part);  // older first
-                    }
-                    before_in_group = reduce_newest_first(part, lane);
-                    tiles_done = true;
+                if (ok) {
+                    __threadfence_block();
+                    cin.A = neg_inf();
+                    cin.m = *(volatile float*)&ring->value[slot].x;
+                    cin.s = *(volatile float*)&ring->value[slot].y;
+                    cin.p = 0u;
                 }
             }
-            if (own_ready && tiles_done && full_group && publish && !group_agg_sent) {
-                // later groups need only this, not our own carry: publish it at once
-                HS_DBG_CHECK(gbase + g < p.rows * p.groups_per_row, kDbgTile, gbase + g, group_agg_sent = true);
-                if (lane == 0 && !group_agg_sent) st_desc(p.gdesc + gbase + g, pack(compose(before_in_group, tile_total), kAgg));
-                group_agg_sent = true;
-            }
-            if (!groups_done) {
-                const uint32_t s = (gg >= 0) ? state_of(gd) : (uint32_t)kInc;  // gg == -1: x_0; beyond: ignored
-                const uint32_t inc_mask = __ballot_sync(0xffffffffu, s == kInc);
-                const uint32_t ok_mask = __ballot_sync(0xffffffffu, s != kNotReady);
-                const uint32_t need = inc_mask ? ((2u << (__ffs(inc_mask) - 1)) - 1u) : 0xffffffffu;
-                if ((ok_mask & need) == need) {
-                    const int lstar = inc_mask ? (__ffs(inc_mask) - 1) : 31;
-                    E gp = identity_elem<SIGNED>();
-                    if (lane <= lstar) gp = (gg >= 0) ? unpack(gd) : x0e;
-                    acc = compose(reduce_newest_first(gp, lane), acc);
-                    if (inc_mask) {
-                        groups_done = true;
-                    } else gwin += 32;  // every group of this window is an aggregate: look further back
+            if (!ok) {
+                if (lane == 0 && !*(volatile int*)&ring->abort) {
+                    record_error(p, kErrLookbackTimeout, q * 32);
+                    ring->abort = 1;
                 }
+                break;
             }
-            if (own_ready && tiles_done && groups_done) break;
-            if (*abort_flag || give_up(p, polls)) { failed = true; return acc; }
-            __nanosleep(own_ready ? p.lb_sleep_ready : p.lb_sleep_idle);  // polls cost L2 bandwidth and issue slots
-        }
-        const E entering = compose(acc, before_in_group);
-        if (closes_group && publish && lane == 0) {
-            E after = compose(entering, tile_total);
+            E after = compose(cin, total);
             renormalise(after);
-            after.A = neg_inf();
-            after.p = 0u;
-            st_desc(p.gdesc + gbase + g, pack(after, kInc));
+            if (lane == 0) {
+                const int slot = (int)(q % kSrvRing);
+                *(volatile float*)&ring->value[slot].x = after.m;
+                *(volatile float*)&ring->value[slot].y = after.s;
+                __threadfence_block();
+                *(volatile unsigned long long*)&ring->done[slot] = (unsigned long long)(q + 1);
+            }
+            if (active) {
+                E ent = starts_row ? x0e : compose(cin, wex);
+                renormalise(ent);
+                ent.A = neg_inf();
+                ent.p = 0u;
+                st_desc(p.edesc + T, pack(ent, kInc));
+            }
         }
-        return entering;
     }
 };
 
@@ -1329,11 +1310,10 @@ constexpr int kLbMaxStages = 5; // input stages per compute warp, at most
 struct alignas(16) Exchange {
     float4 agg[kLbRing][kLbMaxWarps];    // per-warp aggregates of a tile; the publisher warp replaces them in
                                          // place by the per-warp exclusive prefixes within the tile
-    float4 total[kLbRing];               // the tile's aggregate (written by the last compute warp to finish phase 1)
     float4 carry[kLbRing];               // value of x entering the tile (m, s)
-    unsigned long long total_ready[kLbRing];  // mbarrier: the publisher warp has written total and wexcl
+    unsigned long long total_ready[kLbRing];  // mbarrier: the publisher warp has written wexcl and published the tile
     unsigned long long agg_ready[kLbRing];    // mbarrier: all compute warps have delivered their aggregate
-    unsigned long long carry_ready[kLbRing];  // mbarrier: a look-back warp has delivered wexcl and carry
+    unsigned long long carry_ready[kLbRing];  // mbarrier: a look-back warp has delivered the carry
     int abort;
     int pad[3];
 };
@@ -1431,7 +1411,13 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
     if (threadIdx.x == 0 && blockIdx.x == 0) p.ws->started_id = p.call_id;
     __syncthreads();
 
-    const long long G = gridDim.x;
+    // rows of several tiles: the grid's last CTA is the carry server, the others take the tiles
+    const bool served = p.lb_server != 0;
+    if (served && blockIdx.x == gridDim.x - 1) {
+        LB::serve(p, reinterpret_cast<typename LB::ServerRing*>(smem), lane, warp, (int)(blockDim.x >> 5));
+        return;
+    }
+    const long long G = gridDim.x - (served ? 1 : 0);
     const int tpr = p.tiles_per_row;
     const long long first = blockIdx.x;
     const long long my_tiles = first < p.num_tiles ? (p.num_tiles - first + G - 1) / G : 0;
@@ -1459,10 +1445,7 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
             E wex, tile_total;
             warp_scan(mine, lane, wex, tile_total);
             if (lane < W) xc->agg[b][lane] = pack_elem<SIGNED>(wex);  // every lane has read its aggregate by now
-            if (lane == 0) {
-                if (cur.T != p.mute_tile) LB::publish_agg(p, cur.T, tile_total);
-                xc->total[b] = pack_elem<SIGNED>(tile_total);
-            }
+            if (lane == 0 && cur.T != p.mute_tile) LB::publish_agg(p, cur.T, tile_total);
             __syncwarp();
             if (lane == 0) mbar_arrive(total_bar + 8 * b);
         }
@@ -1476,13 +1459,17 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
         const int lb_rows = lb_stride / tpr, lb_rem = lb_stride % tpr;
         for (long long i = warp - W; i < my_tiles; i += NLB, cur.advance(lb_stride, lb_rows, lb_rem, tpr)) {
             const long long T = cur.T;
-            const long long row = cur.row;
-            const int j = cur.j;
             const int b = (int)(i % kLbRing);
             bool failed = false;
             unsigned int npolls = 0;
-            const E carry = LB::run(p, T, j, row, lane, total_bar + 8 * b, (uint32_t)((i / kLbRing) & 1), &xc->total[b],
-                                    &xc->abort, failed, npolls);
+            // (the tile's own aggregate first: the warp must not run ahead of the ring slots the compute warps hold)
+            if (!mbar_wait_abortable(total_bar + 8 * b, (uint32_t)((i / kLbRing) & 1), kCopySpinLimit, &xc->abort)) {
+                if (lane == 0) mbar_arrive(carry_bar + 8 * b);  // (the compute warps look at the abort flag next)
+                break;
+            }
+            E carry;
+            if (served) carry = LB::await_entering(p, T, &xc->abort, failed, npolls);
+            else carry = CE::row_start(p, cur.row);  // every row is a single tile
             if (lane == 0) {
                 if (failed) {
                     record_error(p, kErrLookbackTimeout, T);

@@ -113,7 +113,7 @@ def test_tuning_and_probe_arguments_are_checked_on_the_host(lib):
     import ctypes
     assert lib.heinsen_scan_tune(b"WARPS", 12) == 0 and lib.heinsen_scan_tune(b"WARPS", -1) == 0
     for name in (b"ROWS_PER_WARP", b"STAGES", b"ROW_TICKETS", b"SPANS", b"NO_TMA", b"NO_FLAT", b"NO_PDL", b"LB_STAGES", b"LB_WARPS",
-                 b"LB_GROUP", b"LB_SLEEP_IDLE", b"LB_SLEEP_READY", b"LB_CTAS_PER_SM"):
+                 b"LB_SLEEP_IDLE", b"LB_SLEEP_READY", b"LB_CTAS_PER_SM"):
         assert lib.heinsen_scan_tune(name, -1) == 0, name
     assert lib.heinsen_scan_tune(b"NO_SUCH_KNOB", 1) == 1 and lib.heinsen_scan_tune(None, 1) == 1
     r, s = ctypes.c_double(0), ctypes.c_double(0)

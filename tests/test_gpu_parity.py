@@ -396,9 +396,30 @@ def test_host_buffer_entry_points_signed_and_linear(hs, oracle):
     assert_signed_close(got, np.exp(ref_log) * np.where(ref_sign == 1, -1.0, 1.0), "host log with signs")
 
 
+@pytest.mark.parametrize("rows,n,kind", [
+    (3, 7168 * 40 + 5, "log"),      # 41 tiles per row: rows begin in the middle of the carry server's 32-tile batches
+    (70, 7168 * 2 + 1, "log"),      # 3 tiles per row: ten rows begin inside every batch
+    (1, 7168 * 32, "log"),          # exactly one batch
+    (1, 7168 * 33, "log"),          # one batch and one tile
+    (1, 7168 * 1030 + 17, "log"),   # more batches than the server's hand-over ring has slots, twice over
+    (33, 7168 * 31 + 100, "linear"),  # signed values cross tiles, batches and rows
+    (2, 7168 * 100 + 3, "bf16"),
+])
+def test_lookback_carry_server_batches(hs, oracle, rows, n, kind):
+    """The value of x entering each tile of the single-pass kernel comes from the grid's last CTA, whose warps scan
+    the tiles' aggregates 32 tiles at a time and hand the running value from batch to batch; rows begin anywhere
+    inside a batch.  Every element against the oracle."""
+    if kind == "linear":
+        w = workloads.make(4, rows=rows, n=n)
+        run_linear(hs, oracle, w.tensors, path=hs.PATH_LOOKBACK, signed=True, what=f"{rows} x {n} linear")
+    else:
+        w = workloads.make(5 if kind == "bf16" else 3, rows=rows, n=n)
+        run_log(hs, oracle, w.tensors, path=hs.PATH_LOOKBACK, what=f"{rows} x {n} {kind}")
+
+
 def test_lookback_several_rows_several_groups(hs, oracle):
-    """Look-back path with a few rows, each several descriptor groups long (a group is one wave of tiles),
-    plus a ragged last tile: exercises group aggregates, group values and the row start inside a launch."""
+    """Single-pass path with a few rows, each several rounds of tiles long, plus a ragged last tile: the carry
+    crosses tiles, batches of tiles and the row starts inside a launch."""
     rows, n = 3, 2_650_112 + 40
     w = workloads.make(3, rows=rows, n=n)
     t = w.tensors
@@ -556,8 +577,8 @@ def test_lookback_abort_with_several_tiles_per_cta_returns_promptly(hs):
 
 
 def test_lookback_protocol_stress_smallest_tiles(hs, oracle):
-    """Thousands of tiles of the smallest size (8 compute warps, groups of 2 tiles) exercise the descriptor
-    protocol a hundred times over; every repetition must match the oracle (every wait stays bounded)."""
+    """Thousands of tiles of the smallest size (8 compute warps) exercise the descriptor protocol a hundred
+    times over; every repetition must match the oracle (every wait stays bounded)."""
     n = (1 << 23) + 4096 + 12
     w = workloads.make(3, rows=1, n=n)
     t = w.tensors
@@ -568,7 +589,6 @@ def test_lookback_protocol_stress_smallest_tiles(hs, oracle):
     tol_dev = torch.from_numpy(tol).cuda()
     hs.set_path(hs.PATH_LOOKBACK)
     hs.tune("LB_WARPS", 8)
-    hs.tune("LB_GROUP", 2)
     try:
         ws = hs.new_workspace(1, n, "cuda")
         out = torch.empty_like(la)
@@ -580,7 +600,6 @@ def test_lookback_protocol_stress_smallest_tiles(hs, oracle):
             assert worst <= 1.0, f"repetition {rep}: {worst:.3g} of the tolerance"
     finally:
         hs.tune("LB_WARPS", -1)
-        hs.tune("LB_GROUP", -1)
 
 
 @pytest.mark.parametrize("rows,n,kind", [
