@@ -598,6 +598,12 @@ def test_lookback_protocol_stress_smallest_tiles(hs, oracle):
             hs.check(ws)
             worst = ((out.double() - ref_dev).abs() / tol_dev).max().item()
             assert worst <= 1.0, f"repetition {rep}: {worst:.3g} of the tolerance"
+            # the carry between the tiles is composed in a fixed order (batches of 32 tiles, one after the other),
+            # whatever the order in which the tiles finish: every repetition gives the same bits
+            if rep == 0:
+                first = out.clone()
+            else:
+                assert torch.equal(out, first), f"repetition {rep} differs from the first"
     finally:
         hs.tune("LB_WARPS", -1)
 

@@ -36,6 +36,11 @@ def test_static_scratch_entry_point_matches_regular_entry_point_twice(hs, oracle
         assert hs.lib().heinsen_scan_log_static(la.data_ptr(), lb.data_ptr(), lx0.data_ptr(), out.data_ptr(), rows, n,
                                                 stream) == 0
         hs.check_static("cuda")
+        # (what the loop below does beside the calls, once before the watched region: torch loads the code of a kernel
+        # the first time it runs, and the first copy to the host makes the driver set up its staging memory)
+        out.fill_(float("nan"))
+        to_f64(out)
+        torch.equal(out, regular)
         torch.cuda.synchronize()
         free_before, _ = torch.cuda.mem_get_info()
         torch_before = torch.cuda.memory_allocated()
@@ -48,8 +53,8 @@ def test_static_scratch_entry_point_matches_regular_entry_point_twice(hs, oracle
             # nothing was taken from the device (cudaMalloc and friends would show here) nor through torch
             assert torch.cuda.mem_get_info()[0] == free_before
             assert torch.cuda.memory_allocated() == torch_before
-            # same kernel, same tiles; only the order in which the look-back meets its predecessors may differ
-            assert (out - regular).abs().max().item() <= 2 * float(tol.min()), f"call {call}: static and regular entry differ"
+            # same kernel, same tiles, and the carry between the tiles is composed in a fixed order: the same bits
+            assert torch.equal(out, regular), f"call {call}: static and regular entry differ"
             assert_log_close(to_f64(out), ref, tol, f"static scratch, call {call}, cfg{cid}")
 
 
