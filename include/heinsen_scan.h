@@ -134,7 +134,7 @@ hs_status heinsen_scan_log(const void* log_a, const void* log_b, const void* log
 
 /*
  * Scratch size in bytes for a problem of this shape (any path, any type): a 256-byte
- * header (status words) plus two 16-byte words per tile of the look-back kernel (the
+ * header (status words) plus three 16-byte words per tile of the look-back kernel (the
  * tile's aggregate, the value entering the tile), or one per warp slot of the batched
  * kernel when it shares rows out among its slots -- the carry between parts that the
  * associativity of prefix sums allows

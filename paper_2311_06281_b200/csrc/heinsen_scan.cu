@@ -308,7 +308,7 @@ int choose_path(long long rows, const DeviceInfo& d) {
 size_t workspace_bytes_for(long long rows, long long n, int min_chunk = kMinChunk) {
     // sized for the smallest chunk so that it covers every type
     const long long tpr = lookback_tiles_per_row(n, min_chunk, kLookbackMinWarps);
-    size_t words = (size_t)(rows * tpr * 2);  // a tile's aggregate, and the value entering it
+    size_t words = (size_t)(rows * tpr * 3);  // a tile's aggregate (two words), and the value entering it
     // ... or, for the batched kernel that shares the rows' chunks out among its warp slots, one word per slot
     // (at most 16 warps on each of at most 256 SMs; only shapes with at least one row per slot use it)
     if (rows >= 128 && words < kMaxWarpSlots) words = kMaxWarpSlots;
@@ -484,12 +484,13 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
         warps = W + nlb + 1;  // + the publisher warp
         p.tiles_per_row = (int)lookback_tiles_per_row(p.n, chunk, W);
         p.num_tiles = p.rows * p.tiles_per_row;
-        // rows of several tiles: a word per tile for its aggregate and one for the value entering it
+        // rows of several tiles: two words per tile for its aggregate and one for the value entering it; every word
+        // carries the call's id, so what the workspace held before does not matter and nothing is cleared
         p.lb_server = p.tiles_per_row > 1 ? 1 : 0;
-        const size_t need = sizeof(Header) + (p.lb_server ? (size_t)p.num_tiles * 2 * 16 : 0);
+        const size_t need = sizeof(Header) + (p.lb_server ? (size_t)p.num_tiles * 3 * 16 : 0);
         if (workspace_bytes < need) return HS_ERR_WORKSPACE_TOO_SMALL;
         p.desc = reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(workspace) + sizeof(Header));
-        p.edesc = p.desc + p.num_tiles;
+        p.edesc = p.desc + 2 * p.num_tiles;
         fn = ke.lookback;
         grid = 0;  // set below from occupancy
     }
@@ -551,9 +552,6 @@ hs_status run(Problem& pr, void* workspace, size_t workspace_bytes, cudaStream_t
             cfg.numAttrs = 1;
             e = cudaLaunchKernelExC(&cfg, fn, args);
         } else {
-            // every descriptor starts as "nothing yet"
-            e = cudaMemsetAsync(p.desc, 0, (size_t)p.num_tiles * 2 * 16, stream);
-            if (e != cudaSuccess) return cuda_fail("cudaMemsetAsync", e);
             e = cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(warps * 32), args, smem, stream);
         }
     } else {
@@ -725,8 +723,8 @@ hs_status heinsen_scan_log_static(const void* log_a, const void* log_b, const vo
     pr.din = pr.dout = HS_F32;
     pr.p.in_a = log_a; pr.p.in_b = log_b; pr.p.x0 = log_x0; pr.p.out = log_x;
     pr.p.rows = rows; pr.p.n = n;
-    // run() clears the descriptors it is about to use (cudaMemsetAsync on `stream`), so what the
-    // previous call left in the array does not matter
+    // every descriptor the kernel reads carries the call's id, so what the previous call left in the
+    // array does not matter
     return run(pr, scratch, kStaticScratchBytes, static_cast<cudaStream_t>(stream), HS_PATH_LOOKBACK);
 }
 

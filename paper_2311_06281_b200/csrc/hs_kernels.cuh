@@ -68,8 +68,8 @@ struct Params {
     // look-back kernel only
     int tiles_per_row;
     long long num_tiles;
-    uint4* desc;                // [num_tiles] tile descriptors, zeroed before the launch
-    uint4* edesc;               // [num_tiles] values entering the tiles, zeroed before the launch
+    uint4* desc;                // [2 * num_tiles] the tiles' aggregates, two words each (look-back kernel)
+    uint4* edesc;               // [num_tiles] values entering the tiles
     int lb_server;              // rows of several tiles: the grid's last CTA propagates the carries
     int lb_warps;               // look-back warps per CTA
     unsigned int lb_sleep_idle;   // ns between the carry server's polls of a batch of tile aggregates
@@ -1123,10 +1123,8 @@ batched_span_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, co
 //
 // This is the "by parts" evaluation that the associativity of prefix sums allows, done in one
 // pass over HBM.  Every wait is bounded; when one runs out the CTA records an error and leaves.
-// A descriptor is one 16-byte word, read and written with single 128-bit accesses so that
-// state and payload always belong together:  {A, m, s, tag},  tag = state | parity << 2,
-// state 0 = nothing yet (the descriptor arrays are zeroed before every launch), 1 = a tile's
-// aggregate, 2 = the value of x entering a tile (A = -inf).
+// Descriptors are 16-byte words, each read and written with a single 128-bit access and tagged
+// with the call's id (see Lookback below).
 // Bounded wait that also gives up when `*abort` becomes non-zero: the flag is looked at between the polls,
 // each of which the hardware suspends for a bounded time of its own.
 __device__ __forceinline__ bool mbar_wait_abortable(uint32_t bar, uint32_t parity, uint32_t limit, const int* abort) {
@@ -1155,9 +1153,12 @@ __device__ __forceinline__ Elem<SIGNED> unpack_elem(const float4 v) {
 constexpr int kLbMaxWarps = 16;                     // compute warps per CTA, at most
 constexpr int kSrvRing = 32;                        // hand-over slots between the batches of the carry server
 
-// The carry between tiles goes through two arrays of 16-byte descriptors, one word per tile:
-//   desc[T]  = aggregate of tile T (state 1), written by the tile's CTA right after its phase 1;
-//   edesc[T] = value of x entering tile T (state 2), written by the carry server.
+// The carry between tiles goes through two arrays of 16-byte words in the workspace:
+//   desc[2T], desc[2T+1] = aggregate of tile T, written by the tile's CTA right after its phase 1;
+//   edesc[T]             = value of x entering tile T, written by the carry server.
+// Each word is read and written with one 128-bit access and carries the call's 62-bit id in its upper half: a
+// word counts only if the id is this call's, so the workspace needs no clearing between calls (nor before the
+// first one), and payload and tag cannot be torn apart.
 // The carry server is the last CTA of the grid; it computes no tile.  Its warps take batches of 32 consecutive
 // tiles in turn (lane l <-> tile 32q + l): wait for the 32 aggregates, scan them, take the value entering the
 // batch from the batch before (through the server's shared memory: the only sequential step, a compose and a
@@ -1172,26 +1173,38 @@ struct Lookback {
     using CE = ChunkEngine<MODE, TIn, TOut, K>;
     static constexpr bool SIGNED = CE::SIGNED;
     using E = Elem<SIGNED>;
-    enum : uint32_t { kNotReady = 0, kAgg = 1, kInc = 2 };
-
-    __device__ static __forceinline__ Desc pack(const E& e, uint32_t state) {
-        Desc d;
-        d.lo = (unsigned long long)__float_as_uint(e.A) | ((unsigned long long)__float_as_uint(e.m) << 32);
-        d.hi = (unsigned long long)__float_as_uint(e.s) | ((unsigned long long)(state | ((e.p >> 31) << 2)) << 32);
-        return d;
-    }
-    __device__ static __forceinline__ uint32_t state_of(const Desc& d) { return (uint32_t)(d.hi >> 32) & 3u; }
-    __device__ static __forceinline__ E unpack(const Desc& d) {
-        E e;
-        e.A = __uint_as_float((uint32_t)d.lo);
-        e.m = __uint_as_float((uint32_t)(d.lo >> 32));
-        e.s = __uint_as_float((uint32_t)d.hi);
-        e.p = SIGNED ? ((((uint32_t)(d.hi >> 32)) >> 2) & 1u) << 31 : 0u;
-        return e;
-    }
+    // A tile's aggregate as two words {A, m, id} and {s, parity, id}, the value entering a tile as one word
+    // {m, s, id}: a word belongs to this call exactly if its upper half is the call's id.
     __device__ static __forceinline__ void publish_agg(const Params& p, long long T, const E& e) {
         HS_DBG_CHECK(T >= 0 && T < p.num_tiles, kDbgTile, T, return);
-        st_desc(p.desc + T, pack(e, kAgg));
+        Desc d1, d2;
+        d1.lo = (unsigned long long)__float_as_uint(e.A) | ((unsigned long long)__float_as_uint(e.m) << 32);
+        d2.lo = (unsigned long long)__float_as_uint(e.s) | ((unsigned long long)(e.p >> 31) << 32);
+        d1.hi = d2.hi = p.call_id;
+        st_desc(p.desc + 2 * T, d1);
+        st_desc(p.desc + 2 * T + 1, d2);
+    }
+    __device__ static __forceinline__ E unpack_agg(const Desc& d1, const Desc& d2) {
+        E e;
+        e.A = __uint_as_float((uint32_t)d1.lo);
+        e.m = __uint_as_float((uint32_t)(d1.lo >> 32));
+        e.s = __uint_as_float((uint32_t)d2.lo);
+        e.p = SIGNED ? ((uint32_t)(d2.lo >> 32) & 1u) << 31 : 0u;
+        return e;
+    }
+    __device__ static __forceinline__ Desc pack_value(const Params& p, const E& e) {
+        Desc d;
+        d.lo = (unsigned long long)__float_as_uint(e.m) | ((unsigned long long)__float_as_uint(e.s) << 32);
+        d.hi = p.call_id;
+        return d;
+    }
+    __device__ static __forceinline__ E unpack_value(const Desc& d) {
+        E e;
+        e.A = neg_inf();
+        e.m = __uint_as_float((uint32_t)d.lo);
+        e.s = __uint_as_float((uint32_t)(d.lo >> 32));
+        e.p = 0u;
+        return e;
     }
 
     __device__ static __forceinline__ bool give_up(const Params& p, unsigned int& polls) {
@@ -1212,11 +1225,11 @@ struct Lookback {
             ++total_polls;
             d.lo = __shfl_sync(0xffffffffu, d.lo, 0);
             d.hi = __shfl_sync(0xffffffffu, d.hi, 0);
-            if (state_of(d) == kInc) break;
+            if (d.hi == p.call_id) break;
             if (__any_sync(0xffffffffu, *abort_flag || give_up(p, polls))) { failed = true; break; }
             __nanosleep(p.lb_sleep_ready);
         }
-        return unpack(d);
+        return unpack_value(d);
     }
 
     // The carry server (all warps of the grid's last CTA).  `ring` is kSrvRing hand-over slots in its shared memory.
@@ -1244,19 +1257,23 @@ struct Lookback {
             E x0e = identity_elem<SIGNED>();
             if (starts_row) x0e = CE::row_start(p, row);
             // the batch's aggregates
-            Desc d;
-            d.lo = 0ull; d.hi = 0ull;
+            Desc d1, d2;
+            d1.lo = 0ull; d1.hi = 0ull;
+            d2 = d1;
             unsigned int polls = 0;
             bool ok = true;
             while (true) {
-                if (active && state_of(d) != kAgg) d = ld_desc(p.desc + T);
-                if (__all_sync(0xffffffffu, !active || state_of(d) == kAgg)) break;
+                if (active && !(d1.hi == p.call_id && d2.hi == p.call_id)) {
+                    d1 = ld_desc(p.desc + 2 * T);
+                    d2 = ld_desc(p.desc + 2 * T + 1);
+                }
+                if (__all_sync(0xffffffffu, !active || (d1.hi == p.call_id && d2.hi == p.call_id))) break;
                 if (__any_sync(0xffffffffu, *(volatile int*)&ring->abort || give_up(p, polls))) { ok = false; break; }
                 __nanosleep(p.lb_sleep_idle);
             }
             E part = identity_elem<SIGNED>();
             if (ok) {
-                if (active) part = unpack(d);
+                if (active) part = unpack_agg(d1, d2);
                 if (starts_row) part = compose(x0e, part);  // a value (A = -inf): forgets what came before the row
             }
             E wex, total;
@@ -1296,9 +1313,7 @@ struct Lookback {
             if (active) {
                 E ent = starts_row ? x0e : compose(cin, wex);
                 renormalise(ent);
-                ent.A = neg_inf();
-                ent.p = 0u;
-                st_desc(p.edesc + T, pack(ent, kInc));
+                st_desc(p.edesc + T, pack_value(p, ent));
             }
         }
     }
