@@ -417,6 +417,31 @@ def test_lookback_carry_server_batches(hs, oracle, rows, n, kind):
         run_log(hs, oracle, w.tensors, path=hs.PATH_LOOKBACK, what=f"{rows} x {n} {kind}")
 
 
+@pytest.mark.parametrize("path", ["batched", "lookback"])
+def test_workspace_needs_no_initialisation(hs, oracle, path):
+    """The workspace may hold anything: random bytes, or what a call on another problem left there.  Every word a
+    kernel reads from it (row tickets, hand-over words, the tiles' aggregates and entering values) counts only if it
+    carries this call's id."""
+    hs.set_path(getattr(hs, "PATH_" + path.upper()))
+    shapes = [(3, 7168 * 9 + 100), (2, 7168 * 40)] if path == "lookback" else [(2500, 2048), (9000, 600)]
+    nbytes = max(hs.workspace_bytes(r, n) for r, n in shapes)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    g = torch.Generator(device="cuda")
+    g.manual_seed(1234)
+    for fill in ("random", "ones", "previous call", "previous call"):
+        if fill == "random":
+            ws.copy_(torch.randint(0, 256, (nbytes,), dtype=torch.uint8, device="cuda", generator=g))
+        elif fill == "ones":
+            ws.fill_(0xFF)
+        for rows, n in shapes:  # (the second shape runs on what the first one left, and the next round on both)
+            w = workloads.make(3 if path == "lookback" else 2, rows=rows, n=n, seed=rows)
+            t = w.tensors
+            out = hs.scan_log(to_dev(t["log_a"]), to_dev(t["log_b"]), to_dev(t["log_x0"]), workspace=ws)
+            hs.check(ws)
+            ref, _ = oracle.scan_log(t["log_a"], t["log_b"], t["log_x0"])
+            assert_log_close(to_f64(out), ref, tol_positive(t["log_a"].astype(np.float64), ref), f"{fill}, {rows} x {n}")
+
+
 def test_lookback_several_rows_several_groups(hs, oracle):
     """Single-pass path with a few rows, each several rounds of tiles long, plus a ragged last tile: the carry
     crosses tiles, batches of tiles and the row starts inside a launch."""
