@@ -1408,14 +1408,20 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
     const uint32_t agg_bar = smem_u32(&xc->agg_ready[0]), carry_bar = smem_u32(&xc->carry_ready[0]);
     const uint32_t total_bar = smem_u32(&xc->total_ready[0]);
 
-    if (threadIdx.x == 0) {
-        xc->abort = 0;
-        for (int b = 0; b < kLbRing; ++b) {
-            mbar_init(agg_bar + 8 * b, W);
-            mbar_init(total_bar + 8 * b, 1);
-            mbar_init(carry_bar + 8 * b, 1);
+    // (every compute warp initialises its own mbarriers, thread 0 those of the exchange: one thread initialising
+    // all of them takes more than a microsecond, which a short launch feels)
+    if (lane == 0) {
+        if (warp < W) {
+            for (int i = 0; i < kLbMaxStages; ++i) mbar_init(warp_bars + 8 * (warp * kLbMaxStages + i), 1);
         }
-        for (int i = 0; i < W * kLbMaxStages; ++i) mbar_init(warp_bars + 8 * i, 1);
+        if (warp == 0) {
+            xc->abort = 0;
+            for (int b = 0; b < kLbRing; ++b) {
+                mbar_init(agg_bar + 8 * b, W);
+                mbar_init(total_bar + 8 * b, 1);
+                mbar_init(carry_bar + 8 * b, 1);
+            }
+        }
         fence_mbar_init();
     }
     // Programmatic dependent launch, as in the batched kernel: when the host launches the single-tile form with
