@@ -860,26 +860,6 @@ struct Run {
         bad = false;
     }
 
-    // The K parity masks of the run as 16 bits (K == 16), P[t] at bit 16 + t, and back; with adopt() the
-    // look-back kernel carries A_t and the parities of a kLinear run from its first phase to its second
-    // instead of taking the logarithms of a_t twice.
-    __device__ __forceinline__ uint32_t parity_bits() const {
-        uint32_t bits = 0u;
-#pragma unroll
-        for (int t = 0; t < K; ++t)
-            bits = (bits >> 1) | (MODE == kLinear ? (__float_as_uint(Pf[t]) & kSignBit) : SIGNED ? P[t] : 0u);
-        return bits;
-    }
-    __device__ __forceinline__ void adopt(const float* a_parked, uint32_t bits) {
-#pragma unroll
-        for (int t = 0; t < K; ++t) {
-            A[t] = a_parked[t];
-            if (MODE == kLinear) Pf[t] = __uint_as_float(0x3f800000u | ((bits << (K - 1 - t)) & kSignBit));
-            else if (SIGNED) P[t] = (bits << (K - 1 - t)) & kSignBit;
-        }
-        bad = false;
-    }
-
     // Apply the value entering the run and produce the outputs, in two steps so that a caller can store the
     // outputs piece by piece instead of holding all K of them:
     //   prepare() : the run's common factors, and whether the fast form can be trusted -- it cannot when an
@@ -890,6 +870,7 @@ struct Run {
     struct Applied {
         float M, C, w;
         bool ok;
+        float hM;  // (outputs<.., G = true> only) exp(M / 2), set by the caller
     };
     __device__ __forceinline__ Applied prepare(const E& entering) const {
         const float Mc = entering.m, Sc = entering.s;  // Mc is finite (>= kEmpty); r may be -inf
@@ -901,9 +882,12 @@ struct Run {
         a.w = (d >= 0.0f) ? ed : 1.0f;
         const float S1 = fmaf(s[0], a.w, a.C);
         a.ok = (fabsf(S1) >= 8.67361738e-19f /* 2^-60 */) || (Sc == 0.0f && r == neg_inf());
+        a.hM = 0.0f;
         return a;
     }
-    template <int T0, int N>
+    // G (kLinear, look-back kernel): A[t] holds g_t = +-exp(A_t / 2), the sign that of the product a_1..a_t, instead of
+    // A_t, and x_t = (g_t h)|g_t h| S_t with h = exp(M / 2): no transcendental and no sign factor in this phase.
+    template <int T0, int N, bool G = false>
     __device__ __forceinline__ void outputs(const Applied& a, float* out_mag, uint32_t* out_sign) const {
         static_assert(T0 % 2 == 0 && N % 2 == 0, "outputs are produced in pairs");
         const float2 w2 = pk(a.w), C2 = pk(a.C);
@@ -911,7 +895,12 @@ struct Run {
         for (int i = 0; i < N; i += 2) {
             const int t = T0 + i;
             const float2 S = fma2(pk(s[t], s[t + 1]), w2, C2);
-            if (MODE == kLinear) {
+            if (MODE == kLinear && G) {
+                const float2 gh = mul2(pk(A[t], A[t + 1]), pk(a.hM));
+                const float2 x = mul2(gh, S);
+                out_mag[i] = x.x * fabsf(gh.x);
+                out_mag[i + 1] = x.y * fabsf(gh.y);
+            } else if (MODE == kLinear) {
                 // exp(A_t + M) as the square of exp((A_t + M) / 2): the exponent range of fp32 twice over
                 const float2 arg = fma2(pk(A[t], A[t + 1]), pk(0.5f), pk(a.M * (0.5f * kLog2e)));  // (A_t: binary logarithms)
                 const float2 h = pk(ex2(arg.x), ex2(arg.y));

@@ -263,30 +263,31 @@ struct ChunkEngine {
 
     // The outputs of a run whose fast form holds, into the output buffer (and the signs to global memory): unit
     // by unit, so that no more than one unit's worth of outputs is live at a time.
-    template <bool PLAIN, int J = 0>
+    template <bool PLAIN, int J = 0, bool G = false>
     __device__ static __forceinline__ void emit_units(const R_& run, const typename R_::Applied& ap, uint32_t sm_out,
                                                       const Offsets& off) {
         if constexpr (J < OUT_UNITS) {
             constexpr int PER = Storage<TOut>::kPerUnit;
             float o[PER];
             uint32_t sg[MODE == kLogSigned ? PER : 1];
-            run.template outputs<J * PER, PER>(ap, o, sg);
+            run.template outputs<J * PER, PER, G>(ap, o, sg);
             sts128(sm_out + off.out[J], Storage<TOut>::pack_signed(o, sg));
-            emit_units<PLAIN, J + 1>(run, ap, sm_out, off);
+            emit_units<PLAIN, J + 1, G>(run, ap, sm_out, off);
         }
     }
-    template <bool PLAIN>
+    // (G: the run holds g_t instead of A_t, see Run::outputs)
+    template <bool PLAIN, bool G = false>
     __device__ static __forceinline__ void emit_outputs(const Params& p, const R_& run, const typename R_::Applied& ap,
                                                         uint32_t sm_out, const Offsets& off, const Wide& wd, long long idx0,
                                                         long long left) {
         if (SIGN_TENSORS || (PLAIN && wd.on)) {
             float out_mag[K];
             uint32_t out_sign[MODE == kLogSigned ? K : 1];
-            run.template outputs<0, K>(ap, out_mag, out_sign);
+            run.template outputs<0, K, G>(ap, out_mag, out_sign);
             write_outputs<PLAIN>(sm_out, off, wd, out_mag, out_sign);
             if (SIGN_TENSORS) store_signs(p.sign_x, idx0, left, p.sign_vec_ok != 0, out_sign);
         } else {
-            emit_units<PLAIN>(run, ap, sm_out, off);
+            emit_units<PLAIN, 0, G>(run, ap, sm_out, off);
         }
     }
 
@@ -1340,7 +1341,6 @@ struct LanePark {
     float r;              // reference of the lane's run
     Elem<SIGNED> excl;    // parts of the chunk before the lane's run
     bool slow;            // the chunk took the tracked form in phase 1 (warp-uniform)
-    uint32_t par;         // kLinear: parity masks of the lane's run (Run::parity_bits)
 };
 
 // One input stage of a compute warp: [a-tensor chunk][b-tensor chunk][park].  The partial sums
@@ -1519,7 +1519,7 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
     auto st_park = [&](int st) { return wb + st * ST::BYTES + ST::PARK_OFF; };
     LanePark<SIGNED> lp[4];  // lp[d]: the tile that went through phase 1 d iterations ago
 #pragma unroll
-    for (int d = 0; d < 4; ++d) { lp[d].r = neg_inf(); lp[d].excl = identity_elem<SIGNED>(); lp[d].slow = false; lp[d].par = 0u; }
+    for (int d = 0; d < 4; ++d) { lp[d].r = neg_inf(); lp[d].excl = identity_elem<SIGNED>(); lp[d].slow = false; }
     const uint32_t bars = warp_bars + warp * (8 * kLbMaxStages);
 
     // TMA helpers (same box geometry as WarpPipe, buffers laid out per stage here)
@@ -1619,6 +1619,14 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                 E total;
                 const typename CE::Wide wd = CE::wide_of(p, row, PLAIN);
                 CE::template phase1<PLAIN>(p, st_a(st), st_b(st), off, lm, lane, row, col0, colbase + CHUNK > p.n, wd, pd, total);
+                if (MODE == kLinear && !pd.slow) {
+                    // phase 2 gets g_t = +-exp(A_t / 2) instead of A_t and the parities (see Run::outputs); where that
+                    // would leave fp32's range, the chunk keeps its inputs and phase 2 takes the tracked form
+                    float amx = 0.0f;
+#pragma unroll
+                    for (int t = 0; t < K; t += 2) amx = max3(amx, fabsf(pd.run.A[t]), fabsf(pd.run.A[t + 1]));
+                    if (__any_sync(0xffffffffu, !(amx <= 240.0f))) pd.slow = true;
+                }
                 if (!pd.slow) {  // park the partial sums (a slow chunk keeps its inputs instead)
                     const uint32_t pb = st_park(st);
                     // (wide staging: a lane's inputs reach into the unit after its own, where its neighbour parks;
@@ -1627,12 +1635,22 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
 #pragma unroll
                     for (int jx = 0; jx < K / 4; ++jx) sts128(pb + park_off[jx], Storage<float>::pack(pd.run.s + 4 * jx));
                     if (MODE == kLinear) {
-                        // ... and A_t over the a-tensor chunk, the parities in a register: phase 2 would
-                        // otherwise take the logarithm of every a_t a second time
+                        // ... and g_t over the a-tensor chunk: phase 2 would otherwise take the logarithm of every
+                        // a_t a second time
                         const uint32_t ab = st_a(st);
 #pragma unroll
-                        for (int jx = 0; jx < K / 4; ++jx) sts128(ab + park_off[jx], Storage<float>::pack(pd.run.A + 4 * jx));
-                        lp[0].par = pd.run.parity_bits();
+                        for (int jx = 0; jx < K / 4; ++jx) {
+                            float g[4];
+#pragma unroll
+                            for (int q = 0; q < 4; q += 2) {
+                                const int t = 4 * jx + q;
+                                const float2 h = mul2(pk(pd.run.A[t], pd.run.A[t + 1]), pk(0.5f));
+                                const float2 gg = mul2(pk(ex2(h.x), ex2(h.y)), pk(pd.run.Pf[t], pd.run.Pf[t + 1]));
+                                g[q] = gg.x;
+                                g[q + 1] = gg.y;
+                            }
+                            sts128(ab + park_off[jx], Storage<float>::pack(g));
+                        }
                     }
                 }
                 lp[0].r = pd.run.r;
@@ -1680,8 +1698,8 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                     uint32_t sa[MODE == kLogSigned ? K : 1];
                     if (MODE == kLinear) {
 #pragma unroll
-                        for (int jx = 0; jx < K / 4; ++jx) Storage<float>::unpack(lds128(sm_a + park_off[jx]), va + 4 * jx);
-                        run.adopt(va, mine.par);
+                        for (int jx = 0; jx < K / 4; ++jx) Storage<float>::unpack(lds128(sm_a + park_off[jx]), run.A + 4 * jx);
+                        run.bad = false;
                     } else {
                         if (PLAIN) Shifted<TIn, K>::read_signed(sm_a, off.in, wd.phi_a, va, sa);
                         else R_::load_a_signed(sm_a, off.in, va, sa);
@@ -1699,9 +1717,10 @@ lookback_scan_kernel(const Params p, const __grid_constant__ CUtensorMap tm_a, c
                     run.r = mine.r;
 #pragma unroll
                     for (int jx = 0; jx < K / 4; ++jx) Storage<float>::unpack(lds128(pb + park_off[jx]), run.s + 4 * jx);
-                    const typename R_::Applied ap = run.prepare(entering);
+                    typename R_::Applied ap = run.prepare(entering);
                     ok = __all_sync(0xffffffffu, ap.ok);  // also: every lane has read its parked sums
-                    if (ok) CE::template emit_outputs<PLAIN>(p, run, ap, pb, off, wd, row * p.n + col0, left);
+                    if (MODE == kLinear) ap.hM = ex2(ap.M * (0.5f * kLog2e));
+                    if (ok) CE::template emit_outputs<PLAIN, MODE == kLinear>(p, run, ap, pb, off, wd, row * p.n + col0, left);
                 }
                 if (!ok) {
                     // where the lane's inputs are now: as staged (shifted) when the chunk kept them, at the lane's

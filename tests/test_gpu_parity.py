@@ -257,6 +257,42 @@ def test_zeros_resets_and_wide_range(hs, oracle, path):
 
 
 @pytest.mark.parametrize("path", ["batched", "lookback"])
+def test_linear_products_that_leave_fp32_inside_a_run(hs, oracle, path):
+    """scan_linear with stretches of tiny and of huge |a_t|: the product of a lane's 16 factors leaves fp32's range
+    (below 2^-240 or above 2^240) although every x_t stays representable.  The look-back kernel hands exp(A_t / 2)
+    from its first phase to its second and must fall back to the tracked form on such chunks; the row-batched kernel
+    keeps A_t itself.  Tiny stretches forget the past (x_t ~ b_t); huge factors are followed by tiny ones."""
+    rng = np.random.default_rng(21)
+    rows, n = 3, 7168 * 3 + 100
+    a = rng.uniform(0.5, 1.0, (rows, n)).astype(np.float32) * rng.choice([-1, 1], (rows, n)).astype(np.float32)
+    b = rng.normal(size=(rows, n)).astype(np.float32)
+    x0 = rng.normal(size=rows).astype(np.float32)
+    a[0, 1000:1400] = rng.choice([-1, 1], 400).astype(np.float32) * np.float32(3e-6)     # 2^-18 each: 2^-290 per run
+    a[1, 5000:9000] = rng.choice([-1, 1], 4000).astype(np.float32) * np.float32(1e-7)
+    a[2, 300:340:2] = np.float32(2e5)                                                    # up ...
+    a[2, 301:341:2] = np.float32(-5e-6)                                                  # ... and down again, pairwise
+    a[2, 12000:12020] = np.float32(4e4)                                                  # 20 factors of 2^15: 2^300,
+    b[2, 12000:12020] = 0.0
+    a[2, 12020:12040] = np.float32(2.5e-5)                                               # taken back by 20 of 2^-15
+    b[2, 12020:12040] = 0.0
+    b[2, 10000:12000] = 0.0
+    a[2, 10000:12000] = np.float32(0.93)                    # x ~ 1e-63 when the climb begins (below fp32, not below the carry)
+    hs.set_path(getattr(hs, "PATH_" + path.upper()))
+    ws = hs.new_workspace(rows, n, "cuda")
+    x = hs.scan_linear(to_dev(a), to_dev(b), to_dev(x0), workspace=ws)
+    hs.check(ws)
+    ref = oracle.scan_linear(a, b, x0)
+    got = to_f64(x)
+    assert np.abs(ref).max() < 1e38 and np.isfinite(got).all()
+    assert np.abs(ref[2, 12019]) > 1e20                     # the climb really happened
+    assert_signed_close(got, ref, f"linear wide range/{path}")
+    np.testing.assert_allclose(got[2, 12010:12020], ref[2, 12010:12020], rtol=1e-3)
+    # where the past is forgotten the result is b_t to fp32 accuracy, whatever the scale of the row
+    np.testing.assert_allclose(got[0, 1001:1400], ref[0, 1001:1400], rtol=2e-5, atol=1e-6)
+    np.testing.assert_allclose(got[1, 5001:9000], ref[1, 5001:9000], rtol=2e-5, atol=1e-6)
+
+
+@pytest.mark.parametrize("path", ["batched", "lookback"])
 def test_linear_zeros_and_cancellation(hs, oracle, path):
     rng = np.random.default_rng(12)
     rows, n = 4, 2500
